@@ -1,0 +1,407 @@
+// AudioKV eviction pass: CPU oracle.
+//
+// TEST INFRASTRUCTURE ONLY. This file is the plain, slow, fp64 statement of what
+// the eviction pass computes. Only the tests, the smoke check and the benchmark's
+// CPU-baseline leg may call it; the CUDA library never does, and the two share no
+// code. Every function follows one passage of the AudioKV paper (cited at the
+// function) in the paper's own order and notation; nothing is blocked, fused or
+// reordered. Inputs in bf16 are decoded exactly to double.
+//
+// Parallelism: OpenMP over (layer, KV head) only; each head is computed serially.
+//
+// Pins (see tests/test_oracle_*.py): direct O(n^2) DFT, numpy.fft, closed forms,
+// invariants and brute force. Parity unpinned by the paper: the width T of the
+// cosine transition band and the default values of rho and alpha (the paper gives
+// the shape "cosine" and the ranges only); the conventions are documented at
+// akvo_sss below.
+
+#include <algorithm>
+#include <cmath>
+#include <complex>
+#include <cstdint>
+#include <cstring>
+#include <numeric>
+#include <vector>
+
+namespace {
+
+constexpr int DT_F32 = 0;
+constexpr int DT_BF16 = 1;
+
+inline double load_elem(const void* base, int dtype, int64_t idx) {
+  if (dtype == DT_F32) {
+    float f;
+    std::memcpy(&f, static_cast<const char*>(base) + 4 * idx, 4);
+    return static_cast<double>(f);
+  }
+  uint16_t h;
+  std::memcpy(&h, static_cast<const char*>(base) + 2 * idx, 2);
+  uint32_t u = static_cast<uint32_t>(h) << 16;  // bf16 is the top half of an fp32
+  float f;
+  std::memcpy(&f, &u, 4);
+  return static_cast<double>(f);
+}
+
+inline int elem_size(int dtype) { return dtype == DT_F32 ? 4 : 2; }
+
+using cplx = std::complex<double>;
+
+// e^{-2 pi i t / n} for t in [0, n), evaluated in long double from the reduced
+// index so that the table is exact to double rounding.
+std::vector<cplx> unit_roots(int n) {
+  std::vector<cplx> w(n);
+  const long double two_pi = 6.283185307179586476925286766559005768L;
+  for (int t = 0; t < n; ++t) {
+    long double a = two_pi * static_cast<long double>(t) / static_cast<long double>(n);
+    w[t] = cplx(static_cast<double>(cosl(a)), static_cast<double>(-sinl(a)));
+  }
+  return w;
+}
+
+int smallest_factor(int n) {
+  for (int p = 2; static_cast<int64_t>(p) * p <= n; ++p)
+    if (n % p == 0) return p;
+  return n;
+}
+
+// Decimation-in-time DFT of any length: split by the smallest prime factor p
+// into p interleaved sub-sequences, transform each, and combine with the
+// definition of the DFT. A prime length is the O(n^2) definition itself.
+// in: n values at stride `stride`; out: n contiguous values.
+// roots: table for the top-level length N; this level uses roots[t * (N / n)].
+void dft_any(const cplx* in, int stride, int n, cplx* out, const std::vector<cplx>& roots, int N) {
+  const int step = N / n;
+  if (n == 1) {
+    out[0] = in[0];
+    return;
+  }
+  const int p = smallest_factor(n);
+  if (p == n) {
+    for (int k = 0; k < n; ++k) {
+      cplx acc(0.0, 0.0);
+      for (int j = 0; j < n; ++j) {
+        int64_t t = (static_cast<int64_t>(j) * k) % n;
+        acc += in[static_cast<int64_t>(j) * stride] * roots[t * step];
+      }
+      out[k] = acc;
+    }
+    return;
+  }
+  const int m = n / p;
+  std::vector<cplx> sub(static_cast<size_t>(n));
+  for (int c = 0; c < p; ++c)
+    dft_any(in + static_cast<int64_t>(c) * stride, stride * p, m, sub.data() + static_cast<size_t>(c) * m, roots, N);
+  for (int k = 0; k < n; ++k) {
+    cplx acc(0.0, 0.0);
+    for (int c = 0; c < p; ++c) {
+      int64_t t = (static_cast<int64_t>(c) * k) % n;
+      acc += sub[static_cast<size_t>(c) * m + (k % m)] * roots[t * step];
+    }
+    out[k] = acc;
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+// ---------------------------------------------------------------------------
+// Step 1: token importance. Section 3.3 describes the per-head importance
+// sequence as the attention a head's recent ("decoding window") queries give to
+// past tokens, aggregated over the window; the SnapKV lineage the paper builds on
+// fixes the rest. For KV head h, window row i (token position P+i, P = L-W) and
+// group member g (query head h*G+g):
+//     z_j = scale * <Q[i, hG+g, :], K[j, h, :]>   for j in [0, P+i]   (causal)
+//     p_j = exp(z_j - max z) / sum_j exp(z_j - max z)
+//     s_h[j] += p_j                                for j in [0, P)
+// i.e. the SUM over window rows and group members (the paper says "averaged";
+// the two differ by the constant 1/(W*G), to which every later step is
+// equivariant). Window keys (j >= P) take part in the softmax but get no score;
+// their total mass is returned separately so that row sums can be checked.
+//
+// q: [n_layers][W][Hq][d] by strides (elements), k: [n_layers][L][Hkv][d] by strides.
+// s: [n_layers][Hkv][P] double. window_mass: [n_layers][Hkv] double or NULL.
+int akvo_score(const void* q, const void* k, int dtype, int n_layers, int W, int Hq, int Hkv, int d, int L,
+               int64_t q_stride_layer, int64_t q_stride_tok, int64_t q_stride_head, int64_t k_stride_layer,
+               int64_t k_stride_tok, int64_t k_stride_head, double scale, double* s, double* window_mass) {
+  if (W < 1 || L <= W || Hkv < 1 || Hq % Hkv != 0 || d < 1) return -1;
+  const int P = L - W;
+  const int G = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+  for (int l = 0; l < n_layers; ++l) {
+    for (int h = 0; h < Hkv; ++h) {
+      std::vector<double> Kd(static_cast<size_t>(L) * d);
+      for (int j = 0; j < L; ++j)
+        for (int t = 0; t < d; ++t)
+          Kd[static_cast<size_t>(j) * d + t] =
+              load_elem(k, dtype, l * k_stride_layer + j * k_stride_tok + h * k_stride_head + t);
+      std::vector<double> z(L), qrow(d);
+      double* acc = s + (static_cast<size_t>(l) * Hkv + h) * P;
+      for (int j = 0; j < P; ++j) acc[j] = 0.0;
+      double wm = 0.0;
+      for (int i = 0; i < W; ++i) {
+        for (int g = 0; g < G; ++g) {
+          for (int t = 0; t < d; ++t)
+            qrow[t] = load_elem(q, dtype, l * q_stride_layer + i * q_stride_tok + (h * G + g) * q_stride_head + t);
+          const int nvis = P + i + 1;
+          double m = -INFINITY;
+          for (int j = 0; j < nvis; ++j) {
+            double dot = 0.0;
+            const double* kr = &Kd[static_cast<size_t>(j) * d];
+            for (int t = 0; t < d; ++t) dot += qrow[t] * kr[t];
+            z[j] = scale * dot;
+            m = std::max(m, z[j]);
+          }
+          double Z = 0.0;
+          for (int j = 0; j < nvis; ++j) Z += std::exp(z[j] - m);
+          for (int j = 0; j < P; ++j) acc[j] += std::exp(z[j] - m) / Z;
+          for (int j = P; j < nvis; ++j) wm += std::exp(z[j] - m) / Z;
+        }
+      }
+      if (window_mass) window_mass[static_cast<size_t>(l) * Hkv + h] = wm;
+    }
+  }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
+// One-sided DFT of a real sequence, F_k = sum_j x_j e^{-2 pi i jk/n}, k = 0..n/2
+// (Section 3.3, the RFFT equation). direct != 0: the O(n^2) sum as written;
+// otherwise the recursive prime-factor splitting above (same values, faster).
+int akvo_rfft(const double* x, int n, int direct, double* re, double* im) {
+  if (n < 1) return -1;
+  const int Kb = n / 2;
+  std::vector<cplx> roots = unit_roots(n);
+  if (direct) {
+    for (int k = 0; k <= Kb; ++k) {
+      cplx acc(0.0, 0.0);
+      for (int j = 0; j < n; ++j) acc += x[j] * roots[(static_cast<int64_t>(j) * k) % n];
+      re[k] = acc.real();
+      im[k] = acc.imag();
+    }
+    return 0;
+  }
+  std::vector<cplx> in(n), out(n);
+  for (int j = 0; j < n; ++j) in[j] = cplx(x[j], 0.0);
+  dft_any(in.data(), 1, n, out.data(), roots, n);
+  for (int k = 0; k <= Kb; ++k) {
+    re[k] = out[k].real();
+    im[k] = out[k].imag();
+  }
+  return 0;
+}
+
+// Inverse of the above to a real sequence of length n (Section 3.3, the IRFFT
+// equation, with the usual 1/n on the inverse):
+//   x_j = (1/n) [ F_0 + 2 sum_{1<=k<n/2} Re(F_k e^{+2 pi i jk/n}) + (n even) F_{n/2} (-1)^j ]
+// Imaginary parts of F_0 and (n even) F_{n/2} do not enter, as in any real inverse.
+int akvo_irfft(const double* re, const double* im, int n, int direct, double* x) {
+  if (n < 1) return -1;
+  const int Kb = n / 2;
+  std::vector<cplx> roots = unit_roots(n);
+  if (direct) {
+    for (int j = 0; j < n; ++j) {
+      double acc = re[0];
+      for (int k = 1; 2 * k < n; ++k) {
+        cplx w = std::conj(roots[(static_cast<int64_t>(j) * k) % n]);
+        acc += 2.0 * (re[k] * w.real() - im[k] * w.imag());
+      }
+      if (n % 2 == 0) acc += (j % 2 == 0) ? re[Kb] : -re[Kb];
+      x[j] = acc / n;
+    }
+    return 0;
+  }
+  // Full Hermitian spectrum, then x = conj(DFT(conj(F))) / n.
+  std::vector<cplx> full(n), out(n);
+  full[0] = cplx(re[0], 0.0);
+  for (int k = 1; 2 * k < n; ++k) {
+    full[k] = cplx(re[k], -im[k]);      // conj(F_k)
+    full[n - k] = cplx(re[k], im[k]);   // conj(F_{n-k}) = F_k
+  }
+  if (n % 2 == 0) full[Kb] = cplx(re[Kb], 0.0);
+  dft_any(full.data(), 1, n, out.data(), roots, n);
+  for (int j = 0; j < n; ++j) x[j] = out[j].real() / n;
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Step 2: Spectral Score Smoothing (Section 3.3, in the paper's order).
+//   F = RFFT(x);  m_k^2 = |F_k|^2;  E(k) = sum_{i<=k} m_i^2  (one-sided sum as
+//   written: DC included, interior bins not doubled);  k* = the smallest k with
+//   E(k) >= rho * E(n/2);  mask w_i = 1 for i <= k*;  F~ = F .* w;
+//   x~ = IRFFT(F~, n);  out = (1 - alpha) x + alpha x~.
+// Transition band: the paper asks for a short cosine-shaped band at the cut-off
+// without giving its width or placement. Reading used here: T bins after k*,
+//   w_i = (1 + cos(pi (i - k*) / (T + 1))) / 2   for k* < i <= k* + T,  0 beyond,
+// which keeps w_i = 1 for every i <= k* exactly as the mask equation states, makes
+// T = 0 the paper's binary mask, and keeps rho = 1 an identity.
+// force_kstar >= 0 replaces the computed k* (used by the tests' near-tie
+// protocol); the computed value is still reported through kstar_out.
+// margin_out: min over the two bins deciding k* of |E(k) - rho E(n/2)| / E(n/2)
+// (how close the decision was). energy_out: E(k) for k = 0..n/2, or NULL.
+int akvo_sss(const double* x, int n, double rho, double alpha, int T, int force_kstar, int direct, double* out,
+             int* kstar_out, double* margin_out, double* energy_out) {
+  if (n < 1 || T < 0) return -1;
+  const int Kb = n / 2;
+  std::vector<double> re(Kb + 1), im(Kb + 1), E(Kb + 1);
+  akvo_rfft(x, n, direct, re.data(), im.data());
+  double run = 0.0;
+  for (int k = 0; k <= Kb; ++k) {
+    run += re[k] * re[k] + im[k] * im[k];
+    E[k] = run;
+  }
+  const double thr = rho * E[Kb];
+  int kstar = Kb;
+  for (int k = 0; k <= Kb; ++k) {
+    if (E[k] >= thr) {
+      kstar = k;
+      break;
+    }
+  }
+  if (kstar_out) *kstar_out = kstar;
+  if (margin_out) {
+    double tot = E[Kb] > 0.0 ? E[Kb] : 1.0;
+    double mg = std::fabs(E[kstar] - thr) / tot;
+    if (kstar > 0) mg = std::min(mg, std::fabs(E[kstar - 1] - thr) / tot);
+    *margin_out = mg;
+  }
+  if (energy_out) std::copy(E.begin(), E.end(), energy_out);
+  if (force_kstar >= 0) kstar = std::min(force_kstar, Kb);
+  const double pi = 3.14159265358979323846;
+  for (int i = 0; i <= Kb; ++i) {
+    double w;
+    if (i <= kstar)
+      w = 1.0;
+    else if (i <= kstar + T)
+      w = 0.5 * (1.0 + std::cos(pi * (i - kstar) / (T + 1)));
+    else
+      w = 0.0;
+    re[i] *= w;
+    im[i] *= w;
+  }
+  std::vector<double> xt(n);
+  akvo_irfft(re.data(), im.data(), n, direct, xt.data());
+  for (int j = 0; j < n; ++j) out[j] = (1.0 - alpha) * x[j] + alpha * xt[j];
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Step 3: head-wise budgets (Section 3.1, the allocation equation
+//   b = w + r + B_score * S / sum S,
+// of which Section 3.2's floor(B * S_hit / sum S_hit) is the case w = r = 0).
+// The sums run over all N = layers * heads of one request. Integer reading, so
+// that the budgets are exact and add up to B:
+//   S_q = round-half-up(S * 2^24);  floor f = w + r per head;  R = B - N f is
+//   B_score;  room per head cap = L - f.  Shares t_h = floor(R S_q[h] / sum S_q);
+//   a head whose share exceeds cap is fixed at cap and leaves the pool (its cap
+//   leaves R), and the shares are recomputed; what the floors leave over goes one
+//   token each by descending remainder (R S_q[h] mod sum), ties by ascending flat
+//   head index, skipping heads that are full.  All-zero scores split R evenly
+//   (the first R mod |pool| heads by index get one more).  b = f + t.
+// Returns 0, or -1 when N f > B, B > N L, f > L, or a score is negative, NaN or > 128.
+int akvo_allocate(const float* S, int N, int64_t B, int w, int r, int L, int32_t* b) {
+  if (N < 1 || w < 0 || r < 0 || L < 1) return -1;
+  const int64_t f = static_cast<int64_t>(w) + r;
+  if (f > L) return -1;
+  if (N * f > B || B > static_cast<int64_t>(N) * L) return -1;
+  std::vector<int64_t> Sq(N), t(N, 0);
+  for (int h = 0; h < N; ++h) {
+    double v = static_cast<double>(S[h]);
+    if (!(v >= 0.0) || v > 128.0) return -1;
+    Sq[h] = static_cast<int64_t>(std::floor(v * 16777216.0 + 0.5));
+  }
+  const int64_t cap = L - f;
+  int64_t R = B - N * f;
+  std::vector<char> active(N, 1);
+  while (true) {
+    int64_t sum = 0;
+    int nA = 0;
+    for (int h = 0; h < N; ++h)
+      if (active[h]) {
+        sum += Sq[h];
+        ++nA;
+      }
+    if (nA == 0) break;
+    if (sum == 0) {
+      int64_t base = R / nA, extra = R % nA;
+      int rank = 0;
+      for (int h = 0; h < N; ++h)
+        if (active[h]) {
+          t[h] = base + (rank < extra ? 1 : 0);
+          ++rank;
+        }
+      break;
+    }
+    bool over = false;
+    std::vector<int64_t> share(N, 0), rem(N, 0);
+    for (int h = 0; h < N; ++h)
+      if (active[h]) {
+        const __int128 prod = static_cast<__int128>(R) * Sq[h];
+        share[h] = static_cast<int64_t>(prod / sum);
+        rem[h] = static_cast<int64_t>(prod % sum);
+        if (share[h] > cap) over = true;
+      }
+    if (over) {
+      for (int h = 0; h < N; ++h)
+        if (active[h] && share[h] > cap) {
+          t[h] = cap;
+          active[h] = 0;
+          R -= cap;
+        }
+      continue;
+    }
+    int64_t given = 0;
+    std::vector<int> order;
+    for (int h = 0; h < N; ++h)
+      if (active[h]) {
+        t[h] = share[h];
+        given += share[h];
+        order.push_back(h);
+      }
+    int64_t left = R - given;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int c) { return rem[a] > rem[c]; });
+    while (left > 0) {
+      bool any = false;
+      for (int h : order) {
+        if (left == 0) break;
+        if (t[h] < cap) {
+          ++t[h];
+          --left;
+          any = true;
+        }
+      }
+      if (!any) return -2;  // cannot happen while R <= |pool| * cap
+    }
+    break;
+  }
+  for (int h = 0; h < N; ++h) b[h] = static_cast<int32_t>(f + t[h]);
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Step 4a: per-head top-k (the paper's Top-K selection on the smoothed scores).
+// Order: score descending, index ascending among equals; the k chosen indices are
+// returned in ascending order.
+int akvo_select(const double* s_hat, int P, int k, int32_t* idx_out) {
+  if (k < 0 || k > P) return -1;
+  std::vector<int32_t> order(P);
+  std::iota(order.begin(), order.end(), 0);
+  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t c) { return s_hat[a] > s_hat[c]; });
+  std::vector<int32_t> kept(order.begin(), order.begin() + k);
+  std::sort(kept.begin(), kept.end());
+  std::copy(kept.begin(), kept.end(), idx_out);
+  return 0;
+}
+
+// Step 4b: eviction keeps only the selected rows. Copies row idx[i] of one head's
+// cache ([tokens][d] at stride_tok elements) to row i of a packed [n_idx][d] output.
+int akvo_gather(const void* src, int dtype, int d, int64_t stride_tok, const int32_t* idx, int n_idx, void* dst) {
+  const int es = elem_size(dtype);
+  for (int i = 0; i < n_idx; ++i)
+    std::memcpy(static_cast<char*>(dst) + static_cast<size_t>(i) * d * es,
+                static_cast<const char*>(src) + static_cast<size_t>(idx[i]) * stride_tok * es,
+                static_cast<size_t>(d) * es);
+  return 0;
+}
+
+}  // extern "C"

@@ -1,0 +1,177 @@
+"""Seeded synthetic workloads for the AudioKV eviction pass.
+
+This module only draws inputs. It holds none of the method's arithmetic and is
+the one piece of code that both the CUDA parity tests and the CPU oracle's tests
+use, so that the two sides see identical bytes.
+
+The paper evaluates on speech corpora with Qwen2.5-Omni, Qwen3-Omni and Gemma-3n
+checkpoints. Neither is available offline, so the inputs here reproduce the
+shapes of those models' attention stacks and the structure the paper argues from:
+audio tokens vary slowly along time (an AR(1) process along the token axis), text
+tokens are independent, the first tokens may be attention sinks with a large key
+norm, and only a few heads are strongly audio-critical (Beta(0.5, 2) scores).
+
+Layouts (elements, last dimension contiguous):
+  K, V : [n_layers][n_kv_heads][sum_L][head_dim]  -- requests concatenated along tokens
+  Q    : [n_req][n_layers][W][n_q_heads][head_dim] -- the last W query rows of each request
+  S    : [n_req][n_layers][n_kv_heads] float32     -- audio-criticality score per KV head
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+from scipy.signal import lfilter
+
+
+@dataclasses.dataclass
+class WorkloadSpec:
+    name: str
+    dtype: str                    # "f32" | "bf16"
+    n_layers: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    seq_lens: List[int]           # one entry per request
+    audio_frac: List[float]       # fraction of each request's tokens that are audio
+    n_sink: int                   # leading tokens whose K rows are scaled by 8
+    window: int = 32
+    keep: float = 0.4
+    ar_rho: float = 0.95
+    ar_rho_range: Optional[Sequence[float]] = None   # per-(layer, head) rho ~ U(lo, hi) when set
+    head_score_dist: str = "beta"  # "beta" -> Beta(0.5, 2); "uniform" -> U(0, 1)
+    rho: float = 0.5              # SSS cut-off ratio
+    alpha: float = 0.5            # SSS mixing coefficient
+    transition_bins: int = 4      # SSS cosine band width T
+
+
+def config(i: int, seed: int = 0) -> WorkloadSpec:
+    """The five benchmark configurations (index as in the benchmark's list)."""
+    if i == 0:
+        return WorkloadSpec("c1_tiny_f32", "f32", 1, 8, 2, 64, [1024], [768 / 1024], 1, head_score_dist="uniform")
+    if i == 1:
+        return WorkloadSpec("c2_qwen25omni7b_L8k", "bf16", 28, 28, 4, 128, [8192], [7500 / 8192], 0)
+    if i == 2:
+        return WorkloadSpec("c3_qwen25omni7b_L32k", "bf16", 28, 28, 4, 128, [32768], [0.9], 0,
+                            ar_rho_range=(0.85, 0.99))
+    if i == 3:
+        return WorkloadSpec("c4_qwen3omni30b_L16k", "bf16", 48, 32, 4, 128, [16384], [0.85], 4)
+    if i == 4:
+        rng = np.random.Generator(np.random.Philox(key=[seed, 0xC5]))
+        lens = [int(math.floor(math.exp(rng.uniform(math.log(2048), math.log(32768))))) for _ in range(8)]
+        fr = [float(rng.uniform(0.80, 0.95)) for _ in range(8)]
+        return WorkloadSpec("c5_gemma3n_e4b_ragged8", "bf16", 35, 8, 2, 256, lens, fr, 0)
+    raise ValueError(i)
+
+
+def kept_total(spec: WorkloadSpec, L: int) -> int:
+    """Total rows one request keeps over all heads at the spec's retention ratio: floor(c * N * L)."""
+    n = spec.n_layers * spec.n_kv_heads
+    return int(math.floor(spec.keep * n * L))
+
+
+def base_per_head(spec: WorkloadSpec, L: int) -> int:
+    """Uniform base allocation r used by the benchmark workloads: a tenth of a uniform head's non-window share."""
+    return max(0, int(math.floor(0.1 * (math.floor(spec.keep * L) - spec.window))))
+
+
+@dataclasses.dataclass
+class Workload:
+    spec: WorkloadSpec
+    q: np.ndarray                 # raw storage: float32, or uint16 holding bf16 bits
+    k: np.ndarray
+    v: np.ndarray
+    head_scores: np.ndarray       # float32 [n_req][n_layers][n_kv_heads]
+    cu_seqlen: np.ndarray         # int64 [n_req + 1] token offsets of the requests
+    total_budget: np.ndarray      # int64 [n_req]
+    base: int                     # r (tokens per head)
+
+    @property
+    def n_req(self) -> int:
+        return len(self.spec.seq_lens)
+
+    @property
+    def sum_L(self) -> int:
+        return int(self.cu_seqlen[-1])
+
+    def kv_strides(self):
+        """(layer, token, head) strides of K and V in elements."""
+        s = self.spec
+        return (s.n_kv_heads * self.sum_L * s.head_dim, s.head_dim, self.sum_L * s.head_dim)
+
+    def q_strides(self):
+        """(request, layer, token, head) strides of Q in elements."""
+        s = self.spec
+        per_tok = s.n_q_heads * s.head_dim
+        return (s.n_layers * s.window * per_tok, s.window * per_tok, per_tok, s.head_dim)
+
+    def torch_dtype(self):
+        return torch.float32 if self.spec.dtype == "f32" else torch.bfloat16
+
+    def as_torch(self, a: np.ndarray) -> torch.Tensor:
+        t = torch.from_numpy(a)
+        return t if self.spec.dtype == "f32" or a.dtype != np.uint16 else t.view(torch.bfloat16)
+
+
+def _store(x: np.ndarray, dtype: str) -> np.ndarray:
+    """Round once (nearest even) to the storage type; bf16 is returned as its uint16 bit pattern."""
+    if dtype == "f32":
+        return np.ascontiguousarray(x, dtype=np.float32)
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.uint16).numpy()
+
+
+def _ar1_inplace(x: np.ndarray, rho: float) -> None:
+    """x[t] <- rho x[t-1] + sqrt(1 - rho^2) x[t] along axis 0, x[0] kept: stationary, unit variance."""
+    if x.shape[0] < 2:
+        return
+    g = math.sqrt(1.0 - rho * rho)
+    drive = x * g
+    drive[0] = x[0]
+    x[...] = lfilter([1.0], [1.0, -rho], drive, axis=0)
+
+
+def generate(spec: WorkloadSpec, seed: int = 0, layers: Optional[int] = None) -> Workload:
+    """Draw one workload. `layers` truncates the stack (the first `layers` layers) for small parity cases;
+    budgets are then computed for the truncated stack."""
+    if layers is not None:
+        spec = dataclasses.replace(spec, n_layers=int(layers))
+    NL, Hq, Hkv, d, W = spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.window
+    lens = list(spec.seq_lens)
+    cu = np.zeros(len(lens) + 1, dtype=np.int64)
+    cu[1:] = np.cumsum(lens)
+    sumL = int(cu[-1])
+    G = Hq // Hkv
+    st = np.uint16 if spec.dtype == "bf16" else np.float32
+    k = np.zeros((NL, Hkv, sumL, d), dtype=st)
+    v = np.zeros((NL, Hkv, sumL, d), dtype=st)
+    q = np.zeros((len(lens), NL, W, Hq, d), dtype=st)
+    S = np.zeros((len(lens), NL, Hkv), dtype=np.float32)
+    for r, L in enumerate(lens):
+        n_audio = int(round(spec.audio_frac[r] * L))
+        rng_s = np.random.Generator(np.random.Philox(key=[seed, 1000 + r]))
+        if spec.head_score_dist == "uniform":
+            S[r] = rng_s.uniform(0.0, 1.0, size=(NL, Hkv)).astype(np.float32)
+        else:
+            S[r] = rng_s.beta(0.5, 2.0, size=(NL, Hkv)).astype(np.float32)
+        for l in range(NL):
+            rng = np.random.Generator(np.random.Philox(key=[seed, (r << 20) + l + 1]))
+            for h in range(Hkv):
+                rho = spec.ar_rho if spec.ar_rho_range is None else float(rng.uniform(*spec.ar_rho_range))
+                for dst, is_k in ((k, True), (v, False)):
+                    x = rng.standard_normal(size=(L, d), dtype=np.float32)
+                    _ar1_inplace(x[:n_audio], rho)
+                    if is_k and spec.n_sink:
+                        x[: spec.n_sink] *= 8.0
+                    dst[l, h, cu[r]:cu[r] + L] = _store(x, spec.dtype)
+                # window queries of this KV head's group; window tokens inside the audio segment continue an AR(1) chain
+                xq = rng.standard_normal(size=(W, G * d), dtype=np.float32)
+                n_aw = max(0, min(W, n_audio - (L - W)))
+                _ar1_inplace(xq[:n_aw], rho)
+                q[r, l, :, h * G:(h + 1) * G, :] = _store(xq, spec.dtype).reshape(W, G, d)
+    B = np.array([kept_total(spec, L) for L in lens], dtype=np.int64)
+    base = base_per_head(spec, min(lens))
+    return Workload(spec, q, k, v, S, cu, B, base)
