@@ -1,0 +1,187 @@
+/* audiokv.h -- C boundary of the B200 (sm_100a) AudioKV eviction pass.
+ *
+ * The pass runs once after prefill. For every request, layer and KV head it
+ *   1. scores each prefix token by the attention the last W queries give it
+ *      (Section 3.3: the per-head importance sequence over a decoding window),
+ *   2. smooths that sequence in the frequency domain (Section 3.3: Spectral Score
+ *      Smoothing, the RFFT / energy cut-off / mask / IRFFT / residual-mix equations),
+ *   3. turns per-head audio-criticality scores into integer budgets (Section 3.1,
+ *      b = w + r + B_score * S / sum S; Section 3.2's floor rule is the case w = r = 0),
+ *   4. keeps the top-scoring tokens of each head plus the window and copies their
+ *      K and V rows into a compacted cache (the paper's Top-K selection and eviction).
+ *
+ * Conventions
+ *   - Every data pointer is DEVICE memory owned by the caller unless marked "host".
+ *     The library allocates only inside audiokv_create and frees only in audiokv_destroy.
+ *   - Every compute call is asynchronous on the given CUDA stream, never synchronises
+ *     the device and never throws. It returns AUDIOKV_OK or a negative status. Problems
+ *     seen by a kernel (a bounded wait that ran out) are written to a status word
+ *     that audiokv_last_device_status reads.
+ *   - Q, K and V share one element type (`dtype`); the last dimension (head_dim) is
+ *     contiguous; bases and strides of K/V/Q rows must be 16-byte aligned.
+ *   - L_r is the number of cached tokens of request r (prompt incl. the window),
+ *     W the window, P_r = L_r - W the number of eviction candidates (prefix tokens).
+ *   - Heads are numbered flat: u = (r * n_layers + l) * n_kv_heads + h.
+ *   - Score buffers are fp32, packed: head u of request r starts at
+ *       score_offset(r) + (l * n_kv_heads + h) * P_r,
+ *     score_offset(r) = sum_{r' < r} n_layers * n_kv_heads * P_{r'};
+ *     audiokv_scores_len() gives the total length.
+ *   - Compacted outputs are packed in flat head order: head u owns rows
+ *     [cu_kept[u], cu_kept[u+1]) of k_out / v_out ([rows][head_dim]) and of kept_idx;
+ *     inside a head the kept prefix tokens come in ascending token order, then the
+ *     W window tokens.
+ */
+#ifndef AUDIOKV_H_
+#define AUDIOKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { AUDIOKV_F32 = 0, AUDIOKV_BF16 = 1 };
+
+enum {
+  AUDIOKV_OK = 0,
+  AUDIOKV_EINVAL = -1,       /* an argument is out of range or inconsistent            */
+  AUDIOKV_EALIGN = -2,       /* a pointer or stride breaks the 16-byte rule            */
+  AUDIOKV_EUNSUPPORTED = -3, /* shape outside what the kernels are built for           */
+  AUDIOKV_EWORKSPACE = -4,   /* the context's workspace is too small for these params  */
+  AUDIOKV_ECUDA = -5,        /* a CUDA runtime call failed (see audiokv_last_cuda_error)*/
+  AUDIOKV_ETIMEOUT = -6,     /* a kernel gave up a bounded wait                        */
+  AUDIOKV_EDEVICE = -7       /* a kernel found an index out of range                   */
+};
+
+typedef struct audiokv_ctx audiokv_ctx; /* opaque: device workspace, tables, status word */
+typedef void* audiokv_stream;           /* a cudaStream_t                                */
+
+/* Problem description; plain data in HOST memory, read during the call only. */
+typedef struct {
+  int32_t dtype;                 /* AUDIOKV_F32 | AUDIOKV_BF16                                   */
+  int32_t n_layers;              /* layers evicted in this call (>= 1)                           */
+  int32_t n_q_heads;             /* query heads per layer; a multiple of n_kv_heads              */
+  int32_t n_kv_heads;
+  int32_t head_dim;              /* 64, 128 or 256                                               */
+  int32_t n_req;                 /* requests in the (ragged) batch, 1..AUDIOKV_MAX_REQ           */
+  const int32_t* seq_len;        /* host [n_req]: L_r, each > window                             */
+  int32_t window;                /* W >= 1: the last W tokens are the observation window         */
+  /* element (not byte) offsets: Q(r,l,i,a,t) = r*q_stride_req + l*q_stride_layer + i*q_stride_tok + a*q_stride_head + t */
+  int64_t q_stride_req, q_stride_layer, q_stride_tok, q_stride_head;
+  /* K/V(r,l,h,j,t) = kv_req_offset[r] + l*kv_stride_layer + h*kv_stride_head + j*kv_stride_tok + t */
+  int64_t kv_stride_layer, kv_stride_tok, kv_stride_head;
+  const int64_t* kv_req_offset;  /* host [n_req], or NULL for all-zero                           */
+  float softmax_scale;           /* <= 0 selects 1/sqrt(head_dim)                                */
+  float rho;                     /* SSS energy cut-off ratio, in (0, 1]                          */
+  float alpha;                   /* SSS mixing coefficient, in [0, 1]                            */
+  int32_t transition_bins;       /* T >= 0: cosine band of T bins after the cut-off; 0 = binary mask */
+  int32_t base_per_head;         /* r >= 0: uniform base allocation per head, in tokens          */
+} audiokv_params;
+
+#define AUDIOKV_MAX_REQ 64
+#define AUDIOKV_MAX_SEQ_LEN 131072
+
+/* ---- host-side helpers (no GPU work) ------------------------------------------------ */
+
+/* Text for a status code. Never NULL. */
+const char* audiokv_strerror(int status);
+
+/* Total kept rows of one request at retention ratio c (the paper's "KV-cache retention
+ * ratio"): floor(c * n_heads_total * L), clamped to [n_heads_total * window, n_heads_total * L].
+ * n_heads_total = n_layers * n_kv_heads. Compute it once and hand the same integer to
+ * every consumer. Returns -1 for arguments out of range. */
+int64_t audiokv_budget_from_ratio(double c, int32_t n_heads_total, int32_t seq_len, int32_t window);
+
+/* Number of fp32 elements of a packed score buffer for these params (sum_r N * P_r), or a
+ * negative status. */
+int64_t audiokv_scores_len(const audiokv_params* p);
+
+/* Bytes of workspace audiokv_create must be given so that every call below works for
+ * these params (0 on invalid params). Grows with sum_r L_r; a few MB per 100k tokens. */
+size_t audiokv_workspace_bytes(const audiokv_params* p);
+
+/* ---- context ------------------------------------------------------------------------- */
+
+/* Creates a context on `device` with a workspace of `workspace_bytes` (cudaMalloc; the only
+ * allocation the library makes). *ctx is set on success. */
+int audiokv_create(audiokv_ctx** ctx, int device, size_t workspace_bytes);
+
+/* Frees the workspace. The caller makes sure no call on this context is still running. */
+int audiokv_destroy(audiokv_ctx* ctx);
+
+/* The status word the kernels write (0, AUDIOKV_ETIMEOUT or AUDIOKV_EDEVICE). Synchronises
+ * with the work of earlier calls by a blocking copy on `stream`. */
+int audiokv_last_device_status(audiokv_ctx* ctx, audiokv_stream stream);
+
+/* Text of the last CUDA error a call on this context met (empty string if none). */
+const char* audiokv_last_cuda_error(const audiokv_ctx* ctx);
+
+/* Kernels launched by calls on this context since it was created (for accounting). */
+int64_t audiokv_launch_count(const audiokv_ctx* ctx);
+
+/* ---- the four steps ------------------------------------------------------------------- */
+
+/* Step 1 -- importance scores (Section 3.3, importance sequence over the decoding window).
+ * For window row i (token P+i), query head a of KV head h's group and key j <= P+i:
+ *   z = softmax_scale * <Q[i,a,:], K[j,h,:]>, p = softmax over the visible j; then
+ *   scores_h[j] = sum over the W rows and the group's query heads of p, for j < P.
+ * q_win: the window's queries (layout by q_stride_*). k: the key cache (kv_stride_*).
+ * scores: packed fp32 output (see top). bf16 inputs use tensor cores with fp32
+ * accumulation; f32 inputs use fp32 FMA (no TF32). */
+int audiokv_score(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k, float* scores,
+                  audiokv_stream stream);
+
+/* Step 2 -- Spectral Score Smoothing (Section 3.3). Per head, on x = scores (length n = P):
+ *   F = RFFT(x); E(k) = sum_{i<=k} |F_i|^2; k* = min{k : E(k) >= rho * E(n/2)};
+ *   w_i = 1 (i <= k*), (1 + cos(pi (i-k*)/(T+1)))/2 (k* < i <= k*+T), 0 beyond;
+ *   x~ = IRFFT(F .* w, n); smoothed = (1 - alpha) x + alpha x~.
+ * Any n >= 1 (mixed radix for smooth lengths, chirp-z otherwise). `smoothed` may equal
+ * `scores`. kstar_or_null: optional int32 [total heads] receiving k*. */
+int audiokv_smooth(audiokv_ctx* ctx, const audiokv_params* p, const float* scores, float* smoothed,
+                   int32_t* kstar_or_null, audiokv_stream stream);
+
+/* Step 3 -- head-wise budgets (Section 3.1 allocation rule; Section 3.2's rule when
+ * window and base are taken out). Per request, over its N = n_layers * n_kv_heads heads:
+ * every head gets window + base_per_head rows; the rest of total_budget[r] is shared in
+ * proportion to head_scores (integer arithmetic on round(S * 2^24): floors, then the
+ * left-over rows by largest remainder, lower head index first); no head exceeds L_r
+ * (excess is re-shared). The budgets of a request add up to total_budget[r] exactly.
+ * head_scores: device fp32 [n_req][n_layers][n_kv_heads], each in [0, 128].
+ * total_budget: HOST int64 [n_req], N*(W+base) <= B_r <= N*L_r (else AUDIOKV_EINVAL).
+ * budgets: device int32 [total heads] (window included).
+ * cu_kept: device int32 [total heads + 1], exclusive prefix sum of budgets. */
+int audiokv_allocate(audiokv_ctx* ctx, const audiokv_params* p, const float* head_scores,
+                     const int64_t* total_budget, int32_t* budgets, int32_t* cu_kept, audiokv_stream stream);
+
+/* Step 4 -- Top-K selection and eviction. Per head u: the budgets[u] - W prefix tokens
+ * with the largest smoothed score (ties: lower token index), in ascending token order,
+ * then the window tokens P..L-1; their indices go to kept_idx and their K and V rows,
+ * copied bit for bit, to k_out and v_out, all at rows [cu_kept[u], cu_kept[u+1]).
+ * k_out / v_out must not overlap k / v. NaN scores give an unspecified selection. */
+int audiokv_select_gather(audiokv_ctx* ctx, const audiokv_params* p, const float* smoothed, const int32_t* budgets,
+                          const int32_t* cu_kept, const void* k, const void* v, void* k_out, void* v_out,
+                          int32_t* kept_idx, audiokv_stream stream);
+
+/* The whole pass in one call: allocate, score, smooth, select, gather, with the
+ * intermediate score buffers in the context's workspace. Arguments as above; budgets and
+ * cu_kept are outputs. k_out, v_out and kept_idx need sum_r total_budget[r] rows. */
+int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k, const void* v,
+                  const float* head_scores, const int64_t* total_budget, void* k_out, void* v_out,
+                  int32_t* kept_idx, int32_t* budgets, int32_t* cu_kept, audiokv_stream stream);
+
+/* Same pass with every buffer in HOST memory (pageable or pinned): copies the inputs to
+ * the device (into the workspace, which must have been sized with
+ * audiokv_workspace_bytes_host), runs audiokv_evict, copies kept_idx, budgets, cu_kept,
+ * k_out and v_out back and waits for the stream. q/k/v extents are given in elements. */
+int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, int64_t q_elems, const void* k,
+                       const void* v, int64_t kv_elems, const float* head_scores, const int64_t* total_budget,
+                       void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* cu_kept,
+                       audiokv_stream stream);
+size_t audiokv_workspace_bytes_host(const audiokv_params* p, int64_t q_elems, int64_t kv_elems,
+                                    const int64_t* total_budget);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AUDIOKV_H_ */

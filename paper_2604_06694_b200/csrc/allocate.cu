@@ -1,0 +1,184 @@
+// Head-wise budgets in exact integer arithmetic: one thread block per request.
+//
+// Every head gets window + base rows; the remaining rows R of the request's total are
+// shared in proportion to S_q = round-half-up(S * 2^24): floors first, heads whose share
+// would exceed the rows they have are fixed at that cap and taken out of the pool (and
+// the shares recomputed), and the rows the floors leave over go one each to the largest
+// remainders, lower head index first. All-zero scores split R evenly.
+#include "common.cuh"
+
+namespace akv {
+namespace {
+
+constexpr int kAllocThreads = 256;
+
+struct BudgetArgs {
+  int64_t total[AUDIOKV_MAX_REQ];
+};
+
+__device__ __forceinline__ long long block_sum_ll(long long v, long long* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  long long t = 0;
+  for (int w = 0; w < kAllocThreads / 32; ++w) t += red[w];
+  return t;
+}
+
+__global__ void __launch_bounds__(kAllocThreads)
+allocate_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restrict__ head_scores, BudgetArgs args,
+                int32_t* __restrict__ budgets, int* __restrict__ status) {
+  extern __shared__ long long sm[];
+  const int N = sh.heads_per_req;
+  long long* Sq = sm;            // [N] quantised scores
+  long long* tk = Sq + N;        // [N] share above the floor
+  long long* rem = tk + N;       // [N] remainders
+  int* active = reinterpret_cast<int*>(rem + N);  // [N] 1 while the head is in the pool
+  int* give = active + N;                         // [N] 1 when the head receives a left-over row this turn
+  __shared__ long long red[kAllocThreads / 32];
+
+  const int r = blockIdx.x;
+  const ReqDesc rq = reqs[r];
+  const float* S = head_scores + static_cast<int64_t>(r) * N;
+  const long long f = static_cast<long long>(sh.window) + sh.base_per_head;
+  const long long cap = rq.L - f;
+  long long R = args.total[r] - static_cast<long long>(N) * f;
+
+  for (int h = threadIdx.x; h < N; h += kAllocThreads) {
+    const double v = static_cast<double>(S[h]);
+    long long q = 0;
+    if (!(v >= 0.0) || v > 128.0) {
+      atomicExch(status, AUDIOKV_EINVAL);  // invalid score: treated as zero
+    } else {
+      q = static_cast<long long>(floor(v * 16777216.0 + 0.5));
+    }
+    Sq[h] = q;
+    tk[h] = 0;
+    active[h] = 1;
+  }
+  __syncthreads();
+
+  for (int round = 0; round <= N; ++round) {
+    long long lsum = 0, lcnt = 0;
+    for (int h = threadIdx.x; h < N; h += kAllocThreads)
+      if (active[h]) {
+        lsum += Sq[h];
+        ++lcnt;
+      }
+    const long long sum = block_sum_ll(lsum, red);
+    const long long nA = block_sum_ll(lcnt, red);
+    if (nA == 0) break;
+    if (sum == 0) {
+      // even split by rank inside the pool
+      for (int h = threadIdx.x; h < N; h += kAllocThreads)
+        if (active[h]) {
+          int rank = 0;
+          for (int g = 0; g < h; ++g) rank += active[g];
+          tk[h] = R / nA + (rank < R % nA ? 1 : 0);
+        }
+      break;
+    }
+    long long lover = 0;
+    for (int h = threadIdx.x; h < N; h += kAllocThreads)
+      if (active[h]) {
+        const long long prod = R * Sq[h];  // R < 2^31 and S_q <= 2^31: no overflow
+        const long long sh_ = prod / sum;
+        tk[h] = sh_;
+        rem[h] = prod - sh_ * sum;
+        if (sh_ > cap) ++lover;
+      }
+    const long long n_over = block_sum_ll(lover, red);
+    if (n_over > 0) {
+      for (int h = threadIdx.x; h < N; h += kAllocThreads)
+        if (active[h] && tk[h] > cap) {
+          tk[h] = cap;
+          active[h] = 0;
+        }
+      R -= n_over * cap;
+      __syncthreads();
+      continue;
+    }
+    long long lgiven = 0;
+    for (int h = threadIdx.x; h < N; h += kAllocThreads)
+      if (active[h]) lgiven += tk[h];
+    long long left = R - block_sum_ll(lgiven, red);
+    // hand out the left-over rows by descending remainder, ties by ascending index, skipping full heads
+    while (left > 0) {
+      long long lelig = 0;
+      for (int h = threadIdx.x; h < N; h += kAllocThreads)
+        if (active[h] && tk[h] < cap) ++lelig;
+      const long long n_elig = block_sum_ll(lelig, red);
+      if (n_elig == 0) break;
+      for (int h = threadIdx.x; h < N; h += kAllocThreads)
+        if (active[h] && tk[h] < cap) {
+          long long rank = 0;
+          for (int g = 0; g < N; ++g)
+            if (active[g] && tk[g] < cap && (rem[g] > rem[h] || (rem[g] == rem[h] && g < h))) ++rank;
+          give[h] = rank < left ? 1 : 0;
+        } else {
+          give[h] = 0;
+        }
+      __syncthreads();  // the increments are applied after every thread has ranked against the old shares
+      for (int h = threadIdx.x; h < N; h += kAllocThreads)
+        if (give[h]) tk[h] += 1;
+      left -= n_elig < left ? n_elig : left;
+      __syncthreads();
+    }
+    break;
+  }
+  __syncthreads();
+  for (int h = threadIdx.x; h < N; h += kAllocThreads)
+    budgets[rq.head_base + h] = static_cast<int32_t>(f + tk[h]);
+}
+
+// cu_kept = exclusive prefix sum of budgets over all heads (single block).
+__global__ void __launch_bounds__(1024) cu_kept_kernel(const int32_t* __restrict__ budgets, int total,
+                                                      int32_t* __restrict__ cu_kept) {
+  __shared__ int wsum[32];
+  const int per = (total + 1023) / 1024;
+  const int a = min(total, static_cast<int>(threadIdx.x) * per), b = min(total, a + per);
+  int local = 0;
+  for (int i = a; i < b; ++i) local += budgets[i];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = local;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) wsum[warp] = inc;
+  __syncthreads();
+  int ws = wsum[lane], winc = ws;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(0xffffffffu, winc, o);
+    if (lane >= o) winc += t;
+  }
+  int run = __shfl_sync(0xffffffffu, winc - ws, warp) + inc - local;
+  for (int i = a; i < b; ++i) {
+    cu_kept[i] = run;
+    run += budgets[i];
+  }
+  if (a < b && b == total) cu_kept[total] = run;  // the one non-empty range that ends at `total`
+  if (total == 0 && threadIdx.x == 0) cu_kept[0] = 0;
+}
+
+}  // namespace
+
+cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float* head_scores,
+                            const int64_t* h_total_budget, int32_t* budgets, int32_t* cu_kept, int* status,
+                            Launch ln) {
+  BudgetArgs args;
+  for (int r = 0; r < sh.n_req; ++r) args.total[r] = h_total_budget[r];
+  const size_t smem = static_cast<size_t>(sh.heads_per_req) * (3 * sizeof(long long) + 2 * sizeof(int));
+  cudaError_t e = cudaFuncSetAttribute(allocate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  allocate_kernel<<<sh.n_req, kAllocThreads, smem, ln.stream>>>(sh, d_reqs, head_scores, args, budgets, status);
+  cu_kept_kernel<<<1, 1024, 0, ln.stream>>>(budgets, sh.total_heads, cu_kept);
+  *ln.launch_counter += 2;
+  return cudaGetLastError();
+}
+
+}  // namespace akv

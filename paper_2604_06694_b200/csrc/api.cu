@@ -1,0 +1,554 @@
+// C boundary of the AudioKV eviction pass: argument checks, the per-shape plan (request
+// table, FFT plans and tables, workspace layout) and the launch sequence of each entry point.
+#include <math.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace akv;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kSssSmemComplex = 25600;  // 200 KB of float2: the largest work buffer kept in shared memory
+constexpr int kSimtSlabKeys = 512;
+constexpr int kMaxRows = 1024;          // W * G
+constexpr int kMaxHeadsPerReq = 2048;
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {  // byte offsets inside the workspace
+  size_t status, reqs, plans, tables, stats, fft_scratch, scores, kstar, end;
+};
+
+struct Plan {
+  bool valid = false;
+  audiokv_params p{};
+  std::vector<int32_t> seq_len;
+  std::vector<int64_t> kv_off;
+  Shape sh{};
+  std::vector<ReqDesc> reqs;
+  std::vector<FftPlan> fft;
+  int64_t table_len = 0;        // float2 elements
+  int64_t scores_len = 0;
+  int max_L = 0, max_P = 0;
+  int n_slab = 0;
+  int sss_grid = 0;
+  size_t sss_smem = 0;
+  int64_t scratch_per_block = 0;  // float2 elements
+  Layout lay{};
+};
+
+}  // namespace
+
+struct audiokv_ctx {
+  int device = 0;
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  Plan plan;
+  bool plan_uploaded = false;
+  cudaEvent_t plan_ready = nullptr;
+  int64_t launches = 0;
+  std::string cuda_error;
+};
+
+namespace {
+
+int esize(int dtype) { return dtype == AUDIOKV_F32 ? 4 : 2; }
+
+int check_params(const audiokv_params* p) {
+  if (!p || !p->seq_len) return AUDIOKV_EINVAL;
+  if (p->dtype != AUDIOKV_F32 && p->dtype != AUDIOKV_BF16) return AUDIOKV_EINVAL;
+  if (p->n_layers < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads) return AUDIOKV_EINVAL;
+  if (p->n_req < 1 || p->n_req > AUDIOKV_MAX_REQ || p->window < 1) return AUDIOKV_EINVAL;
+  if (!(p->rho > 0.f && p->rho <= 1.f) || !(p->alpha >= 0.f && p->alpha <= 1.f)) return AUDIOKV_EINVAL;
+  if (p->transition_bins < 0 || p->base_per_head < 0) return AUDIOKV_EINVAL;
+  for (int r = 0; r < p->n_req; ++r) {
+    if (p->seq_len[r] <= p->window || p->seq_len[r] > AUDIOKV_MAX_SEQ_LEN) return AUDIOKV_EINVAL;
+    if (p->kv_req_offset && p->kv_req_offset[r] < 0) return AUDIOKV_EINVAL;
+  }
+  if (p->head_dim != 64 && p->head_dim != 128 && p->head_dim != 256) return AUDIOKV_EUNSUPPORTED;
+  const int64_t rows = static_cast<int64_t>(p->window) * (p->n_q_heads / p->n_kv_heads);
+  if (rows > kMaxRows) return AUDIOKV_EUNSUPPORTED;
+  if (static_cast<int64_t>(p->n_layers) * p->n_kv_heads > kMaxHeadsPerReq) return AUDIOKV_EUNSUPPORTED;
+  const int per16 = 16 / esize(p->dtype);
+  const int64_t strides[] = {p->q_stride_req, p->q_stride_layer, p->q_stride_tok, p->q_stride_head,
+                             p->kv_stride_layer, p->kv_stride_tok, p->kv_stride_head};
+  for (int64_t s : strides) {
+    if (s < 0) return AUDIOKV_EINVAL;
+    if (s % per16) return AUDIOKV_EALIGN;
+  }
+  if (p->kv_req_offset)
+    for (int r = 0; r < p->n_req; ++r)
+      if (p->kv_req_offset[r] % per16) return AUDIOKV_EALIGN;
+  return AUDIOKV_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool same_plan(const Plan& pl, const audiokv_params* p) {
+  if (!pl.valid) return false;
+  const audiokv_params& a = pl.p;
+  if (a.dtype != p->dtype || a.n_layers != p->n_layers || a.n_q_heads != p->n_q_heads ||
+      a.n_kv_heads != p->n_kv_heads || a.head_dim != p->head_dim || a.n_req != p->n_req || a.window != p->window ||
+      a.q_stride_req != p->q_stride_req || a.q_stride_layer != p->q_stride_layer ||
+      a.q_stride_tok != p->q_stride_tok || a.q_stride_head != p->q_stride_head ||
+      a.kv_stride_layer != p->kv_stride_layer || a.kv_stride_tok != p->kv_stride_tok ||
+      a.kv_stride_head != p->kv_stride_head || a.softmax_scale != p->softmax_scale || a.rho != p->rho ||
+      a.alpha != p->alpha || a.transition_bins != p->transition_bins || a.base_per_head != p->base_per_head)
+    return false;
+  for (int r = 0; r < p->n_req; ++r) {
+    if (pl.seq_len[r] != p->seq_len[r]) return false;
+    if (pl.kv_off[r] != (p->kv_req_offset ? p->kv_req_offset[r] : 0)) return false;
+  }
+  return true;
+}
+
+// Radix sequence for a complex length N: primes 11..127 first (descending), then 7, 5, 3, 4s, 2.
+// Returns false when N has a prime factor above 127.
+bool factor_len(int N, FftSeq* sq) {
+  sq->N = N;
+  sq->n_pass = 0;
+  int rest = N, twos = 0;
+  while (rest % 2 == 0) {
+    rest /= 2;
+    ++twos;
+  }
+  std::vector<int> odd;
+  for (int q = 3; q <= 127 && rest > 1; q += 2)
+    while (rest % q == 0) {
+      odd.push_back(q);
+      rest /= q;
+    }
+  if (rest != 1) return false;
+  std::vector<int> seq;
+  for (auto it = odd.rbegin(); it != odd.rend(); ++it) seq.push_back(*it);
+  for (int i = 0; i < twos / 2; ++i) seq.push_back(4);
+  if (twos % 2) seq.push_back(2);
+  if (seq.size() > static_cast<size_t>(kMaxRadices)) return false;
+  for (size_t i = 0; i < seq.size(); ++i) sq->radix[i] = seq[i];
+  sq->n_pass = static_cast<int>(seq.size());
+  return true;
+}
+
+void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
+  memset(fp, 0, sizeof(*fp));
+  fp->n = n;
+  fp->packed = (n % 2 == 0) ? 1 : 0;
+  fp->N = fp->packed ? n / 2 : n;
+  const int N = fp->N;
+  int buf_len = N;
+  if (factor_len(N, &fp->seq)) {
+    fp->bluestein = 0;
+    fp->M = 0;
+  } else {
+    fp->bluestein = 1;
+    int M = 1;
+    while (M < 2 * N - 1) M *= 2;
+    fp->M = M;
+    factor_len(M, &fp->seq);
+    buf_len = M;
+  }
+  fp->in_smem = buf_len <= kSssSmemComplex ? 1 : 0;
+  fp->seq.tw_offset = *table_len;
+  *table_len += fp->seq.N;
+  if (fp->packed) {
+    fp->post_offset = *table_len;
+    *table_len += N / 2 + 1;
+  }
+  if (fp->bluestein) {
+    fp->chirp_offset = *table_len;
+    *table_len += N;
+    fp->filter_offset = *table_len;
+    *table_len += fp->M;
+  }
+}
+
+int build_plan(const audiokv_params* p, Plan* pl) {
+  int rc = check_params(p);
+  if (rc) return rc;
+  pl->valid = false;
+  pl->p = *p;
+  pl->seq_len.assign(p->seq_len, p->seq_len + p->n_req);
+  pl->kv_off.assign(p->n_req, 0);
+  if (p->kv_req_offset) pl->kv_off.assign(p->kv_req_offset, p->kv_req_offset + p->n_req);
+  pl->p.seq_len = nullptr;
+  pl->p.kv_req_offset = nullptr;
+
+  Shape& sh = pl->sh;
+  sh.dtype = p->dtype;
+  sh.n_layers = p->n_layers;
+  sh.n_q_heads = p->n_q_heads;
+  sh.n_kv_heads = p->n_kv_heads;
+  sh.head_dim = p->head_dim;
+  sh.n_req = p->n_req;
+  sh.window = p->window;
+  sh.group = p->n_q_heads / p->n_kv_heads;
+  sh.heads_per_req = p->n_layers * p->n_kv_heads;
+  sh.total_heads = sh.heads_per_req * p->n_req;
+  sh.q_stride_layer = p->q_stride_layer;
+  sh.q_stride_tok = p->q_stride_tok;
+  sh.q_stride_head = p->q_stride_head;
+  sh.kv_stride_layer = p->kv_stride_layer;
+  sh.kv_stride_tok = p->kv_stride_tok;
+  sh.kv_stride_head = p->kv_stride_head;
+  sh.softmax_scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(static_cast<float>(p->head_dim));
+  sh.scale_log2e = static_cast<float>(static_cast<double>(sh.softmax_scale) * 1.4426950408889634);
+  sh.rho = p->rho;
+  sh.alpha = p->alpha;
+  sh.transition_bins = p->transition_bins;
+  sh.base_per_head = p->base_per_head;
+
+  pl->reqs.assign(p->n_req, ReqDesc{});
+  pl->fft.clear();
+  pl->table_len = 0;
+  pl->scores_len = 0;
+  pl->max_L = pl->max_P = 0;
+  for (int r = 0; r < p->n_req; ++r) {
+    ReqDesc& d = pl->reqs[r];
+    d.L = p->seq_len[r];
+    d.P = d.L - p->window;
+    d.head_base = r * sh.heads_per_req;
+    d.kv_offset = pl->kv_off[r];
+    d.q_offset = r * p->q_stride_req;
+    d.score_offset = pl->scores_len;
+    pl->scores_len += static_cast<int64_t>(sh.heads_per_req) * d.P;
+    pl->max_L = d.L > pl->max_L ? d.L : pl->max_L;
+    pl->max_P = d.P > pl->max_P ? d.P : pl->max_P;
+    int found = -1;
+    for (size_t i = 0; i < pl->fft.size(); ++i)
+      if (pl->fft[i].n == d.P) found = static_cast<int>(i);
+    if (found < 0) {
+      FftPlan fp;
+      build_fft_plan(d.P, &fp, &pl->table_len);
+      pl->fft.push_back(fp);
+      found = static_cast<int>(pl->fft.size()) - 1;
+    }
+    d.fft_plan = found;
+  }
+  pl->n_slab = (pl->max_L + kSimtSlabKeys - 1) / kSimtSlabKeys;
+  pl->sss_grid = sh.total_heads < 148 ? sh.total_heads : 148;
+  int smem_c = 2;
+  pl->scratch_per_block = 0;
+  for (const FftPlan& fp : pl->fft) {
+    const int len = fp.bluestein ? fp.M : fp.N;
+    if (fp.in_smem) smem_c = len > smem_c ? len : smem_c;
+    else pl->scratch_per_block = len > pl->scratch_per_block ? len : pl->scratch_per_block;
+  }
+  pl->sss_smem = static_cast<size_t>(smem_c) * sizeof(float2);
+
+  Layout& L = pl->lay;
+  size_t off = 0;
+  L.status = off;      off = align_up(off + 64);
+  L.reqs = off;        off = align_up(off + sizeof(ReqDesc) * AUDIOKV_MAX_REQ);
+  L.plans = off;       off = align_up(off + sizeof(FftPlan) * kMaxPlans);
+  L.tables = off;      off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->table_len));
+  L.stats = off;       off = align_up(off + sizeof(float2) * static_cast<size_t>(sh.total_heads) * pl->n_slab * sh.window * sh.group);
+  L.fft_scratch = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->scratch_per_block) * pl->sss_grid);
+  L.scores = off;      off = align_up(off + sizeof(float) * static_cast<size_t>(pl->scores_len));
+  L.kstar = off;       off = align_up(off + sizeof(int32_t) * static_cast<size_t>(sh.total_heads));
+  L.end = off;
+  pl->valid = true;
+  return AUDIOKV_OK;
+}
+
+int cuda_fail(audiokv_ctx* ctx, cudaError_t e) {
+  ctx->cuda_error = cudaGetErrorString(e);
+  return AUDIOKV_ECUDA;
+}
+
+// Makes ctx->plan match p and its tables resident on the device (stream-ordered).
+int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
+  if (!ctx) return AUDIOKV_EINVAL;
+  cudaError_t e = cudaSetDevice(ctx->device);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  if (!same_plan(ctx->plan, p)) {
+    int rc = build_plan(p, &ctx->plan);
+    if (rc) return rc;
+    ctx->plan_uploaded = false;
+  }
+  Plan& pl = ctx->plan;
+  if (pl.lay.end > ctx->ws_bytes) return AUDIOKV_EWORKSPACE;
+  if (!ctx->plan_uploaded) {
+    // earlier calls on other streams may still read the old tables
+    if ((e = cudaStreamWaitEvent(stream, ctx->plan_ready, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaMemsetAsync(ctx->ws + pl.lay.status, 0, 64, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.reqs, pl.reqs.data(), sizeof(ReqDesc) * pl.reqs.size(),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+      return cuda_fail(ctx, e);
+    if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.plans, pl.fft.data(), sizeof(FftPlan) * pl.fft.size(),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+      return cuda_fail(ctx, e);
+    Launch ln{stream, &ctx->launches};
+    e = launch_fft_tables(static_cast<int>(pl.fft.size()), reinterpret_cast<float2*>(ctx->ws + pl.lay.tables),
+                          reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans), ln);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaEventRecord(ctx->plan_ready, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->plan_uploaded = true;
+  } else {
+    if ((e = cudaStreamWaitEvent(stream, ctx->plan_ready, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+  }
+  return AUDIOKV_OK;
+}
+
+const ReqDesc* d_reqs(audiokv_ctx* c) { return reinterpret_cast<const ReqDesc*>(c->ws + c->plan.lay.reqs); }
+int* d_status(audiokv_ctx* c) { return reinterpret_cast<int*>(c->ws + c->plan.lay.status); }
+
+int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cudaStream_t stream) {
+  Plan& pl = ctx->plan;
+  Launch ln{stream, &ctx->launches};
+  cudaError_t e = launch_score_simt(pl.sh, d_reqs(ctx), q, k, scores, reinterpret_cast<float2*>(ctx->ws + pl.lay.stats),
+                                    pl.n_slab, kSimtSlabKeys, ln);
+  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
+}
+
+int do_smooth(audiokv_ctx* ctx, const float* scores, float* smoothed, int32_t* kstar, cudaStream_t stream) {
+  Plan& pl = ctx->plan;
+  Launch ln{stream, &ctx->launches};
+  cudaError_t e = launch_sss(pl.sh, d_reqs(ctx), reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans),
+                             reinterpret_cast<const float2*>(ctx->ws + pl.lay.tables), scores, smoothed, kstar,
+                             reinterpret_cast<float2*>(ctx->ws + pl.lay.fft_scratch), pl.scratch_per_block,
+                             pl.sss_grid, pl.sss_smem, ln);
+  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
+}
+
+int check_budgets(const Plan& pl, const int64_t* total_budget) {
+  if (!total_budget) return AUDIOKV_EINVAL;
+  const int64_t N = pl.sh.heads_per_req, f = static_cast<int64_t>(pl.sh.window) + pl.sh.base_per_head;
+  for (int r = 0; r < pl.sh.n_req; ++r) {
+    if (f > pl.reqs[r].L) return AUDIOKV_EINVAL;
+    if (total_budget[r] < N * f || total_budget[r] > N * pl.reqs[r].L) return AUDIOKV_EINVAL;
+  }
+  return AUDIOKV_OK;
+}
+
+int do_allocate(audiokv_ctx* ctx, const float* head_scores, const int64_t* total_budget, int32_t* budgets,
+                int32_t* cu_kept, cudaStream_t stream) {
+  Plan& pl = ctx->plan;
+  int rc = check_budgets(pl, total_budget);
+  if (rc) return rc;
+  Launch ln{stream, &ctx->launches};
+  cudaError_t e = launch_allocate(pl.sh, d_reqs(ctx), head_scores, total_budget, budgets, cu_kept, d_status(ctx), ln);
+  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
+}
+
+int do_select_gather(audiokv_ctx* ctx, const float* smoothed, const int32_t* budgets, const int32_t* cu_kept,
+                     const void* k, const void* v, void* k_out, void* v_out, int32_t* kept_idx, cudaStream_t stream) {
+  Plan& pl = ctx->plan;
+  Launch ln{stream, &ctx->launches};
+  cudaError_t e = launch_select(pl.sh, d_reqs(ctx), smoothed, budgets, cu_kept, kept_idx, pl.max_P, d_status(ctx), ln);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  e = launch_gather(pl.sh, d_reqs(ctx), cu_kept, kept_idx, k, v, k_out, v_out, ln);
+  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* audiokv_strerror(int status) {
+  switch (status) {
+    case AUDIOKV_OK: return "ok";
+    case AUDIOKV_EINVAL: return "invalid argument";
+    case AUDIOKV_EALIGN: return "pointer or stride not 16-byte aligned";
+    case AUDIOKV_EUNSUPPORTED: return "shape not supported";
+    case AUDIOKV_EWORKSPACE: return "workspace too small";
+    case AUDIOKV_ECUDA: return "CUDA runtime error";
+    case AUDIOKV_ETIMEOUT: return "a kernel gave up a bounded wait";
+    case AUDIOKV_EDEVICE: return "a kernel found an index out of range";
+    default: return "unknown status";
+  }
+}
+
+int64_t audiokv_budget_from_ratio(double c, int32_t n_heads_total, int32_t seq_len, int32_t window) {
+  if (!(c >= 0.0 && c <= 1.0) || n_heads_total < 1 || seq_len < 1 || window < 0 || window > seq_len) return -1;
+  const int64_t hi = static_cast<int64_t>(n_heads_total) * seq_len, lo = static_cast<int64_t>(n_heads_total) * window;
+  int64_t b = static_cast<int64_t>(floor(c * static_cast<double>(hi)));
+  return b < lo ? lo : (b > hi ? hi : b);
+}
+
+int64_t audiokv_scores_len(const audiokv_params* p) {
+  int rc = check_params(p);
+  if (rc) return rc;
+  int64_t n = 0;
+  for (int r = 0; r < p->n_req; ++r)
+    n += static_cast<int64_t>(p->n_layers) * p->n_kv_heads * (p->seq_len[r] - p->window);
+  return n;
+}
+
+size_t audiokv_workspace_bytes(const audiokv_params* p) {
+  Plan pl;
+  if (build_plan(p, &pl)) return 0;
+  return pl.lay.end;
+}
+
+size_t audiokv_workspace_bytes_host(const audiokv_params* p, int64_t q_elems, int64_t kv_elems,
+                                    const int64_t* total_budget) {
+  Plan pl;
+  if (build_plan(p, &pl) || !total_budget || q_elems < 0 || kv_elems < 0) return 0;
+  const size_t es = esize(p->dtype);
+  int64_t rows = 0;
+  for (int r = 0; r < p->n_req; ++r) rows += total_budget[r];
+  size_t off = pl.lay.end;
+  off = align_up(off + q_elems * es);
+  off = align_up(off + kv_elems * es) ;
+  off = align_up(off + kv_elems * es);
+  off = align_up(off + sizeof(float) * pl.sh.total_heads);
+  off = align_up(off + rows * p->head_dim * es);
+  off = align_up(off + rows * p->head_dim * es);
+  off = align_up(off + rows * sizeof(int32_t));
+  off = align_up(off + sizeof(int32_t) * pl.sh.total_heads);
+  off = align_up(off + sizeof(int32_t) * (pl.sh.total_heads + 1));
+  return off;
+}
+
+int audiokv_create(audiokv_ctx** out, int device, size_t workspace_bytes) {
+  if (!out || workspace_bytes == 0) return AUDIOKV_EINVAL;
+  *out = nullptr;
+  if (cudaSetDevice(device) != cudaSuccess) return AUDIOKV_ECUDA;
+  audiokv_ctx* c = new audiokv_ctx();
+  c->device = device;
+  if (cudaMalloc(&c->ws, workspace_bytes) != cudaSuccess) {
+    delete c;
+    return AUDIOKV_ECUDA;
+  }
+  c->ws_bytes = workspace_bytes;
+  if (cudaEventCreateWithFlags(&c->plan_ready, cudaEventDisableTiming) != cudaSuccess) {
+    cudaFree(c->ws);
+    delete c;
+    return AUDIOKV_ECUDA;
+  }
+  *out = c;
+  return AUDIOKV_OK;
+}
+
+int audiokv_destroy(audiokv_ctx* ctx) {
+  if (!ctx) return AUDIOKV_EINVAL;
+  cudaSetDevice(ctx->device);
+  cudaEventDestroy(ctx->plan_ready);
+  cudaFree(ctx->ws);
+  delete ctx;
+  return AUDIOKV_OK;
+}
+
+int audiokv_last_device_status(audiokv_ctx* ctx, audiokv_stream stream) {
+  if (!ctx || !ctx->plan.valid) return AUDIOKV_EINVAL;
+  int st = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(&st, d_status(ctx), sizeof(int), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return st;
+}
+
+const char* audiokv_last_cuda_error(const audiokv_ctx* ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
+
+int64_t audiokv_launch_count(const audiokv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int audiokv_score(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k, float* scores,
+                  audiokv_stream stream) {
+  if (!q_win || !k || !scores) return AUDIOKV_EINVAL;
+  if (!aligned16(q_win) || !aligned16(k)) return AUDIOKV_EALIGN;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(ctx, p, s);
+  if (rc) return rc;
+  return do_score(ctx, q_win, k, scores, s);
+}
+
+int audiokv_smooth(audiokv_ctx* ctx, const audiokv_params* p, const float* scores, float* smoothed,
+                   int32_t* kstar_or_null, audiokv_stream stream) {
+  if (!scores || !smoothed) return AUDIOKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(ctx, p, s);
+  if (rc) return rc;
+  return do_smooth(ctx, scores, smoothed, kstar_or_null, s);
+}
+
+int audiokv_allocate(audiokv_ctx* ctx, const audiokv_params* p, const float* head_scores,
+                     const int64_t* total_budget, int32_t* budgets, int32_t* cu_kept, audiokv_stream stream) {
+  if (!head_scores || !total_budget || !budgets || !cu_kept) return AUDIOKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(ctx, p, s);
+  if (rc) return rc;
+  return do_allocate(ctx, head_scores, total_budget, budgets, cu_kept, s);
+}
+
+int audiokv_select_gather(audiokv_ctx* ctx, const audiokv_params* p, const float* smoothed, const int32_t* budgets,
+                          const int32_t* cu_kept, const void* k, const void* v, void* k_out, void* v_out,
+                          int32_t* kept_idx, audiokv_stream stream) {
+  if (!smoothed || !budgets || !cu_kept || !k || !v || !k_out || !v_out || !kept_idx) return AUDIOKV_EINVAL;
+  if (!aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out)) return AUDIOKV_EALIGN;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(ctx, p, s);
+  if (rc) return rc;
+  return do_select_gather(ctx, smoothed, budgets, cu_kept, k, v, k_out, v_out, kept_idx, s);
+}
+
+int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k, const void* v,
+                  const float* head_scores, const int64_t* total_budget, void* k_out, void* v_out,
+                  int32_t* kept_idx, int32_t* budgets, int32_t* cu_kept, audiokv_stream stream) {
+  if (!q_win || !k || !v || !head_scores || !total_budget || !k_out || !v_out || !kept_idx || !budgets || !cu_kept)
+    return AUDIOKV_EINVAL;
+  if (!aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+    return AUDIOKV_EALIGN;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(ctx, p, s);
+  if (rc) return rc;
+  Plan& pl = ctx->plan;
+  float* ws_scores = reinterpret_cast<float*>(ctx->ws + pl.lay.scores);
+  int32_t* ws_kstar = reinterpret_cast<int32_t*>(ctx->ws + pl.lay.kstar);
+  if ((rc = do_allocate(ctx, head_scores, total_budget, budgets, cu_kept, s))) return rc;
+  if ((rc = do_score(ctx, q_win, k, ws_scores, s))) return rc;
+  if ((rc = do_smooth(ctx, ws_scores, ws_scores, ws_kstar, s))) return rc;
+  return do_select_gather(ctx, ws_scores, budgets, cu_kept, k, v, k_out, v_out, kept_idx, s);
+}
+
+int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, int64_t q_elems, const void* k,
+                       const void* v, int64_t kv_elems, const float* head_scores, const int64_t* total_budget,
+                       void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* cu_kept,
+                       audiokv_stream stream) {
+  if (!q_win || !k || !v || !head_scores || !total_budget || !k_out || !v_out || !kept_idx || !budgets || !cu_kept)
+    return AUDIOKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(ctx, p, s);
+  if (rc) return rc;
+  Plan& pl = ctx->plan;
+  if (audiokv_workspace_bytes_host(p, q_elems, kv_elems, total_budget) > ctx->ws_bytes) return AUDIOKV_EWORKSPACE;
+  const size_t es = esize(p->dtype);
+  int64_t rows = 0;
+  for (int r = 0; r < p->n_req; ++r) rows += total_budget[r];
+  const int TH = pl.sh.total_heads;
+  size_t off = pl.lay.end;
+  char* dq = ctx->ws + off;   off = align_up(off + q_elems * es);
+  char* dk = ctx->ws + off;   off = align_up(off + kv_elems * es);
+  char* dv = ctx->ws + off;   off = align_up(off + kv_elems * es);
+  char* dS = ctx->ws + off;   off = align_up(off + sizeof(float) * TH);
+  char* dko = ctx->ws + off;  off = align_up(off + rows * p->head_dim * es);
+  char* dvo = ctx->ws + off;  off = align_up(off + rows * p->head_dim * es);
+  char* dki = ctx->ws + off;  off = align_up(off + rows * sizeof(int32_t));
+  char* db = ctx->ws + off;   off = align_up(off + sizeof(int32_t) * TH);
+  char* dcu = ctx->ws + off;
+  cudaError_t e;
+#define AKV_CP(dst, src, n, kind) \
+  if ((e = cudaMemcpyAsync(dst, src, n, kind, s)) != cudaSuccess) return cuda_fail(ctx, e)
+  AKV_CP(dq, q_win, q_elems * es, cudaMemcpyHostToDevice);
+  AKV_CP(dk, k, kv_elems * es, cudaMemcpyHostToDevice);
+  AKV_CP(dv, v, kv_elems * es, cudaMemcpyHostToDevice);
+  AKV_CP(dS, head_scores, sizeof(float) * TH, cudaMemcpyHostToDevice);
+  rc = audiokv_evict(ctx, p, dq, dk, dv, reinterpret_cast<float*>(dS), total_budget, dko, dvo,
+                     reinterpret_cast<int32_t*>(dki), reinterpret_cast<int32_t*>(db), reinterpret_cast<int32_t*>(dcu), s);
+  if (rc) return rc;
+  AKV_CP(k_out, dko, rows * p->head_dim * es, cudaMemcpyDeviceToHost);
+  AKV_CP(v_out, dvo, rows * p->head_dim * es, cudaMemcpyDeviceToHost);
+  AKV_CP(kept_idx, dki, rows * sizeof(int32_t), cudaMemcpyDeviceToHost);
+  AKV_CP(budgets, db, sizeof(int32_t) * TH, cudaMemcpyDeviceToHost);
+  AKV_CP(cu_kept, dcu, sizeof(int32_t) * (TH + 1), cudaMemcpyDeviceToHost);
+#undef AKV_CP
+  if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(ctx, e);
+  return AUDIOKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,96 @@
+// Shared declarations of the CUDA side of the AudioKV eviction pass (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/audiokv.h"
+
+namespace akv {
+
+// One request of the ragged batch, as the kernels see it.
+struct ReqDesc {
+  int32_t L;             // cached tokens
+  int32_t P;             // prefix tokens = L - W
+  int32_t head_base;     // flat index of the request's first head
+  int32_t fft_plan;      // index into the FFT plan table (one per distinct P)
+  int64_t kv_offset;     // element offset of the request inside K / V
+  int64_t q_offset;      // element offset of the request inside Q
+  int64_t score_offset;  // element offset of the request inside a packed score buffer
+};
+
+// Shape data common to all kernels; passed by value.
+struct Shape {
+  int32_t dtype, n_layers, n_q_heads, n_kv_heads, head_dim, n_req, window, group;  // group = G
+  int32_t heads_per_req;  // N = n_layers * n_kv_heads
+  int32_t total_heads;    // n_req * N
+  int64_t q_stride_layer, q_stride_tok, q_stride_head;
+  int64_t kv_stride_layer, kv_stride_tok, kv_stride_head;
+  float scale_log2e;  // softmax_scale * log2(e): logits are taken to base 2
+  float softmax_scale;
+  float rho, alpha;
+  int32_t transition_bins, base_per_head;
+};
+
+// Maps a flat head index to (request, layer, kv head). n_req is small: linear search.
+__device__ __forceinline__ int find_req(const ReqDesc* __restrict__ reqs, int n_req, int heads_per_req, int u) {
+  int r = u / heads_per_req;
+  return r < n_req ? r : n_req - 1;
+}
+
+// ---- FFT plans -------------------------------------------------------------------------
+constexpr int kMaxRadices = 20;
+
+// How one complex transform of length N is carried out (Stockham passes over `radix`).
+struct FftSeq {
+  int32_t N;
+  int32_t n_pass;
+  int32_t radix[kMaxRadices];
+  int64_t tw_offset;  // float2 index of W_N^t, t in [0, N), inside the table area
+};
+
+// Plan for a real sequence of length n (one per distinct prefix length in the batch).
+struct FftPlan {
+  int32_t n;         // real length
+  int32_t packed;    // 1: n even, transform z_m = x_2m + i x_2m+1 of length n/2; 0: length n with zero imaginary part
+  int32_t N;         // complex transform length (n/2 or n)
+  int32_t bluestein; // 1: N goes through a chirp-z convolution of length M (a power of two)
+  int32_t M;         // convolution length (bluestein only)
+  int32_t in_smem;   // 1: the work buffer fits in shared memory
+  FftSeq seq;        // passes for length N (direct) or M (bluestein)
+  int64_t chirp_offset;   // float2 index of c_j = exp(-i pi j^2 / N), j in [0, N)      (bluestein)
+  int64_t filter_offset;  // float2 index of FFT_M of the wrapped conjugate chirp / M    (bluestein)
+  int64_t post_offset;    // float2 index of exp(-2 pi i k / n), k in [0, N/2]           (packed)
+};
+
+constexpr int kMaxPlans = AUDIOKV_MAX_REQ;
+
+// ---- launchers (one per source file) ---------------------------------------------------
+struct Launch {
+  cudaStream_t stream;
+  int64_t* launch_counter;
+};
+
+// score_simt.cu: fp32-FMA scoring for any dtype. stats_ws: float2 [total_heads][n_slab][rows].
+cudaError_t launch_score_simt(const Shape& sh, const ReqDesc* d_reqs, const void* q, const void* k, float* scores,
+                              float2* stats_ws, int n_slab, int slab_keys, Launch ln);
+
+// sss.cu
+cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);
+cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_plans, const float2* d_tables,
+                       const float* scores, float* smoothed, int32_t* kstar, float2* scratch,
+                       int64_t scratch_per_block, int grid, size_t smem_bytes, Launch ln);
+
+// allocate.cu (h_total_budget: host array [n_req])
+cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float* head_scores,
+                            const int64_t* h_total_budget, int32_t* budgets, int32_t* cu_kept, int* status,
+                            Launch ln);
+
+// select_gather.cu
+cudaError_t launch_select(const Shape& sh, const ReqDesc* d_reqs, const float* smoothed, const int32_t* budgets,
+                          const int32_t* cu_kept, int32_t* kept_idx, int max_P, int* status, Launch ln);
+cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t* cu_kept, const int32_t* kept_idx,
+                          const void* k, const void* v, void* k_out, void* v_out, Launch ln);
+
+}  // namespace akv

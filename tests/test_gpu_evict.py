@@ -1,0 +1,156 @@
+"""GPU parity of the whole pass (audiokv_evict and its host-buffer variant) against the oracle."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_06694_b200 import workloads as wl
+from helpers import KSTAR_TIE, check_kept, oracle_dtype, request_views, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2604_06694_b200 import build as akv_build
+    akv_build.build()
+    from paper_2604_06694_b200 import binding
+    return binding
+
+
+def run_evict(B, w, host=False, **over):
+    prob = B.Problem.from_workload(w, **over)
+    s = w.spec
+    TH = prob.total_heads
+    rows = int(w.total_budget.sum())
+    tb = [int(x) for x in w.total_budget]
+    es = w.torch_dtype()
+    dev = "cpu" if host else "cuda"
+    k_out = torch.zeros((rows, s.head_dim), dtype=es, device=dev)
+    v_out = torch.zeros((rows, s.head_dim), dtype=es, device=dev)
+    kept = torch.full((rows,), -1, dtype=torch.int32, device=dev)
+    budgets = torch.zeros(TH, dtype=torch.int32, device=dev)
+    cu = torch.zeros(TH + 1, dtype=torch.int32, device=dev)
+    S = torch.from_numpy(w.head_scores)
+    if host:
+        ws = B.audiokv_workspace_bytes_host(prob, w.q.size, w.k.size, tb)
+        ctx = B.Context(prob, workspace_bytes=ws)
+        B.audiokv_evict_host(ctx, prob, w.as_torch(w.q), w.as_torch(w.k), w.as_torch(w.v), S, tb, k_out, v_out, kept,
+                             budgets, cu)
+    else:
+        ctx = B.Context(prob)
+        B.audiokv_evict(ctx, prob, to_dev(w, w.q), to_dev(w, w.k), to_dev(w, w.v), S.cuda(), tb, k_out, v_out, kept,
+                        budgets, cu)
+        torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    raw = lambda t: t.cpu().view(torch.uint16 if s.dtype == "bf16" else torch.float32).numpy()
+    return dict(k_out=raw(k_out), v_out=raw(v_out), kept=kept.cpu().numpy(), budgets=budgets.cpu().numpy(),
+                cu=cu.cpu().numpy(), launches=ctx.launch_count())
+
+
+def check_against_oracle(w, g, scale=None):
+    """Budgets bit-exact; kept sets equal up to near ties; K/V rows bit-exact given the GPU's indices."""
+    s = w.spec
+    N = s.n_layers * s.n_kv_heads
+    W = s.window
+    n_tie_tokens = 0
+    assert np.array_equal(g["cu"], np.concatenate([[0], np.cumsum(g["budgets"])]))
+    for r, L in enumerate(s.seq_lens):
+        q, k, v, dims, qs, kvs, _ = request_views(w, r)
+        P = L - W
+        res = oracle.evict_request(q, k, v, oracle_dtype(w), dims, qs, kvs, scale or 1.0 / np.sqrt(s.head_dim),
+                                   w.head_scores[r], int(w.total_budget[r]), w.base, float(np.float32(s.rho)),
+                                   float(np.float32(s.alpha)), s.transition_bins)
+        assert np.array_equal(g["budgets"][r * N:(r + 1) * N], res["budgets"].reshape(-1)), f"budgets of request {r}"
+        for l in range(s.n_layers):
+            for h in range(s.n_kv_heads):
+                u = r * N + l * s.n_kv_heads + h
+                a, b = g["cu"][u], g["cu"][u + 1]
+                idx = g["kept"][a:b]
+                n_tie_tokens += check_kept(idx, res["smoothed"][l, h], int(res["budgets"][l, h]) - W, P, W,
+                                           f"req {r} layer {l} head {h}")
+                src_k = w.k[l, h, int(w.cu_seqlen[r]):int(w.cu_seqlen[r]) + L]
+                src_v = w.v[l, h, int(w.cu_seqlen[r]):int(w.cu_seqlen[r]) + L]
+                assert np.array_equal(g["k_out"][a:b], src_k[idx]) and np.array_equal(g["v_out"][a:b], src_v[idx])
+    return n_tie_tokens
+
+
+def test_evict_config1_full(B):
+    w = wl.generate(wl.config(0))
+    g = run_evict(B, w)
+    assert int(g["cu"][-1]) == int(0.4 * 2 * 1024)
+    check_against_oracle(w, g)
+
+
+def test_evict_config2_three_layers(B):
+    w = wl.generate(wl.config(1), layers=3)
+    ties = check_against_oracle(w, run_evict(B, w))
+    assert ties <= 8
+
+
+def test_evict_config4_one_layer_with_sinks(B):
+    w = wl.generate(wl.config(3), layers=1)
+    check_against_oracle(w, run_evict(B, w))
+
+
+def test_evict_ragged_batch_gemma_shape(B):
+    spec = dataclasses.replace(wl.config(4), seq_lens=[2048, 3333, 2500], audio_frac=[0.8, 0.95, 0.9])
+    w = wl.generate(spec, layers=2)
+    g = run_evict(B, w)
+    check_against_oracle(w, g)
+
+
+def test_evict_host_buffers_equal_device_buffers(B):
+    w = wl.generate(wl.config(0), seed=5)
+    a = run_evict(B, w)
+    b = run_evict(B, w, host=True)
+    for key in ("k_out", "v_out", "kept", "budgets", "cu"):
+        assert np.array_equal(a[key], b[key]), key
+
+
+def test_evict_is_deterministic(B):
+    w = wl.generate(wl.config(1), layers=1)
+    a, b = run_evict(B, w), run_evict(B, w)
+    for key in ("k_out", "v_out", "kept", "budgets", "cu"):
+        assert np.array_equal(a[key], b[key]), key
+
+
+def test_evict_degenerate_budgets(B):
+    # window only (nothing kept from the prefix) and everything kept
+    w = wl.generate(wl.config(0))
+    N, L, W = 2, 1024, 32
+    w.base = 0
+    w.total_budget[:] = N * W
+    g = run_evict(B, w)
+    assert list(g["budgets"]) == [W, W] and np.array_equal(g["kept"], np.tile(np.arange(L - W, L), 2))
+    w.total_budget[:] = N * L
+    g = run_evict(B, w)
+    assert list(g["budgets"]) == [L, L] and np.array_equal(g["kept"], np.tile(np.arange(L), 2))
+    assert np.array_equal(g["k_out"].reshape(2, L, 64), w.k[0])
+
+
+def test_evict_without_smoothing_and_uniform_heads(B):
+    # alpha = 0 is the method without SSS; equal head scores give the uniform allocation
+    w = wl.generate(wl.config(0), seed=2)
+    w.head_scores[:] = 0.5
+    w.spec.alpha = 0.0
+    g = run_evict(B, w)
+    assert abs(int(g["budgets"][0]) - int(g["budgets"][1])) <= 1
+    check_against_oracle(w, g)
+
+
+def test_rejections(B):
+    w = wl.generate(wl.config(0))
+    prob = B.Problem.from_workload(w)
+    ctx = B.Context(prob, workspace_bytes=4096)
+    scores = torch.zeros(B.audiokv_scores_len(prob), device="cuda")
+    with pytest.raises(B.AudioKVError) as e:
+        B.audiokv_score(ctx, prob, to_dev(w, w.q), to_dev(w, w.k), scores)
+    assert e.value.status == B.AUDIOKV_EWORKSPACE
+    ctx = B.Context(prob)
+    kd = to_dev(w, w.k)
+    with pytest.raises(B.AudioKVError) as e:
+        B.audiokv_score(ctx, prob, to_dev(w, w.q), kd.reshape(-1)[1:], scores)      # misaligned K
+    assert e.value.status == B.AUDIOKV_EALIGN
