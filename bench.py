@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the AudioKV eviction pass: one step = one audiokv_evict call over the whole
+attention stack of the Qwen2.5-Omni-7B-shaped workload (28 layers, L = 8192).
+
+Prints ONE JSON line (rank 0). `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2604_06694_b200 import workloads as wl  # noqa: E402
+
+METRIC = "evict_pass_us_per_layer"
+UNIT = "us/layer"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+# DRAM bytes per launch (read + write) of each kernel at this workload, from the ncu captures summarised
+# under profiles/ (see the file named there); None where no capture has been taken yet.
+NCU_TRAFFIC_BYTES = {}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def contract_bytes_per_layer(spec, L):
+    """K read once plus kept K and V written (the roofline the benchmark spec defines)."""
+    e = 4 if spec.dtype == "f32" else 2
+    row = spec.n_kv_heads * spec.head_dim * e
+    return L * row + 2 * int(spec.keep * L) * row
+
+
+def kernel_algorithmic_bytes(name, spec, w):
+    """Bytes each kernel must move per launch at this workload (what it reads once plus what it writes)."""
+    e = 4 if spec.dtype == "f32" else 2
+    NL, Hkv, d, W, Hq = spec.n_layers, spec.n_kv_heads, spec.head_dim, spec.window, spec.n_q_heads
+    sumL = int(w.cu_seqlen[-1])
+    k_bytes = NL * Hkv * sumL * d * e
+    q_bytes = len(spec.seq_lens) * NL * W * Hq * d * e
+    score_bytes = 4 * NL * Hkv * (sumL - W * len(spec.seq_lens))
+    kept_rows = int(w.total_budget.sum())
+    if name.startswith("score") and "stats" in name:
+        return k_bytes + q_bytes
+    if name.startswith("score"):
+        return k_bytes + q_bytes + score_bytes
+    if name == "sss":
+        return 2 * score_bytes
+    if name == "select":
+        return score_bytes + 4 * kept_rows
+    if name == "gather":
+        return kept_rows * (4 + 4 * d * e)           # index + K,V row read + K,V row written
+    return 0
+
+
+def run_cuda(args):
+    from paper_2604_06694_b200 import binding as B
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    spec = wl.config(1)
+    w = wl.generate(spec, seed=rank)          # every rank evicts its own request: no exchange step
+    L = spec.seq_lens[0]
+    prob = B.Problem.from_workload(w)
+    tb = [int(x) for x in w.total_budget]
+    rows, TH = sum(tb), prob.total_heads
+    es = w.torch_dtype()
+
+    q, k, v = (w.as_torch(a).cuda() for a in (w.q, w.k, w.v))
+    S = torch.from_numpy(w.head_scores).cuda()
+    k_out = torch.empty((rows, spec.head_dim), dtype=es, device="cuda")
+    v_out = torch.empty_like(k_out)
+    kept = torch.empty(rows, dtype=torch.int32, device="cuda")
+    budgets = torch.empty(TH, dtype=torch.int32, device="cuda")
+    cu = torch.empty(TH + 1, dtype=torch.int32, device="cuda")
+    ws_host = B.audiokv_workspace_bytes_host(prob, w.q.size, w.k.size, tb)
+    ctx = B.Context(prob, device=local, workspace_bytes=ws_host)
+
+    def step():
+        B.audiokv_evict(ctx, prob, q, k, v, S, tb, k_out, v_out, kept, budgets, cu)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    n0 = ctx.launch_count()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    launches = ctx.launch_count() - n0
+    ms_total = e0.elapsed_time(e1)
+    t = torch.tensor([ms_total], device="cuda")
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    clocks = sampler.stop() if sampler else None
+    assert ctx.last_device_status() == 0
+
+    # per-kernel durations: the same loop again with an event after every kernel
+    ctx.profile_enable(True)
+    per_kernel = {}
+    for _ in range(args.steps):
+        step()
+        for name, ms in ctx.profile_read():
+            per_kernel.setdefault(name, []).append(ms)
+    ctx.profile_enable(False)
+    torch.cuda.synchronize()
+
+    # end to end through the host-buffer entry point: pinned host inputs, results read back
+    hq, hk, hv = (w.as_torch(a).pin_memory() for a in (w.q, w.k, w.v))
+    hS = torch.from_numpy(w.head_scores).pin_memory()
+    hko = torch.empty((rows, spec.head_dim), dtype=es).pin_memory()
+    hvo = torch.empty_like(hko).pin_memory()
+    hkept = torch.empty(rows, dtype=torch.int32).pin_memory()
+    hb = torch.empty(TH, dtype=torch.int32).pin_memory()
+    hcu = torch.empty(TH + 1, dtype=torch.int32).pin_memory()
+
+    def step_host():
+        B.audiokv_evict_host(ctx, prob, hq, hk, hv, hS, tb, hko, hvo, hkept, hb, hcu)
+
+    step_host()
+    barrier()
+    n_e2e = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(n_e2e):
+        step_host()
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+    t = torch.tensor([e2e_ms], device="cuda")
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    e2e_ms = float(t.item())
+    h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv, hS))
+    d2h = sum(x.numel() * x.element_size() for x in (hko, hvo, hkept, hb, hcu))
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+    NL = spec.n_layers
+    peaks, peak_kind = measured_peaks()
+    us_layer = ms_step * 1e3 / (NL * world)
+    cbytes = contract_bytes_per_layer(spec, L)
+    hbm_gbs = cbytes * NL * world / (ms_step * 1e-3) / 1e9
+    kern = {n: statistics.mean(v) for n, v in per_kernel.items()}
+    tot = sum(kern.values()) or 1.0
+    dom = max(kern, key=kern.get)
+    dom_bytes = kernel_algorithmic_bytes(dom, spec, w)
+    achieved = dom_bytes / (kern[dom] * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": round(us_layer, 4), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "layers": NL, "q_heads": spec.n_q_heads, "kv_heads": spec.n_kv_heads,
+                   "head_dim": spec.head_dim, "L": L, "window": spec.window, "keep": spec.keep,
+                   "requests_per_gpu": 1, "l2": "inputs larger than L2 (K+V of a step = %d MB)" % (2 * w.k.nbytes // 2**20),
+                   "parallelism": f"replicas x{world}, no collective"},
+        "tokens_heads_per_s": round(L * spec.n_kv_heads * NL * world / (ms_step * 1e-3), 1),
+        "hbm_gbs": round(hbm_gbs, 1),
+        "hbm_frac_of_nominal_8tbs": round(hbm_gbs / NOMINAL_HBM_GBS, 4),
+        "hbm_frac_of_measured": round(hbm_gbs / peaks["hbm_gbs"], 4),
+        "contract_bytes_per_layer": cbytes,
+        "gpu_launches": int(launches),
+        "kernels_ms": {n: round(v, 5) for n, v in kern.items()},
+        "kernel_share": {n: round(v / tot, 4) for n, v in kern.items()},
+        "roofline": {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4), "peak_kind": peak_kind,
+                     "algorithmic_bytes": dom_bytes, "traffic": NCU_TRAFFIC_BYTES.get(dom)},
+        "e2e": {"value": round(e2e_ms * 1e3 / (NL * world), 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+        "clocks": clocks,
+    }
+    if not args.skip_cpu:
+        line["cpu_baseline"] = cpu_baseline(w, spec, budget_s=15.0)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def oracle_pass(w, spec, n_layers):
+    """The oracle's whole pass over the first n_layers layers of request 0; returns seconds."""
+    import oracle
+    L = spec.seq_lens[0]
+    dims = (n_layers, spec.window, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, L)
+    N = n_layers * spec.n_kv_heads
+    Bt = int(np.floor(spec.keep * N * L))
+    t0 = time.perf_counter()
+    oracle.evict_request(w.q[0], w.k, w.v, oracle.BF16, dims, w.q_strides()[1:], w.kv_strides(),
+                         1.0 / np.sqrt(spec.head_dim), w.head_scores[0, :n_layers], Bt, w.base,
+                         float(np.float32(spec.rho)), float(np.float32(spec.alpha)), spec.transition_bins)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(w, spec, budget_s):
+    """The oracle, as it stands, on the host cores: a bounded sample (the first layers) of the same workload."""
+    cores = os.cpu_count() or 1
+    t1 = oracle_pass(w, spec, 1)
+    n = int(max(1, min(spec.n_layers, budget_s / max(t1, 1e-3))))
+    t = oracle_pass(w, spec, n)
+    return {"value": round(t * 1e6 / n, 1), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n} of {spec.n_layers} layers of the same workload, all steps of the pass, OpenMP over heads"}
+
+
+def run_reference(args):
+    """The reference arm for this repository is the CPU oracle (there is no reference implementation to install)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    spec = wl.config(1)
+    sample_layers = 4
+    w = wl.generate(spec, seed=0, layers=sample_layers)
+    for _ in range(max(args.warmup, 1)):
+        oracle_pass(w, spec, sample_layers)
+    ts = [oracle_pass(w, spec, sample_layers) for _ in range(args.steps)]
+    sec = sum(ts) / len(ts)
+    us_layer = sec * 1e6 / sample_layers
+    cores = os.cpu_count() or 1
+    sample = f"each step = the first {sample_layers} of {spec.n_layers} layers (all four steps of the pass)"
+    line = {"impl": "reference", "metric": METRIC, "value": round(us_layer, 1), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": round(sec * 1e3, 3),
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": spec.name, "layers": spec.n_layers, "L": spec.seq_lens[0], "window": spec.window,
+                       "keep": spec.keep, "sample": sample},
+            "cpu_baseline": {"value": round(us_layer, 1), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(us_layer, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline (profiling runs)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

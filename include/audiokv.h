@@ -120,6 +120,17 @@ const char* audiokv_last_cuda_error(const audiokv_ctx* ctx);
 /* Kernels launched by calls on this context since it was created (for accounting). */
 int64_t audiokv_launch_count(const audiokv_ctx* ctx);
 
+/* Per-kernel timing of audiokv_evict, for benchmarks. While enabled, every audiokv_evict call
+ * on this context records a CUDA event on its stream after each kernel it launches (creating
+ * the events on the first enable). After the call, kernel i of the call (0 <= i <
+ * audiokv_profile_count) has the name audiokv_profile_name(ctx, i) and took
+ * audiokv_profile_ms(ctx, i) milliseconds from the end of the kernel before it (blocks until
+ * that kernel has finished; -1 on error). Off by default. */
+int audiokv_profile_enable(audiokv_ctx* ctx, int on);
+int audiokv_profile_count(const audiokv_ctx* ctx);
+const char* audiokv_profile_name(const audiokv_ctx* ctx, int i);
+float audiokv_profile_ms(audiokv_ctx* ctx, int i);
+
 /* ---- the four steps ------------------------------------------------------------------- */
 
 /* Step 1 -- importance scores (Section 3.3, importance sequence over the decoding window).

@@ -72,6 +72,14 @@ def lib() -> ctypes.CDLL:
         L.audiokv_last_cuda_error.argtypes = [vp]
         L.audiokv_launch_count.restype = i64
         L.audiokv_launch_count.argtypes = [vp]
+        L.audiokv_profile_enable.argtypes = [vp, ctypes.c_int]
+        L.audiokv_profile_enable.restype = ctypes.c_int
+        L.audiokv_profile_count.argtypes = [vp]
+        L.audiokv_profile_count.restype = ctypes.c_int
+        L.audiokv_profile_name.argtypes = [vp, ctypes.c_int]
+        L.audiokv_profile_name.restype = ctypes.c_char_p
+        L.audiokv_profile_ms.argtypes = [vp, ctypes.c_int]
+        L.audiokv_profile_ms.restype = ctypes.c_float
         L.audiokv_score.argtypes = [vp, pp, vp, vp, vp, vp]
         L.audiokv_smooth.argtypes = [vp, pp, vp, vp, vp, vp]
         L.audiokv_allocate.argtypes = [vp, pp, vp, ctypes.POINTER(i64), vp, vp, vp]
@@ -193,6 +201,15 @@ class Context:
 
     def launch_count(self) -> int:
         return int(lib().audiokv_launch_count(self.h))
+
+    def profile_enable(self, on: bool) -> None:
+        self._check(lib().audiokv_profile_enable(self.h, int(on)), "audiokv_profile_enable")
+
+    def profile_read(self):
+        """[(kernel name, milliseconds)] of the last audiokv_evict call made while profiling was on."""
+        n = lib().audiokv_profile_count(self.h)
+        return [(lib().audiokv_profile_name(self.h, i).decode(), float(lib().audiokv_profile_ms(self.h, i)))
+                for i in range(n)]
 
     def last_device_status(self) -> int:
         return int(lib().audiokv_last_device_status(self.h, _stream()))

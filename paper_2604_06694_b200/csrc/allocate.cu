@@ -176,8 +176,9 @@ cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float*
   cudaError_t e = cudaFuncSetAttribute(allocate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   allocate_kernel<<<sh.n_req, kAllocThreads, smem, ln.stream>>>(sh, d_reqs, head_scores, args, budgets, status);
+  ln.done("allocate");
   cu_kept_kernel<<<1, 1024, 0, ln.stream>>>(budgets, sh.total_heads, cu_kept);
-  *ln.launch_counter += 2;
+  ln.done("cu_kept");
   return cudaGetLastError();
 }
 

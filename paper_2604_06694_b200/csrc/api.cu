@@ -52,6 +52,7 @@ struct audiokv_ctx {
   bool plan_uploaded = false;
   cudaEvent_t plan_ready = nullptr;
   int64_t launches = 0;
+  Profiler prof;
   std::string cuda_error;
 };
 
@@ -282,7 +283,7 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
     if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.plans, pl.fft.data(), sizeof(FftPlan) * pl.fft.size(),
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess)
       return cuda_fail(ctx, e);
-    Launch ln{stream, &ctx->launches};
+    Launch ln{stream, &ctx->launches, &ctx->prof};
     e = launch_fft_tables(static_cast<int>(pl.fft.size()), reinterpret_cast<float2*>(ctx->ws + pl.lay.tables),
                           reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans), ln);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
@@ -294,12 +295,22 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
   return AUDIOKV_OK;
 }
 
+// Starts the per-kernel timing of one call (event 0), when profiling is on.
+void profile_begin(audiokv_ctx* ctx, cudaStream_t stream) {
+  Profiler& pf = ctx->prof;
+  if (!pf.on) return;
+  pf.n = 0;
+  cudaEventRecord(pf.ev[0], stream);
+  pf.name[0] = "begin";
+  pf.n = 1;
+}
+
 const ReqDesc* d_reqs(audiokv_ctx* c) { return reinterpret_cast<const ReqDesc*>(c->ws + c->plan.lay.reqs); }
 int* d_status(audiokv_ctx* c) { return reinterpret_cast<int*>(c->ws + c->plan.lay.status); }
 
 int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cudaStream_t stream) {
   Plan& pl = ctx->plan;
-  Launch ln{stream, &ctx->launches};
+  Launch ln{stream, &ctx->launches, &ctx->prof};
   cudaError_t e = launch_score_simt(pl.sh, d_reqs(ctx), q, k, scores, reinterpret_cast<float2*>(ctx->ws + pl.lay.stats),
                                     pl.n_slab, kSimtSlabKeys, ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
@@ -307,7 +318,7 @@ int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cuda
 
 int do_smooth(audiokv_ctx* ctx, const float* scores, float* smoothed, int32_t* kstar, cudaStream_t stream) {
   Plan& pl = ctx->plan;
-  Launch ln{stream, &ctx->launches};
+  Launch ln{stream, &ctx->launches, &ctx->prof};
   cudaError_t e = launch_sss(pl.sh, d_reqs(ctx), reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans),
                              reinterpret_cast<const float2*>(ctx->ws + pl.lay.tables), scores, smoothed, kstar,
                              reinterpret_cast<float2*>(ctx->ws + pl.lay.fft_scratch), pl.scratch_per_block,
@@ -330,7 +341,7 @@ int do_allocate(audiokv_ctx* ctx, const float* head_scores, const int64_t* total
   Plan& pl = ctx->plan;
   int rc = check_budgets(pl, total_budget);
   if (rc) return rc;
-  Launch ln{stream, &ctx->launches};
+  Launch ln{stream, &ctx->launches, &ctx->prof};
   cudaError_t e = launch_allocate(pl.sh, d_reqs(ctx), head_scores, total_budget, budgets, cu_kept, d_status(ctx), ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
@@ -338,7 +349,7 @@ int do_allocate(audiokv_ctx* ctx, const float* head_scores, const int64_t* total
 int do_select_gather(audiokv_ctx* ctx, const float* smoothed, const int32_t* budgets, const int32_t* cu_kept,
                      const void* k, const void* v, void* k_out, void* v_out, int32_t* kept_idx, cudaStream_t stream) {
   Plan& pl = ctx->plan;
-  Launch ln{stream, &ctx->launches};
+  Launch ln{stream, &ctx->launches, &ctx->prof};
   cudaError_t e = launch_select(pl.sh, d_reqs(ctx), smoothed, budgets, cu_kept, kept_idx, pl.max_P, d_status(ctx), ln);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   e = launch_gather(pl.sh, d_reqs(ctx), cu_kept, kept_idx, k, v, k_out, v_out, ln);
@@ -429,6 +440,8 @@ int audiokv_destroy(audiokv_ctx* ctx) {
   if (!ctx) return AUDIOKV_EINVAL;
   cudaSetDevice(ctx->device);
   cudaEventDestroy(ctx->plan_ready);
+  for (cudaEvent_t e : ctx->prof.ev)
+    if (e) cudaEventDestroy(e);
   cudaFree(ctx->ws);
   delete ctx;
   return AUDIOKV_OK;
@@ -447,6 +460,34 @@ int audiokv_last_device_status(audiokv_ctx* ctx, audiokv_stream stream) {
 const char* audiokv_last_cuda_error(const audiokv_ctx* ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
 
 int64_t audiokv_launch_count(const audiokv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int audiokv_profile_enable(audiokv_ctx* ctx, int on) {
+  if (!ctx) return AUDIOKV_EINVAL;
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return AUDIOKV_ECUDA;
+  Profiler& pf = ctx->prof;
+  if (on && !pf.ev[0]) {
+    for (cudaEvent_t& e : pf.ev)
+      if (cudaEventCreate(&e) != cudaSuccess) return AUDIOKV_ECUDA;
+  }
+  pf.on = on != 0;
+  pf.n = 0;
+  return AUDIOKV_OK;
+}
+
+int audiokv_profile_count(const audiokv_ctx* ctx) { return ctx && ctx->prof.n > 0 ? ctx->prof.n - 1 : 0; }
+
+const char* audiokv_profile_name(const audiokv_ctx* ctx, int i) {
+  if (!ctx || i < 0 || i + 1 >= ctx->prof.n) return "";
+  return ctx->prof.name[i + 1];
+}
+
+float audiokv_profile_ms(audiokv_ctx* ctx, int i) {
+  if (!ctx || i < 0 || i + 1 >= ctx->prof.n) return -1.f;
+  float ms = -1.f;
+  if (cudaEventSynchronize(ctx->prof.ev[i + 1]) != cudaSuccess) return -1.f;
+  if (cudaEventElapsedTime(&ms, ctx->prof.ev[i], ctx->prof.ev[i + 1]) != cudaSuccess) return -1.f;
+  return ms;
+}
 
 int audiokv_score(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k, float* scores,
                   audiokv_stream stream) {
@@ -500,6 +541,7 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
   Plan& pl = ctx->plan;
   float* ws_scores = reinterpret_cast<float*>(ctx->ws + pl.lay.scores);
   int32_t* ws_kstar = reinterpret_cast<int32_t*>(ctx->ws + pl.lay.kstar);
+  profile_begin(ctx, s);
   if ((rc = do_allocate(ctx, head_scores, total_budget, budgets, cu_kept, s))) return rc;
   if ((rc = do_score(ctx, q_win, k, ws_scores, s))) return rc;
   if ((rc = do_smooth(ctx, ws_scores, ws_scores, ws_kstar, s))) return rc;

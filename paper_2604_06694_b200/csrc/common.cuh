@@ -67,9 +67,28 @@ struct FftPlan {
 constexpr int kMaxPlans = AUDIOKV_MAX_REQ;
 
 // ---- launchers (one per source file) ---------------------------------------------------
+// Optional per-kernel timing: an event after every kernel launch of one call.
+struct Profiler {
+  static constexpr int kMax = 32;
+  bool on = false;
+  int n = 0;                 // events recorded in the current call (event 0 = start of the call)
+  cudaEvent_t ev[kMax] = {};
+  const char* name[kMax] = {};
+};
+
 struct Launch {
   cudaStream_t stream;
   int64_t* launch_counter;
+  Profiler* prof;
+  // Counts one kernel launch and, when profiling, records the event that ends it.
+  void done(const char* kernel_name) const {
+    *launch_counter += 1;
+    if (prof && prof->on && prof->n < Profiler::kMax) {
+      cudaEventRecord(prof->ev[prof->n], stream);
+      prof->name[prof->n] = kernel_name;
+      prof->n += 1;
+    }
+  }
 };
 
 // score_simt.cu: fp32-FMA scoring for any dtype. stats_ws: float2 [total_heads][n_slab][rows].

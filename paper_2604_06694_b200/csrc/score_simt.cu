@@ -212,8 +212,9 @@ cudaError_t launch_typed(const Shape& sh, const ReqDesc* d_reqs, const void* q, 
   if ((e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   dim3 grid(n_slab, sh.total_heads);
   k1<<<grid, kThreads, smem, ln.stream>>>(sh, d_reqs, (const T*)q, (const T*)k, scores, stats_ws, n_slab, slab_keys);
+  ln.done("score_simt_stats");
   k2<<<grid, kThreads, smem, ln.stream>>>(sh, d_reqs, (const T*)q, (const T*)k, scores, stats_ws, n_slab, slab_keys);
-  *ln.launch_counter += 2;
+  ln.done("score_simt_colsum");
   return cudaGetLastError();
 }
 

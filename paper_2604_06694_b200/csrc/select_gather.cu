@@ -178,7 +178,7 @@ cudaError_t launch_select(const Shape& sh, const ReqDesc* d_reqs, const float* s
   const int grid = sh.total_heads < 148 * 4 ? sh.total_heads : 148 * 4;
   select_kernel<<<grid, kSelThreads, smem, ln.stream>>>(sh, d_reqs, smoothed, budgets, cu_kept, kept_idx, smem_keys,
                                                         status);
-  *ln.launch_counter += 1;
+  ln.done("select");
   return cudaGetLastError();
 }
 
@@ -189,7 +189,7 @@ cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t*
   const int chunks_per_row = sh.head_dim / elems_per_chunk;
   gather_kernel<<<148 * 8, 256, 0, ln.stream>>>(sh, d_reqs, cu_kept, kept_idx, (const uint4*)k, (const uint4*)v,
                                                  (uint4*)k_out, (uint4*)v_out, chunks_per_row, elems_per_chunk);
-  *ln.launch_counter += 1;
+  ln.done("gather");
   return cudaGetLastError();
 }
 

@@ -497,8 +497,9 @@ fft_filter_kernel(const FftPlan* __restrict__ plans, float2* __restrict__ tables
 
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln) {
   fft_table_kernel<<<dim3(32, n_plans), 256, 0, ln.stream>>>(d_plans, n_plans, d_tables);
+  ln.done("fft_table");
   fft_filter_kernel<<<n_plans, kSssThreads, 0, ln.stream>>>(d_plans, d_tables);
-  *ln.launch_counter += 2;
+  ln.done("fft_filter");
   return cudaGetLastError();
 }
 
@@ -509,7 +510,7 @@ cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_
   if (e != cudaSuccess) return e;
   sss_kernel<<<grid, kSssThreads, smem_bytes, ln.stream>>>(sh, d_reqs, d_plans, d_tables, scores, smoothed, kstar,
                                                            scratch, scratch_per_block);
-  *ln.launch_counter += 1;
+  ln.done("sss");
   return cudaGetLastError();
 }
 
