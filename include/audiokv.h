@@ -192,6 +192,27 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
 size_t audiokv_workspace_bytes_host(const audiokv_params* p, int64_t q_elems, int64_t kv_elems,
                                     const int64_t* total_budget);
 
+/* Step 1 for callers that cannot allocate device memory (the paper has no counterpart: this
+ * is a deployment variant of audiokv_score, same arguments and same result).
+ * Who needs it: code running under a memory pool or arena whose owner forbids cudaMalloc
+ * once serving has started, plug-ins that receive a stream and buffers but no allocator, and
+ * callers that must avoid the device-wide synchronisation an allocation may cause. It takes
+ * no context: its scratch (the per-slab softmax statistics and the request table) is a fixed
+ * 8 MiB array inside the library image, which every GPU that loads the library holds until
+ * the process exits. It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Limit: n_req * n_layers * n_kv_heads * ceil(max L / 512) * W * G * 8 bytes must fit in
+ *     8 MiB - 4 KiB (e.g. 28 layers x 4 KV heads at L = 8192, W = 32, G = 7 needs 3.1 MiB);
+ *     larger problems return AUDIOKV_EWORKSPACE. fp32 FMA arithmetic for both element types.
+ *   - The first call on a device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on one GPU share the array: two calls whose kernels may overlap on the GPU
+ *     (different streams without an ordering between them) race on it. Calls ordered on one
+ *     stream are safe; nothing needs clearing between calls, since the first kernel writes every
+ *     scratch entry the second one reads.
+ * device: CUDA device ordinal (made current). Other arguments as audiokv_score. */
+int audiokv_score_noalloc(int device, const audiokv_params* p, const void* q_win, const void* k, float* scores,
+                          audiokv_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

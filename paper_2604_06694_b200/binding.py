@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.audiokv_profile_ms.argtypes = [vp, ctypes.c_int]
         L.audiokv_profile_ms.restype = ctypes.c_float
         L.audiokv_score.argtypes = [vp, pp, vp, vp, vp, vp]
+        L.audiokv_score_noalloc.argtypes = [ctypes.c_int, pp, vp, vp, vp, vp]
+        L.audiokv_score_noalloc.restype = ctypes.c_int
         L.audiokv_smooth.argtypes = [vp, pp, vp, vp, vp, vp]
         L.audiokv_allocate.argtypes = [vp, pp, vp, ctypes.POINTER(i64), vp, vp, vp]
         L.audiokv_select_gather.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -218,6 +220,18 @@ class Context:
 def audiokv_score(ctx: Context, prob: Problem, q_win: torch.Tensor, k: torch.Tensor, scores: torch.Tensor) -> None:
     ctx._check(lib().audiokv_score(ctx.h, prob.ref, _dev(q_win, "q_win"), _dev(k, "k"), _dev(scores, "scores"),
                                    _stream()), "audiokv_score")
+
+
+def audiokv_score_noalloc(prob: Problem, q_win: torch.Tensor, k: torch.Tensor, scores: torch.Tensor,
+                          device: Optional[int] = None) -> None:
+    """audiokv_score for callers that may not allocate device memory: no context, the scratch is a fixed
+    8 MiB array inside the library (shared by all calls on the GPU, so keep calls ordered on one stream).
+    Raises AudioKVError(AUDIOKV_EWORKSPACE) when the problem needs more scratch than that."""
+    dev = q_win.device.index if device is None else device
+    rc = lib().audiokv_score_noalloc(dev, prob.ref, _dev(q_win, "q_win"), _dev(k, "k"), _dev(scores, "scores"),
+                                     _stream())
+    if rc != 0:
+        raise AudioKVError(rc, "audiokv_score_noalloc")
 
 
 def audiokv_smooth(ctx: Context, prob: Problem, scores: torch.Tensor, smoothed: torch.Tensor,

@@ -237,3 +237,120 @@ cudaError_t launch_score_simt(const Shape& sh, const ReqDesc* d_reqs, const void
 }
 
 }  // namespace akv
+
+// ---------------------------------------------------------------------------------------
+// Scoring without any allocation.
+//
+// Some hosts of this library may not allocate device memory at the moment they need the
+// scores: code that runs inside a memory-pool or arena whose owner forbids cudaMalloc once
+// serving has started, plug-ins that are handed a stream and buffers but no allocator, and
+// callers that must not risk the implicit device synchronisation an allocation can cause.
+// For them the scratch of the two-sweep scoring (the per-slab row statistics) and the small
+// request table live in one fixed array that is part of the library image: every GPU that
+// loads the library holds kNoAllocBytes of it until the process exits.
+#include <mutex>
+
+namespace akv {
+namespace {
+
+constexpr size_t kNoAllocBytes = 8u << 20;     // 8 MiB per GPU, fixed
+constexpr size_t kNoAllocTableBytes = 4096;    // request table at the front, statistics after it
+constexpr int kNoAllocMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+std::mutex g_noalloc_mu;
+void* g_noalloc_ptr[kNoAllocMaxDevices] = {};  // device address of the array, per device ordinal
+
+// The array's name is only a host-side handle; kernels need the address the runtime reports
+// for the current device.
+cudaError_t noalloc_scratch(int device, void** out) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  if (!g_noalloc_ptr[device]) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[device] = p;
+  }
+  *out = g_noalloc_ptr[device];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace akv
+
+extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const void* q_win, const void* k,
+                                     float* scores, audiokv_stream stream) {
+  using namespace akv;
+  if (!p || !p->seq_len || !q_win || !k || !scores) return AUDIOKV_EINVAL;
+  if (device < 0 || device >= kNoAllocMaxDevices) return AUDIOKV_EINVAL;
+  if (p->dtype != AUDIOKV_F32 && p->dtype != AUDIOKV_BF16) return AUDIOKV_EINVAL;
+  if (p->n_layers < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads) return AUDIOKV_EINVAL;
+  if (p->n_req < 1 || p->n_req > AUDIOKV_MAX_REQ || p->window < 1) return AUDIOKV_EINVAL;
+  if (p->head_dim != 64 && p->head_dim != 128 && p->head_dim != 256) return AUDIOKV_EUNSUPPORTED;
+  const int G = p->n_q_heads / p->n_kv_heads;
+  const int64_t R = static_cast<int64_t>(p->window) * G;
+  if (R > 1024) return AUDIOKV_EUNSUPPORTED;
+  const int per16 = p->dtype == AUDIOKV_F32 ? 4 : 8;
+  const int64_t strides[] = {p->q_stride_req, p->q_stride_layer, p->q_stride_tok, p->q_stride_head,
+                             p->kv_stride_layer, p->kv_stride_tok, p->kv_stride_head};
+  for (int64_t s : strides) {
+    if (s < 0) return AUDIOKV_EINVAL;
+    if (s % per16) return AUDIOKV_EALIGN;
+  }
+  if ((reinterpret_cast<uintptr_t>(q_win) | reinterpret_cast<uintptr_t>(k)) & 15u) return AUDIOKV_EALIGN;
+  static_assert(sizeof(ReqDesc) * AUDIOKV_MAX_REQ <= kNoAllocTableBytes, "request table must fit its slot");
+
+  Shape sh{};
+  sh.dtype = p->dtype;
+  sh.n_layers = p->n_layers;
+  sh.n_q_heads = p->n_q_heads;
+  sh.n_kv_heads = p->n_kv_heads;
+  sh.head_dim = p->head_dim;
+  sh.n_req = p->n_req;
+  sh.window = p->window;
+  sh.group = G;
+  sh.heads_per_req = p->n_layers * p->n_kv_heads;
+  sh.total_heads = sh.heads_per_req * p->n_req;
+  sh.q_stride_layer = p->q_stride_layer;
+  sh.q_stride_tok = p->q_stride_tok;
+  sh.q_stride_head = p->q_stride_head;
+  sh.kv_stride_layer = p->kv_stride_layer;
+  sh.kv_stride_tok = p->kv_stride_tok;
+  sh.kv_stride_head = p->kv_stride_head;
+  sh.softmax_scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(static_cast<float>(p->head_dim));
+  sh.scale_log2e = static_cast<float>(static_cast<double>(sh.softmax_scale) * 1.4426950408889634);
+
+  ReqDesc reqs[AUDIOKV_MAX_REQ];
+  int max_L = 0;
+  int64_t score_off = 0;
+  for (int r = 0; r < p->n_req; ++r) {
+    const int L = p->seq_len[r];
+    if (L <= p->window || L > AUDIOKV_MAX_SEQ_LEN) return AUDIOKV_EINVAL;
+    const int64_t off = p->kv_req_offset ? p->kv_req_offset[r] : 0;
+    if (off < 0) return AUDIOKV_EINVAL;
+    if (off % per16) return AUDIOKV_EALIGN;
+    reqs[r] = ReqDesc{L, L - p->window, r * sh.heads_per_req, 0, off, r * p->q_stride_req, score_off};
+    score_off += static_cast<int64_t>(sh.heads_per_req) * (L - p->window);
+    max_L = L > max_L ? L : max_L;
+  }
+  constexpr int kSlabKeys = 512;
+  const int n_slab = (max_L + kSlabKeys - 1) / kSlabKeys;
+  const size_t need = sizeof(float2) * static_cast<size_t>(sh.total_heads) * n_slab * static_cast<size_t>(R);
+  if (need > kNoAllocBytes - kNoAllocTableBytes) return AUDIOKV_EWORKSPACE;  // beyond the fixed scratch
+
+  if (cudaSetDevice(device) != cudaSuccess) return AUDIOKV_ECUDA;
+  void* base = nullptr;
+  if (noalloc_scratch(device, &base) != cudaSuccess) return AUDIOKV_ECUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The table is staged by the runtime before this returns, so the local array may go out of scope.
+  if (cudaMemcpyAsync(base, reqs, sizeof(ReqDesc) * p->n_req, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return AUDIOKV_ECUDA;
+  int64_t launches = 0;
+  Launch ln{s, &launches, nullptr};
+  // Sweep 1 writes every statistics entry that sweep 2 reads, so nothing has to start at zero.
+  cudaError_t e = launch_score_simt(sh, static_cast<const ReqDesc*>(base), q_win, k, scores,
+                                    reinterpret_cast<float2*>(static_cast<unsigned char*>(base) + kNoAllocTableBytes),
+                                    n_slab, kSlabKeys, ln);
+  return e == cudaSuccess ? AUDIOKV_OK : AUDIOKV_ECUDA;
+}
