@@ -14,7 +14,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kSssSmemComplex = 25600;  // 200 KB of float2: the largest work buffer kept in shared memory
-constexpr int kSimtSlabKeys = 512;
+constexpr int kSlabKeys = 256;          // keys per slab of the softmax statistics (two K tiles of the tensor-core kernel)
 constexpr int kMaxRows = 1024;          // W * G
 constexpr int kMaxHeadsPerReq = 2048;
 
@@ -230,7 +230,7 @@ int build_plan(const audiokv_params* p, Plan* pl) {
     }
     d.fft_plan = found;
   }
-  pl->n_slab = (pl->max_L + kSimtSlabKeys - 1) / kSimtSlabKeys;
+  pl->n_slab = (pl->max_L + kSlabKeys - 1) / kSlabKeys;
   pl->sss_grid = sh.total_heads < 148 ? sh.total_heads : 148;
   int smem_c = 2;
   pl->scratch_per_block = 0;
@@ -311,8 +311,13 @@ int* d_status(audiokv_ctx* c) { return reinterpret_cast<int*>(c->ws + c->plan.la
 int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cudaStream_t stream) {
   Plan& pl = ctx->plan;
   Launch ln{stream, &ctx->launches, &ctx->prof};
-  cudaError_t e = launch_score_simt(pl.sh, d_reqs(ctx), q, k, scores, reinterpret_cast<float2*>(ctx->ws + pl.lay.stats),
-                                    pl.n_slab, kSimtSlabKeys, ln);
+  float2* stats = reinterpret_cast<float2*>(ctx->ws + pl.lay.stats);
+  cudaError_t e = cudaErrorNotSupported;
+  if (score_umma_takes(pl.sh))
+    e = launch_score_umma(pl.sh, pl.reqs.data(), d_reqs(ctx), q, k, scores, stats, pl.n_slab, kSlabKeys,
+                          d_status(ctx), ln);
+  if (e == cudaErrorNotSupported)  // fp32 inputs, W * G above 256, or strides the copy engine cannot take
+    e = launch_score_simt(pl.sh, d_reqs(ctx), q, k, scores, stats, pl.n_slab, kSlabKeys, ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 

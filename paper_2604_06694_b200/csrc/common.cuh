@@ -95,6 +95,15 @@ struct Launch {
 cudaError_t launch_score_simt(const Shape& sh, const ReqDesc* d_reqs, const void* q, const void* k, float* scores,
                               float2* stats_ws, int n_slab, int slab_keys, Launch ln);
 
+// score_umma.cu: bf16 scoring on the tcgen05 tensor cores (same statistics buffer). score_umma_takes says
+// whether the shape fits the kernel; the launcher returns cudaErrorNotSupported when the strides
+// cannot be described to the copy engine, and the caller then scores with launch_score_simt.
+// h_reqs: host copy of the request table (the tensor maps are encoded on the host).
+bool score_umma_takes(const Shape& sh);
+cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ReqDesc* d_reqs, const void* q,
+                              const void* k, float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status,
+                              Launch ln);
+
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);
 cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_plans, const float2* d_tables,

@@ -1,0 +1,681 @@
+// Importance scores for bf16 inputs on the tcgen05 tensor cores (sm_100a).
+//
+// The score of key j is the sum, over the W window rows and the G query heads of a KV
+// head, of softmax probabilities. A column sum mixes rows with different normalisers,
+// so the keys are swept twice:
+//   sweep 1  D[row][key]  = Q K^T  (query rows on the TMEM lanes): every thread owns one
+//            row and keeps its running maximum and sum of exp2 over the keys of a slab;
+//            one (max, sum) pair per (head, slab, row) goes to the statistics buffer.
+//   sweep 2  D[key][row]  = K Q^T  (keys on the TMEM lanes): every thread owns one key
+//            and adds exp2(z - max - log2 sum) over the rows; no cross-thread reduction.
+// Both sweeps are one persistent kernel (one CTA per SM) with three roles:
+//   warp 8    TMA producer: the Q tile of a head once, K tiles of 128 keys through a ring;
+//   warp 9    MMA issuer: tcgen05.mma, bf16 x bf16 -> fp32 in TMEM, two accumulator buffers;
+//   warps 0-7 two groups of 128 threads that read the accumulators (tcgen05.ld) and do the
+//             softmax arithmetic.
+// Q and K tiles are K-major with the 128-byte swizzle, so the same shared-memory tile is
+// the A operand of one sweep and the B operand of the other.
+// Every wait on an mbarrier is bounded: when one runs out the CTA stops, the kernel
+// writes AUDIOKV_ETIMEOUT to the status word and returns with its TMEM released.
+#include <cuda.h>
+#include <stddef.h>
+
+#include "common.cuh"
+
+namespace akv {
+namespace {
+
+constexpr int kTileKeys = 128;    // keys per K tile (UMMA M in sweep 2, N in sweep 1)
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr int kThreads = 320;
+constexpr int kAccCols = 256;     // TMEM columns of one accumulator buffer
+constexpr uint32_t kTmemCols = 512;
+constexpr int kMaxStages = 8;
+constexpr long long kWaitCycles = 2000000000LL;  // about one second
+constexpr int kSmemLimit = 232448;               // 227 KB
+
+struct TmapPack {
+  CUtensorMap q;                   // 5-D: (d, query head, window row, layer, request)
+  CUtensorMap k[AUDIOKV_MAX_REQ];  // 4-D per request: (d, token, KV head, layer)
+};
+
+struct UmmaArgs {
+  Shape sh;
+  const ReqDesc* reqs;
+  float2* stats;
+  float* scores;
+  int* status;
+  int n_slab;     // slabs per head in the statistics buffer
+  int slab_keys;  // keys per slab, a multiple of kTileKeys
+  int n_units;    // (head, slab) units of this sweep
+  int q_rows;     // rows of the Q tile in shared memory: 128 or 256
+  int r_pad;      // W * G rounded up to 16
+  int n_stages;   // K ring depth
+};
+
+struct Small {
+  alignas(16) float negc[2][2][256];  // sweep 2: -(max + log2 sum) per row; one copy per group and head parity (read as float4)
+  alignas(16) float2 mrg[2][128];     // sweep 1, one row block: the second group's partial statistics
+  alignas(16) ReqDesc reqs[AUDIOKV_MAX_REQ];
+  alignas(8) uint64_t k_full[kMaxStages];
+  uint64_t k_empty[kMaxStages];
+  uint64_t q_full, q_empty;
+  uint64_t acc_full[2], acc_empty[2];
+  uint64_t grp_bar[2];  // one per epilogue group (128 arrivals)
+  uint64_t all_bar;     // both groups (256 arrivals)
+  uint64_t drain;       // stop path only: the MMAs still in flight
+  uint32_t tmem_base;
+  int abort;
+};
+static_assert(offsetof(Small, negc) % 16 == 0 && offsetof(Small, k_full) % 8 == 0, "alignment of the small shared area");
+
+// ---- PTX wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait. Returns false when the CTA is stopping (this or another wait ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort,
+                                          long long limit = kWaitCycles) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 63u) == 0) {
+      if (*abort) return false;
+      if (clock64() - t0 > limit) {
+        *abort = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], "
+      "[%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile with the 128-byte swizzle: rows of
+// 128 bytes, groups of 8 rows 1024 bytes apart. `saddr` may point 32 * k bytes into the
+// first row to select the k-th slice of 16 elements along K.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  uint64_t d = static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);  // start address
+  d |= static_cast<uint64_t>(1) << 16;                          // leading-dimension offset (unused here)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                  // stride between 8-row groups
+  d |= static_cast<uint64_t>(1) << 46;                          // descriptor version of sm_100
+  d |= static_cast<uint64_t>(2) << 61;                          // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, tile M x N.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) |
+         (static_cast<uint32_t>(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The mbarrier gets one arrival when every MMA issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 (16) consecutive fp32 columns of this thread's TMEM lane; returns when the data is in registers.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      "tcgen05.wait::ld.sync.aligned;\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+      "tcgen05.wait::ld.sync.aligned;\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---- schedule ----------------------------------------------------------------------------
+// A unit is one slab of one head. Units are numbered request by request, head by head.
+struct Unit {
+  int u, r, l, h, slab, kt0, n_tiles, P;
+};
+template <int SWEEP>
+__device__ __forceinline__ Unit decode_unit(const Shape& sh, const ReqDesc* reqs, int idx, int slab_keys) {
+  Unit U{};
+  int base = 0;
+  for (int r = 0; r < sh.n_req; ++r) {
+    const int range = SWEEP == 1 ? reqs[r].L : reqs[r].P;  // sweep 2 needs the prefix keys only
+    const int slabs = (range + slab_keys - 1) / slab_keys;
+    const int cnt = slabs * sh.heads_per_req;
+    if (idx < base + cnt || r == sh.n_req - 1) {
+      const int local = idx - base;
+      const int hr = local / slabs;
+      U.slab = local - hr * slabs;
+      U.r = r;
+      U.u = reqs[r].head_base + hr;
+      U.l = hr / sh.n_kv_heads;
+      U.h = hr - U.l * sh.n_kv_heads;
+      U.kt0 = U.slab * slab_keys;
+      const int end = min(range, U.kt0 + slab_keys);
+      U.n_tiles = (end - U.kt0 + kTileKeys - 1) / kTileKeys;
+      U.P = reqs[r].P;
+      return U;
+    }
+    base += cnt;
+  }
+  return U;
+}
+
+// Sweep 1, 32 logits of one row: running maximum (raw dot products) and sum of exp2.
+template <bool MASKED>
+__device__ __forceinline__ void stats_chunk(float (&z)[32], int col0, int last_col, float sl, float& m_run, float& Z) {
+  if (MASKED) {
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+      if (col0 + c > last_col) z[c] = -INFINITY;
+  }
+  float cm = z[0];
+#pragma unroll
+  for (int c = 1; c < 32; ++c) cm = fmaxf(cm, z[c]);
+  if (MASKED && cm == -INFINITY) return;
+  const float m_new = fmaxf(m_run, cm);
+  Z *= ex2((m_run - m_new) * sl);  // first chunk: exp2(-inf) = 0
+  m_run = m_new;
+  const float nb = -m_new * sl;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+  for (int c = 0; c < 32; c += 4) {
+    a0 += ex2(fmaf(z[c], sl, nb));
+    a1 += ex2(fmaf(z[c + 1], sl, nb));
+    a2 += ex2(fmaf(z[c + 2], sl, nb));
+    a3 += ex2(fmaf(z[c + 3], sl, nb));
+  }
+  Z += (a0 + a1) + (a2 + a3);
+}
+
+template <int SWEEP, int D>
+__global__ void __launch_bounds__(kThreads, 1)
+score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  constexpr int KB = D / 64;                 // 64-element (128-byte) blocks along the head dimension
+  constexpr int kKBlk = kTileKeys * 128;     // bytes of one such block of a K tile
+  constexpr int kKStage = KB * kKBlk;
+  const int q_blk = a.q_rows * 128;
+  uint8_t* q_s = smem;
+  uint8_t* k_s = q_s + KB * q_blk;
+  Small* sm = reinterpret_cast<Small*>(k_s + a.n_stages * kKStage);
+  volatile int* abort = &sm->abort;
+
+  const Shape& sh = a.sh;
+  const int R = sh.window * sh.group, G = sh.group;
+  const bool both = SWEEP == 1 && R > 128;   // sweep 1 with two row blocks: each group reads its own block of every tile
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int S = a.n_stages;
+
+  // ---- set-up ----
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(smem_u32(&sm->k_full[s]), 1);
+      mbar_init(smem_u32(&sm->k_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&sm->q_full), 1);
+    mbar_init(smem_u32(&sm->q_empty), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sm->acc_full[b]), 1);
+      mbar_init(smem_u32(&sm->acc_empty[b]), both ? 8 : 4);
+      mbar_init(smem_u32(&sm->grp_bar[b]), 128);
+    }
+    mbar_init(smem_u32(&sm->all_bar), 256);
+    mbar_init(smem_u32(&sm->drain), 1);
+    sm->abort = 0;
+    fence_barrier_init();
+  }
+  for (int r = threadIdx.x; r < sh.n_req; r += kThreads) sm->reqs[r] = a.reqs[r];
+  {  // rows of the Q tile that no copy ever writes must read as zero
+    uint4* qz = reinterpret_cast<uint4*>(q_s);
+    const int n16 = KB * q_blk / 16;
+    for (int i = threadIdx.x; i < n16; i += kThreads) qz[i] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async();
+  }
+  if (warp == kProducerWarp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sm->tmem_base;
+  const ReqDesc* reqs = sm->reqs;
+
+  const int unit_begin = static_cast<int>(static_cast<int64_t>(blockIdx.x) * a.n_units / gridDim.x);
+  const int unit_end = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * a.n_units / gridDim.x);
+  // Sweep 2 walks the units backwards: the heads sweep 1 touched last are the ones still in L2.
+  auto unit_index = [&](int n) { return SWEEP == 2 ? a.n_units - 1 - n : n; };
+
+  if (warp == kProducerWarp) {
+    if (lane == 0) {
+      // ---- TMA producer ----
+      int it = 0, heads = 0, prev_u = -1;
+      bool ok = true;
+      for (int n = unit_begin; n < unit_end && ok; ++n) {
+        const Unit U = decode_unit<SWEEP>(sh, reqs, unit_index(n), a.slab_keys);
+        if (U.u != prev_u) {
+          if (heads > 0) ok = mbar_wait(smem_u32(&sm->q_empty), (heads - 1) & 1, abort);  // MMAs on the old Q are done
+          if (!ok) break;
+          const uint32_t bar = smem_u32(&sm->q_full);
+          mbar_expect_tx(bar, static_cast<uint32_t>(R) * D * 2);
+          for (int kb = 0; kb < KB; ++kb)
+            tma_load_5d(smem_u32(q_s + kb * q_blk), &tm.q, bar, kb * 64, U.h * G, 0, U.l, U.r);
+          prev_u = U.u;
+          ++heads;
+        }
+        for (int t = 0; t < U.n_tiles; ++t, ++it) {
+          const int s = it % S;
+          const uint32_t ph = (it / S) & 1;
+          ok = mbar_wait(smem_u32(&sm->k_empty[s]), ph ^ 1, abort);
+          if (!ok) break;
+          const uint32_t bar = smem_u32(&sm->k_full[s]);
+          mbar_expect_tx(bar, kKStage);
+          for (int kb = 0; kb < KB; ++kb)
+            tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r], bar, kb * 64, U.kt0 + t * kTileKeys, U.h,
+                        U.l);
+        }
+      }
+      if (*abort) {  // let the copies still in flight land before the CTA goes away
+        const long long short_limit = 200000000LL;
+        for (int j = it > S ? it - S : 0; j < it; ++j)
+          mbar_wait(smem_u32(&sm->k_full[j % S]), (j / S) & 1, abort, short_limit);
+        if (heads > 0) mbar_wait(smem_u32(&sm->q_full), (heads - 1) & 1, abort, short_limit);
+      }
+    }
+  } else if (warp == kMmaWarp) {
+    if (lane == 0) {
+      // ---- MMA issuer ----
+      int it = 0, heads = 0, prev_u = -1;
+      bool ok = true;
+      const int n_blk = both ? 2 : 1;
+      const uint32_t idesc = SWEEP == 1 ? umma_idesc(128, kTileKeys) : umma_idesc(kTileKeys, a.r_pad);
+      for (int n = unit_begin; n < unit_end && ok; ++n) {
+        const Unit U = decode_unit<SWEEP>(sh, reqs, unit_index(n), a.slab_keys);
+        if (U.u != prev_u) {
+          if (prev_u != -1) umma_commit(smem_u32(&sm->q_empty));
+          ok = mbar_wait(smem_u32(&sm->q_full), heads & 1, abort);
+          if (!ok) break;
+          tc_fence_after();
+          prev_u = U.u;
+          ++heads;
+        }
+        for (int t = 0; t < U.n_tiles; ++t, ++it) {
+          const int s = it % S;
+          ok = mbar_wait(smem_u32(&sm->k_full[s]), (it / S) & 1, abort);
+          if (!ok) break;
+          const int b = it & 1;
+          ok = mbar_wait(smem_u32(&sm->acc_empty[b]), ((it >> 1) & 1) ^ 1, abort);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_addr = smem_u32(k_s + s * kKStage);
+          const uint32_t q_addr = smem_u32(q_s);
+          for (int blk = 0; blk < n_blk; ++blk) {
+            const uint32_t d_tmem = tmem_base + b * kAccCols + blk * 128;
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb) {
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks) {
+                const uint64_t dq = umma_desc(q_addr + kb * q_blk + blk * (128 * 128) + ks * 32);
+                const uint64_t dk = umma_desc(k_addr + kb * kKBlk + ks * 32);
+                if (SWEEP == 1) umma_bf16(d_tmem, dq, dk, idesc, (kb | ks) != 0);
+                else umma_bf16(d_tmem, dk, dq, idesc, (kb | ks) != 0);
+              }
+            }
+          }
+          umma_commit(smem_u32(&sm->k_empty[s]));
+          umma_commit(smem_u32(&sm->acc_full[b]));
+        }
+      }
+      if (*abort) {  // TMEM must not be released under MMAs that are still running
+        umma_commit(smem_u32(&sm->drain));
+        mbar_wait(smem_u32(&sm->drain), 0, abort, 200000000LL);
+      }
+    }
+  } else {
+    // ---- epilogue: two groups of four warps; warp w reads TMEM lanes 32 (w % 4) .. +31 ----
+    const int g = warp >> 2, quarter = warp & 3;
+    const int gl = quarter * 32 + lane;  // thread index inside the group = TMEM lane
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const float sl = sh.scale_log2e;
+    int it = 0, prev_u = -1, n_done = 0, heads = 0;
+    uint32_t grp_phase = 0, all_phase = 0;
+    bool ok = true;
+    for (int n = unit_begin; n < unit_end && ok; ++n, ++n_done) {
+      const Unit U = decode_unit<SWEEP>(sh, reqs, unit_index(n), a.slab_keys);
+      if (SWEEP == 2 && U.u != prev_u) {
+        // merge the slabs' statistics of this head: negc[row] = -(max + log2 sum); +/-inf rows give 0
+        const int slabs = (reqs[U.r].L + a.slab_keys - 1) / a.slab_keys;
+        const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.n_slab * R;
+        for (int row = gl; row < 256; row += 128) {
+          float c = -INFINITY;
+          if (row < R) {
+            float M = -INFINITY;
+            for (int s = 0; s < slabs; ++s) M = fmaxf(M, hs[static_cast<int64_t>(s) * R + row].x);
+            float Zt = 0.f;
+            for (int s = 0; s < slabs; ++s) {
+              const float2 st = hs[static_cast<int64_t>(s) * R + row];
+              if (st.y > 0.f) Zt += st.y * exp2f(st.x - M);
+            }
+            c = -(M + log2f(Zt));
+          }
+          // two copies by head parity: a slower warp of the group may still read the previous head's
+          sm->negc[g][heads & 1][row] = c;
+        }
+        ++heads;
+        mbar_arrive(smem_u32(&sm->grp_bar[g]));
+        ok = mbar_wait(smem_u32(&sm->grp_bar[g]), grp_phase, abort);
+        grp_phase ^= 1;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+      prev_u = U.u;
+      float m_run = -INFINITY, Z = 0.f;  // sweep 1: this thread's row
+      const int row = (both ? g * 128 : 0) + gl;
+      const int win_i = row / G;         // window row of this query row
+      for (int t = 0; t < U.n_tiles; ++t, ++it) {
+        const int b = it & 1;
+        if (!both && b != g) continue;   // tiles alternate between the groups
+        ok = mbar_wait(smem_u32(&sm->acc_full[b]), (it >> 1) & 1, abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const int kt = U.kt0 + t * kTileKeys;
+        if (SWEEP == 1) {
+          const uint32_t taddr = lane_addr + b * kAccCols + (both ? g * 128 : 0);
+          const bool masked = kt + kTileKeys - 1 > U.P;  // the tile reaches into the window: causal mask, end of request
+          const int last_col = U.P + win_i - kt;         // last visible key of this row, relative to the tile
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float z[32];
+            tmem_ld32(taddr + c * 32, z);
+            if (row < R) {
+              if (masked) stats_chunk<true>(z, c * 32, last_col, sl, m_run, Z);
+              else stats_chunk<false>(z, c * 32, last_col, sl, m_run, Z);
+            }
+          }
+        } else {
+          const uint32_t taddr = lane_addr + b * kAccCols;
+          const float* nc = sm->negc[g][(heads - 1) & 1];
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          const int n32 = a.r_pad >> 5;
+#pragma unroll 1
+          for (int c = 0; c < n32; ++c) {
+            float z[32];
+            tmem_ld32(taddr + c * 32, z);
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              const float4 v = *reinterpret_cast<const float4*>(nc + c * 32 + i);
+              a0 += ex2(fmaf(z[i], sl, v.x));
+              a1 += ex2(fmaf(z[i + 1], sl, v.y));
+              a2 += ex2(fmaf(z[i + 2], sl, v.z));
+              a3 += ex2(fmaf(z[i + 3], sl, v.w));
+            }
+          }
+          if (a.r_pad & 16) {
+            float z[16];
+            tmem_ld16(taddr + n32 * 32, z);
+#pragma unroll
+            for (int i = 0; i < 16; i += 4) {
+              const float4 v = *reinterpret_cast<const float4*>(nc + n32 * 32 + i);
+              a0 += ex2(fmaf(z[i], sl, v.x));
+              a1 += ex2(fmaf(z[i + 1], sl, v.y));
+              a2 += ex2(fmaf(z[i + 2], sl, v.z));
+              a3 += ex2(fmaf(z[i + 3], sl, v.w));
+            }
+          }
+          const int key = kt + gl;
+          if (key < U.P)
+            a.scores[reqs[U.r].score_offset + static_cast<int64_t>(U.u - reqs[U.r].head_base) * U.P + key] =
+                (a0 + a1) + (a2 + a3);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[b]));
+      }
+      if (!ok) break;
+      if (SWEEP == 1) {
+        float2* out = a.stats + (static_cast<int64_t>(U.u) * a.n_slab + U.slab) * R;
+        if (both) {
+          if (row < R) out[row] = make_float2(m_run * sl, Z);
+        } else {
+          // one row block: both groups hold partial statistics of the same rows
+          float2* mg = sm->mrg[n_done & 1];
+          if (g == 1) mg[gl] = make_float2(m_run, Z);
+          mbar_arrive(smem_u32(&sm->all_bar));
+          ok = mbar_wait(smem_u32(&sm->all_bar), all_phase, abort);
+          all_phase ^= 1;
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          if (g == 0 && row < R) {
+            const float2 o = mg[gl];
+            const float M = fmaxf(m_run, o.x);
+            float Zt = 0.f;
+            if (Z > 0.f) Zt += Z * ex2((m_run - M) * sl);
+            if (o.y > 0.f) Zt += o.y * ex2((o.x - M) * sl);
+            out[row] = make_float2(M * sl, Zt);
+          }
+        }
+      }
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && sm->abort) atomicExch(a.status, AUDIOKV_ETIMEOUT);
+  if (warp == kProducerWarp) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess ||
+        qr != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// Byte strides of the outer dimensions; a dimension of extent 1 takes a harmless stride when the
+// caller's is zero. Returns false for a stride the copy engine cannot express.
+bool fill_strides(int rank, const cuuint64_t* dims, const int64_t* elem_strides, cuuint64_t* out) {
+  for (int i = 1; i < rank; ++i) {
+    int64_t s = elem_strides[i - 1] * 2;
+    if (dims[i] == 1 && s <= 0) s = 16;
+    if (s <= 0 || (s & 15) || s >= (static_cast<int64_t>(1) << 40)) return false;
+    out[i - 1] = static_cast<cuuint64_t>(s);
+  }
+  return true;
+}
+
+template <int SWEEP, int D>
+cudaError_t launch_sweep(const TmapPack& tm, const UmmaArgs& args, int grid, size_t smem, cudaStream_t stream) {
+  auto kern = score_umma_kernel<SWEEP, D>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  kern<<<grid, kThreads, smem, stream>>>(tm, args);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool score_umma_takes(const Shape& sh) {
+  if (sh.dtype != AUDIOKV_BF16) return false;
+  const int R = sh.window * sh.group;
+  if (R > 256 || sh.group > 256 || sh.window > 256) return false;
+  const int q_rows = R > 128 ? 256 : 128;
+  const int q_bytes = q_rows * sh.head_dim * 2, stage = kTileKeys * sh.head_dim * 2;
+  const int room = kSmemLimit - 1024 - static_cast<int>(sizeof(Small)) - q_bytes;
+  return room >= 2 * stage;
+}
+
+cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ReqDesc* d_reqs, const void* q,
+                              const void* k, float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status,
+                              Launch ln) {
+  if (!score_umma_takes(sh) || slab_keys % kTileKeys) return cudaErrorNotSupported;
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  const int R = sh.window * sh.group, d = sh.head_dim;
+
+  TmapPack tm;
+  memset(&tm, 0, sizeof(tm));
+  {
+    const cuuint64_t dims[5] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(sh.n_q_heads),
+                                static_cast<cuuint64_t>(sh.window), static_cast<cuuint64_t>(sh.n_layers),
+                                static_cast<cuuint64_t>(sh.n_req)};
+    const int64_t es[4] = {sh.q_stride_head, sh.q_stride_tok, sh.q_stride_layer,
+                           sh.n_req > 1 ? h_reqs[1].q_offset - h_reqs[0].q_offset : 0};
+    cuuint64_t strides[4];
+    if (!fill_strides(5, dims, es, strides)) return cudaErrorNotSupported;
+    const cuuint32_t box[5] = {64u, static_cast<cuuint32_t>(sh.group), static_cast<cuuint32_t>(sh.window), 1u, 1u};
+    const cuuint32_t ones[5] = {1u, 1u, 1u, 1u, 1u};
+    if (enc(&tm.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q), dims, strides, box, ones,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorNotSupported;
+  }
+  int n_units1 = 0, n_units2 = 0;
+  for (int r = 0; r < sh.n_req; ++r) {
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(h_reqs[r].L),
+                                static_cast<cuuint64_t>(sh.n_kv_heads), static_cast<cuuint64_t>(sh.n_layers)};
+    const int64_t es[3] = {sh.kv_stride_tok, sh.kv_stride_head, sh.kv_stride_layer};
+    cuuint64_t strides[3];
+    if (!fill_strides(4, dims, es, strides)) return cudaErrorNotSupported;
+    const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(kTileKeys), 1u, 1u};
+    const cuuint32_t ones[4] = {1u, 1u, 1u, 1u};
+    void* base = const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(k) + h_reqs[r].kv_offset);
+    if (enc(&tm.k[r], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, ones,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorNotSupported;
+    n_units1 += sh.heads_per_req * ((h_reqs[r].L + slab_keys - 1) / slab_keys);
+    n_units2 += sh.heads_per_req * ((h_reqs[r].P + slab_keys - 1) / slab_keys);
+  }
+
+  UmmaArgs args{};
+  args.sh = sh;
+  args.reqs = d_reqs;
+  args.stats = stats_ws;
+  args.scores = scores;
+  args.status = status;
+  args.n_slab = n_slab;
+  args.slab_keys = slab_keys;
+  args.q_rows = R > 128 ? 256 : 128;
+  args.r_pad = (R + 15) / 16 * 16;
+  const int q_bytes = args.q_rows * d * 2, stage = kTileKeys * d * 2;
+  const int room = kSmemLimit - 1024 - static_cast<int>(sizeof(Small)) - q_bytes;
+  args.n_stages = room / stage < kMaxStages ? room / stage : kMaxStages;
+  const size_t smem = 1024 + static_cast<size_t>(q_bytes) + static_cast<size_t>(args.n_stages) * stage + sizeof(Small);
+
+  int dev = 0, n_sm = 0;
+  cudaError_t e;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+
+#define AKV_SWEEP(SW, DD, UNITS)                                                           \
+  args.n_units = (UNITS);                                                                  \
+  e = launch_sweep<SW, DD>(tm, args, (UNITS) < n_sm ? (UNITS) : n_sm, smem, ln.stream);     \
+  if (e != cudaSuccess) return e;                                                          \
+  ln.done(SW == 1 ? "score_umma_stats" : "score_umma_colsum")
+  if (d == 64) {
+    AKV_SWEEP(1, 64, n_units1);
+    AKV_SWEEP(2, 64, n_units2);
+  } else if (d == 128) {
+    AKV_SWEEP(1, 128, n_units1);
+    AKV_SWEEP(2, 128, n_units2);
+  } else {
+    AKV_SWEEP(1, 256, n_units1);
+    AKV_SWEEP(2, 256, n_units2);
+  }
+#undef AKV_SWEEP
+  return cudaSuccess;
+}
+
+}  // namespace akv
