@@ -106,7 +106,7 @@ def kernel_algorithmic_bytes(name, spec, w):
         return k_bytes + q_bytes + score_bytes
     if name == "sss":
         return 2 * score_bytes
-    if name == "select":
+    if name in ("select", "sss_select"):
         return score_bytes + 4 * kept_rows
     if name == "gather":
         return kept_rows * (4 + 4 * d * e)           # index + K,V row read + K,V row written
@@ -179,7 +179,21 @@ def run_cuda(args):
     ctx.profile_enable(False)
     torch.cuda.synchronize()
 
-    # end to end through the host-buffer entry point: pinned host inputs, results read back
+    e2e_ms, h2d, d2h = None, 0, 0
+    if not args.skip_e2e:
+        e2e_ms, h2d, d2h = run_e2e(B, ctx, prob, w, spec, tb, rows, TH, es, barrier, world, args)
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+    report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_ms, h2d, d2h)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def run_e2e(B, ctx, prob, w, spec, tb, rows, TH, es, barrier, world, args):
+    """End to end through the host-buffer entry point: pinned host inputs, results read back."""
     hq, hk, hv = (w.as_torch(a).pin_memory() for a in (w.q, w.k, w.v))
     hS = torch.from_numpy(w.head_scores).pin_memory()
     hko = torch.empty((rows, spec.head_dim), dtype=es).pin_memory()
@@ -205,11 +219,10 @@ def run_cuda(args):
     e2e_ms = float(t.item())
     h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv, hS))
     d2h = sum(x.numel() * x.element_size() for x in (hko, hvo, hkept, hb, hcu))
+    return e2e_ms, h2d, d2h
 
-    if rank != 0:
-        if world > 1:
-            torch.distributed.destroy_process_group()
-        return
+
+def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_ms, h2d, d2h):
     NL = spec.n_layers
     peaks, peak_kind = measured_peaks()
     us_layer = ms_step * 1e3 / (NL * world)
@@ -239,15 +252,14 @@ def run_cuda(args):
         "roofline": {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4), "peak_kind": peak_kind,
                      "algorithmic_bytes": dom_bytes, "traffic": NCU_TRAFFIC_BYTES.get(dom)},
-        "e2e": {"value": round(e2e_ms * 1e3 / (NL * world), 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
+        "e2e": None if e2e_ms is None else
+               {"value": round(e2e_ms * 1e3 / (NL * world), 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
         "clocks": clocks,
     }
     if not args.skip_cpu:
         line["cpu_baseline"] = cpu_baseline(w, spec, budget_s=15.0)
     print(json.dumps(line), flush=True)
-    if world > 1:
-        torch.distributed.destroy_process_group()
 
 
 def oracle_pass(w, spec, n_layers):
@@ -306,6 +318,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline (profiling runs)")
+    ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer end-to-end leg (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -1,4 +1,4 @@
-// Head-wise budgets in exact integer arithmetic: one thread block per request.
+// Head-wise budgets in exact integer arithmetic, and their prefix sums: one thread block per request.
 //
 // Every head gets window + base rows; the remaining rows R of the request's total are
 // shared in proportion to S_q = round-half-up(S * 2^24): floors first, heads whose share
@@ -13,7 +13,8 @@ namespace {
 constexpr int kAllocThreads = 256;
 
 struct BudgetArgs {
-  int64_t total[AUDIOKV_MAX_REQ];
+  int64_t total[AUDIOKV_MAX_REQ];    // B_r
+  int64_t cu_base[AUDIOKV_MAX_REQ];  // rows kept by the requests before r: sum of their B (budgets add up exactly)
 };
 
 __device__ __forceinline__ long long block_sum_ll(long long v, long long* red) {
@@ -29,7 +30,7 @@ __device__ __forceinline__ long long block_sum_ll(long long v, long long* red) {
 
 __global__ void __launch_bounds__(kAllocThreads)
 allocate_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restrict__ head_scores, BudgetArgs args,
-                int32_t* __restrict__ budgets, int* __restrict__ status) {
+                int32_t* __restrict__ budgets, int32_t* __restrict__ cu_kept, int* __restrict__ status) {
   extern __shared__ long long sm[];
   const int N = sh.heads_per_req;
   long long* Sq = sm;            // [N] quantised scores
@@ -131,38 +132,31 @@ allocate_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restr
   __syncthreads();
   for (int h = threadIdx.x; h < N; h += kAllocThreads)
     budgets[rq.head_base + h] = static_cast<int32_t>(f + tk[h]);
-}
 
-// cu_kept = exclusive prefix sum of budgets over all heads (single block).
-__global__ void __launch_bounds__(1024) cu_kept_kernel(const int32_t* __restrict__ budgets, int total,
-                                                      int32_t* __restrict__ cu_kept) {
-  __shared__ int wsum[32];
-  const int per = (total + 1023) / 1024;
-  const int a = min(total, static_cast<int>(threadIdx.x) * per), b = min(total, a + per);
-  int local = 0;
-  for (int i = a; i < b; ++i) local += budgets[i];
+  // cu_kept: exclusive prefix sum of the budgets in flat head order. The request's first row is known
+  // without looking at other requests, because every request keeps exactly total[r] rows.
+  const int per = (N + kAllocThreads - 1) / kAllocThreads;
+  const int a = min(N, static_cast<int>(threadIdx.x) * per), b = min(N, a + per);
+  long long local = 0;
+  for (int h = a; h < b; ++h) local += f + tk[h];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int inc = local;
+  long long inc = local;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    int t = __shfl_up_sync(0xffffffffu, inc, o);
+    const long long t = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= o) inc += t;
   }
-  if (lane == 31) wsum[warp] = inc;
   __syncthreads();
-  int ws = wsum[lane], winc = ws;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int t = __shfl_up_sync(0xffffffffu, winc, o);
-    if (lane >= o) winc += t;
+  if (lane == 31) red[warp] = inc;
+  __syncthreads();
+  long long run = args.cu_base[r] + inc - local;
+  for (int w = 0; w < warp; ++w) run += red[w];
+  for (int h = a; h < b; ++h) {
+    cu_kept[rq.head_base + h] = static_cast<int32_t>(run);
+    run += f + tk[h];
   }
-  int run = __shfl_sync(0xffffffffu, winc - ws, warp) + inc - local;
-  for (int i = a; i < b; ++i) {
-    cu_kept[i] = run;
-    run += budgets[i];
-  }
-  if (a < b && b == total) cu_kept[total] = run;  // the one non-empty range that ends at `total`
-  if (total == 0 && threadIdx.x == 0) cu_kept[0] = 0;
+  if (r == sh.n_req - 1 && threadIdx.x == 0)
+    cu_kept[sh.total_heads] = static_cast<int32_t>(args.cu_base[r] + args.total[r]);
 }
 
 }  // namespace
@@ -171,14 +165,19 @@ cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float*
                             const int64_t* h_total_budget, int32_t* budgets, int32_t* cu_kept, int* status,
                             Launch ln) {
   BudgetArgs args;
-  for (int r = 0; r < sh.n_req; ++r) args.total[r] = h_total_budget[r];
+  int64_t rows = 0;
+  for (int r = 0; r < sh.n_req; ++r) {
+    args.total[r] = h_total_budget[r];
+    args.cu_base[r] = rows;
+    rows += h_total_budget[r];
+  }
+  if (rows > 0x7fffffffLL) return cudaErrorInvalidValue;  // cu_kept is int32
   const size_t smem = static_cast<size_t>(sh.heads_per_req) * (3 * sizeof(long long) + 2 * sizeof(int));
   cudaError_t e = cudaFuncSetAttribute(allocate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  allocate_kernel<<<sh.n_req, kAllocThreads, smem, ln.stream>>>(sh, d_reqs, head_scores, args, budgets, status);
+  allocate_kernel<<<sh.n_req, kAllocThreads, smem, ln.stream>>>(sh, d_reqs, head_scores, args, budgets, cu_kept,
+                                                                 status);
   ln.done("allocate");
-  cu_kept_kernel<<<1, 1024, 0, ln.stream>>>(budgets, sh.total_heads, cu_kept);
-  ln.done("cu_kept");
   return cudaGetLastError();
 }
 

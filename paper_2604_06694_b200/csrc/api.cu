@@ -51,6 +51,8 @@ struct audiokv_ctx {
   Plan plan;
   bool plan_uploaded = false;
   cudaEvent_t plan_ready = nullptr;
+  cudaStream_t side = nullptr;            // audiokv_evict runs the allocation here, beside the scoring
+  cudaEvent_t fork = nullptr, join = nullptr;
   int64_t launches = 0;
   Profiler prof;
   std::string cuda_error;
@@ -159,6 +161,10 @@ void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
   if (fp->packed) {
     fp->post_offset = *table_len;
     *table_len += N / 2 + 1;
+  }
+  if (!fp->bluestein) {
+    fp->pos_offset = *table_len;
+    *table_len += (N + 1) / 2;  // N int32 entries
   }
   if (fp->bluestein) {
     fp->chirp_offset = *table_len;
@@ -321,13 +327,23 @@ int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cuda
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 
-int do_smooth(audiokv_ctx* ctx, const float* scores, float* smoothed, int32_t* kstar, cudaStream_t stream) {
+// Smoothing; with budgets, cu_kept and kept_idx it also selects each head's kept tokens (smoothed may then be null).
+int do_smooth(audiokv_ctx* ctx, const float* scores, float* smoothed, int32_t* kstar, const int32_t* budgets,
+              const int32_t* cu_kept, int32_t* kept_idx, cudaStream_t stream) {
   Plan& pl = ctx->plan;
   Launch ln{stream, &ctx->launches, &ctx->prof};
   cudaError_t e = launch_sss(pl.sh, d_reqs(ctx), reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans),
                              reinterpret_cast<const float2*>(ctx->ws + pl.lay.tables), scores, smoothed, kstar,
                              reinterpret_cast<float2*>(ctx->ws + pl.lay.fft_scratch), pl.scratch_per_block,
-                             pl.sss_grid, pl.sss_smem, ln);
+                             pl.sss_grid, pl.sss_smem, budgets, cu_kept, kept_idx, d_status(ctx), ln);
+  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
+}
+
+int do_gather(audiokv_ctx* ctx, const int32_t* cu_kept, const int32_t* kept_idx, const void* k, const void* v,
+              void* k_out, void* v_out, cudaStream_t stream) {
+  Plan& pl = ctx->plan;
+  Launch ln{stream, &ctx->launches, &ctx->prof};
+  cudaError_t e = launch_gather(pl.sh, d_reqs(ctx), cu_kept, kept_idx, k, v, k_out, v_out, ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 
@@ -357,8 +373,7 @@ int do_select_gather(audiokv_ctx* ctx, const float* smoothed, const int32_t* bud
   Launch ln{stream, &ctx->launches, &ctx->prof};
   cudaError_t e = launch_select(pl.sh, d_reqs(ctx), smoothed, budgets, cu_kept, kept_idx, pl.max_P, d_status(ctx), ln);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
-  e = launch_gather(pl.sh, d_reqs(ctx), cu_kept, kept_idx, k, v, k_out, v_out, ln);
-  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
+  return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, stream);
 }
 
 }  // namespace
@@ -432,7 +447,13 @@ int audiokv_create(audiokv_ctx** out, int device, size_t workspace_bytes) {
     return AUDIOKV_ECUDA;
   }
   c->ws_bytes = workspace_bytes;
-  if (cudaEventCreateWithFlags(&c->plan_ready, cudaEventDisableTiming) != cudaSuccess) {
+  if (cudaEventCreateWithFlags(&c->plan_ready, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->join, cudaEventDisableTiming) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess) {
+    if (c->plan_ready) cudaEventDestroy(c->plan_ready);
+    if (c->fork) cudaEventDestroy(c->fork);
+    if (c->join) cudaEventDestroy(c->join);
     cudaFree(c->ws);
     delete c;
     return AUDIOKV_ECUDA;
@@ -445,6 +466,9 @@ int audiokv_destroy(audiokv_ctx* ctx) {
   if (!ctx) return AUDIOKV_EINVAL;
   cudaSetDevice(ctx->device);
   cudaEventDestroy(ctx->plan_ready);
+  cudaEventDestroy(ctx->fork);
+  cudaEventDestroy(ctx->join);
+  cudaStreamDestroy(ctx->side);
   for (cudaEvent_t e : ctx->prof.ev)
     if (e) cudaEventDestroy(e);
   cudaFree(ctx->ws);
@@ -510,7 +534,7 @@ int audiokv_smooth(audiokv_ctx* ctx, const audiokv_params* p, const float* score
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int rc = prepare(ctx, p, s);
   if (rc) return rc;
-  return do_smooth(ctx, scores, smoothed, kstar_or_null, s);
+  return do_smooth(ctx, scores, smoothed, kstar_or_null, nullptr, nullptr, nullptr, s);
 }
 
 int audiokv_allocate(audiokv_ctx* ctx, const audiokv_params* p, const float* head_scores,
@@ -547,10 +571,25 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
   float* ws_scores = reinterpret_cast<float*>(ctx->ws + pl.lay.scores);
   int32_t* ws_kstar = reinterpret_cast<int32_t*>(ctx->ws + pl.lay.kstar);
   profile_begin(ctx, s);
-  if ((rc = do_allocate(ctx, head_scores, total_budget, budgets, cu_kept, s))) return rc;
+  // The budgets depend on nothing the GPU computes, and only the selection needs them: the allocation
+  // runs on the context's side stream beside the scoring (on the caller's stream while per-kernel
+  // timing is on, so that every kernel is timed alone).
+  const bool beside = !ctx->prof.on;
+  cudaError_t e;
+  if (beside) {
+    if ((e = cudaEventRecord(ctx->fork, s)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaStreamWaitEvent(ctx->side, ctx->fork, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+  }
+  rc = do_allocate(ctx, head_scores, total_budget, budgets, cu_kept, beside ? ctx->side : s);
+  if (beside) {
+    // recorded even after a failed launch, so that the side stream always rejoins the caller's
+    if ((e = cudaEventRecord(ctx->join, ctx->side)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaStreamWaitEvent(s, ctx->join, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+  }
+  if (rc) return rc;
   if ((rc = do_score(ctx, q_win, k, ws_scores, s))) return rc;
-  if ((rc = do_smooth(ctx, ws_scores, ws_scores, ws_kstar, s))) return rc;
-  return do_select_gather(ctx, ws_scores, budgets, cu_kept, k, v, k_out, v_out, kept_idx, s);
+  if ((rc = do_smooth(ctx, ws_scores, nullptr, ws_kstar, budgets, cu_kept, kept_idx, s))) return rc;
+  return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, s);
 }
 
 int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, int64_t q_elems, const void* k,

@@ -62,6 +62,7 @@ struct FftPlan {
   int64_t chirp_offset;   // float2 index of c_j = exp(-i pi j^2 / N), j in [0, N)      (bluestein)
   int64_t filter_offset;  // float2 index of FFT_M of the wrapped conjugate chirp / M    (bluestein)
   int64_t post_offset;    // float2 index of exp(-2 pi i k / n), k in [0, N/2]           (packed)
+  int64_t pos_offset;     // float2 index of an int32 table: slot of bin k after the forward passes (direct)
 };
 
 constexpr int kMaxPlans = AUDIOKV_MAX_REQ;
@@ -106,9 +107,12 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ReqD
 
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);
+// smoothed may be null when budgets, cu_kept and kept_idx are given: the kernel then goes on to the
+// top-k selection of each head from the smoothed scores it holds on chip (step 4a of the pass).
 cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_plans, const float2* d_tables,
                        const float* scores, float* smoothed, int32_t* kstar, float2* scratch,
-                       int64_t scratch_per_block, int grid, size_t smem_bytes, Launch ln);
+                       int64_t scratch_per_block, int grid, size_t smem_bytes, const int32_t* budgets,
+                       const int32_t* cu_kept, int32_t* kept_idx, int* status, Launch ln);
 
 // allocate.cu (h_total_budget: host array [n_req])
 cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float* head_scores,

@@ -1,51 +1,18 @@
 // Per-head top-k by radix select, ordered compaction of the kept indices, and the
 // vectorised gather of the kept K and V rows into the compacted cache.
 #include "common.cuh"
+#include "select.cuh"
 
 namespace akv {
 namespace {
 
-constexpr int kSelThreads = 1024;
-
-// Order-preserving map float -> uint32 (larger float, larger key); -0 and +0 share a key.
-__device__ __forceinline__ uint32_t score_key(float f) {
-  uint32_t u = __float_as_uint(f);
-  if (u == 0x80000000u) u = 0u;
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
-__device__ __forceinline__ int block_excl_scan_int(int v, int* wsum, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
-  __syncthreads();
-  if (lane == 31) wsum[warp] = inc;
-  __syncthreads();
-  int ws = wsum[lane], winc = ws;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int t = __shfl_up_sync(0xffffffffu, winc, o);
-    if (lane >= o) winc += t;
-  }
-  *total = __shfl_sync(0xffffffffu, winc, 31);
-  return __shfl_sync(0xffffffffu, winc - ws, warp) + inc - v;
-}
-
-// One block per head: k-th largest key by four 8-bit radix passes over the head's scores
-// (staged once in shared memory when they fit), then the kept indices in ascending order.
+// One block per head: the head's keys staged once in shared memory when they fit, then select_topk.
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restrict__ smoothed,
               const int32_t* __restrict__ budgets, const int32_t* __restrict__ cu_kept,
               int32_t* __restrict__ kept_idx, int smem_keys, int* __restrict__ status) {
   extern __shared__ uint32_t skeys[];
-  __shared__ int hist[256];
-  __shared__ int wsum[32];
-  __shared__ uint32_t s_prefix;
-  __shared__ int s_want;
+  __shared__ SelectSmem ssm;
 
   for (int u = blockIdx.x; u < sh.total_heads; u += gridDim.x) {
     const int r = u / sh.heads_per_req;
@@ -57,81 +24,15 @@ select_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restric
       if (threadIdx.x == 0) atomicExch(status, AUDIOKV_EDEVICE);
       k = k < 0 ? 0 : P;
     }
-    int32_t* out = kept_idx + cu_kept[u];
     const bool staged = P <= smem_keys;
     __syncthreads();
     if (staged)
       for (int j = threadIdx.x; j < P; j += kSelThreads) skeys[j] = score_key(s[j]);
     __syncthreads();
-    auto key_at = [&](int j) -> uint32_t { return staged ? skeys[j] : score_key(s[j]); };
-
-    uint32_t thr = 0;     // key of the k-th largest element
-    int need_eq = 0;      // how many elements equal to thr are kept (those with the lowest indices)
-    if (k > 0 && k < P) {
-      if (threadIdx.x == 0) {
-        s_prefix = 0u;
-        s_want = k;
-      }
-      for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        for (int b = threadIdx.x; b < 256; b += kSelThreads) hist[b] = 0;
-        __syncthreads();
-        const uint32_t prefix = s_prefix;
-        const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-        for (int j = threadIdx.x; j < P; j += kSelThreads) {
-          const uint32_t key = key_at(j);
-          if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-          int want = s_want, b = 255;
-          for (; b > 0; --b) {
-            if (hist[b] >= want) break;
-            want -= hist[b];
-          }
-          s_prefix = prefix | (static_cast<uint32_t>(b) << shift);
-          s_want = want;
-        }
-        __syncthreads();
-      }
-      thr = s_prefix;
-      need_eq = s_want;
-    } else if (k == P) {
-      thr = 0u;
-      need_eq = P;  // every key is >= 0: keep all
-    }
-
-    // ordered compaction: thread t owns the contiguous index range [a, b)
-    const int per = (P + kSelThreads - 1) / kSelThreads;
-    const int a = min(P, static_cast<int>(threadIdx.x) * per), b = min(P, a + per);
-    int n_eq = 0, n_gt = 0;
-    if (k > 0) {
-      for (int j = a; j < b; ++j) {
-        const uint32_t key = key_at(j);
-        n_eq += key == thr;
-        n_gt += key > thr;
-      }
-    }
-    int tot;
-    const int eq_before = block_excl_scan_int(n_eq, wsum, &tot);
-    int my_eq_kept = min(n_eq, max(0, need_eq - eq_before));
-    if (k == 0) my_eq_kept = 0;
-    int pos = block_excl_scan_int(n_gt + my_eq_kept, wsum, &tot);
-    if (k > 0) {
-      int eq_seen = eq_before;
-      for (int j = a; j < b; ++j) {
-        const uint32_t key = key_at(j);
-        bool keep = key > thr;
-        if (key == thr) {
-          keep = eq_seen < need_eq;
-          ++eq_seen;
-        }
-        if (keep) out[pos++] = j;
-      }
-    }
-    if (tot != k && threadIdx.x == 0) atomicExch(status, AUDIOKV_EDEVICE);
-    for (int i = threadIdx.x; i < W; i += kSelThreads) out[k + i] = P + i;
-    __syncthreads();
+    if (staged)
+      select_topk([&](int j) -> uint32_t { return skeys[j]; }, P, W, k, kept_idx + cu_kept[u], &ssm, status);
+    else
+      select_topk([&](int j) -> uint32_t { return score_key(s[j]); }, P, W, k, kept_idx + cu_kept[u], &ssm, status);
   }
 }
 

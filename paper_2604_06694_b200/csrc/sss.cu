@@ -2,18 +2,19 @@
 //
 // A real sequence of even length n is packed into a complex one of length N = n/2
 // (odd n: length N = n with zero imaginary part). The complex transform is an in-place
-// mixed-radix decimation-in-frequency FFT (radices 4, 2, 3, 5, 7 per thread, any prime up
-// to 127 per warp); its output is left in digit-reversed order and addressed through
+// mixed-radix decimation-in-frequency FFT (radices 4, 2, 3, 5, 7 per thread, larger primes up
+// to 127 as paired O(p^2) sums split over warps); its output is left in digit-reversed order and addressed through
 // pos(k), and the inverse is the matching decimation-in-time chain, so no reordering pass
 // and no second buffer is needed. Lengths with a larger prime factor go through a chirp-z
 // (Bluestein) convolution of power-of-two length M >= 2N - 1 built from the same passes.
 // The work buffer lives in shared memory when it fits, else in a per-block global scratch.
 #include "common.cuh"
+#include "select.cuh"
 
 namespace akv {
 namespace {
 
-constexpr int kSssThreads = 1024;
+constexpr int kSssThreads = kSelThreads;  // 1024: select_topk runs in the same block
 
 __device__ __forceinline__ float2 cmul(float2 a, float2 b) {
   return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
@@ -133,52 +134,93 @@ __device__ __forceinline__ void pass_small(float2* buf, int N, int ns, const flo
   __syncthreads();
 }
 
-// The same pass for a prime radix p <= 128: one warp per butterfly, lane c (+32, +64, +96)
-// accumulates output c from the p inputs, which every lane reads from the buffer.
+// The same pass for an odd prime radix p, 11 <= p <= 127. A length-p DFT is O(p^2); pairing
+// inputs s and p - s (P = a_s + a_{p-s}, Q = a_s - a_{p-s}) gives outputs c and p - c from the
+// same real-by-complex products: X_c = A -/+ iB, A = a_0 + sum_s P_s cos(2 pi s c / p),
+// B = sum_s Q_s sin(2 pi s c / p). Work is split into warp tasks: 32 consecutive butterflies
+// (one per lane) times a chunk of kPrimeChunk output pairs, so the cos/sin reads are
+// broadcasts. A round holds whole butterfly groups only: results stay in registers until
+// every task of the round has read its inputs, then overwrite them.
+constexpr int kPrimeChunk = 6;
+
 template <bool INV>
-__device__ __forceinline__ void pass_generic(float2* buf, int N, int ns, int p, const float2* __restrict__ tw,
-                                             float2* wp /* smem: W_p^t */) {
+__device__ __noinline__ void pass_prime(float2* buf, int N, int ns, int p, const float2* __restrict__ tw,
+                                           float2* cs /* smem [128]: (cos, sin) of 2 pi t / p */) {
   __syncthreads();
-  for (int t = threadIdx.x; t < p; t += kSssThreads) wp[t] = __ldg(tw + t * (N / p));
+  for (int t = threadIdx.x; t < p; t += kSssThreads) {
+    const float2 w = __ldg(tw + t * (N / p));
+    cs[t] = make_float2(w.x, -w.y);
+  }
   __syncthreads();
-  const int m = ns / p, step = N / ns, nb = N / p;
+  const int m = ns / p, step = N / ns, nb = N / p, H = (p - 1) / 2;
+  const int n_chunks = (H + kPrimeChunk - 1) / kPrimeChunk;
+  const int gpr = 32 / n_chunks;  // butterfly groups per round (n_chunks <= 11)
+  const int n_groups = (nb + 31) / 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int t = warp; t < nb; t += kSssThreads / 32) {
-    const int b = t / m, j = t - b * m;
-    float2* base = buf + b * ns + j;
-    float2 acc[4];
-    int idx[4];
+  const int chunk = warp % n_chunks, c0 = 1 + chunk * kPrimeChunk;
+  for (int g0 = 0; g0 < n_groups; g0 += gpr) {
+    const int grp = g0 + warp / n_chunks;
+    const int t = grp * 32 + lane;
+    const bool active = warp < gpr * n_chunks && grp < n_groups && t < nb;
+    float2 A[kPrimeChunk], B[kPrimeChunk];
+    float2 X0 = make_float2(0.f, 0.f);
+    float2* base = buf;
+    int j = 0;
+    if (active) {
+      const int b = t / m;
+      j = t - b * m;
+      base = buf + b * ns + j;
+      const float2 a0 = base[0];
+      X0 = a0;
+      int idx[kPrimeChunk];
 #pragma unroll
-    for (int o = 0; o < 4; ++o) {
-      acc[o] = make_float2(0.f, 0.f);
-      idx[o] = 0;
-    }
-    for (int s = 0; s < p; ++s) {
-      float2 a = base[s * m];
-      if (INV && m > 1) a = cmulc(a, __ldg(tw + j * s * step));
+      for (int o = 0; o < kPrimeChunk; ++o) {
+        A[o] = a0;
+        B[o] = make_float2(0.f, 0.f);
+        idx[o] = c0 + o;  // (s * c) mod p at s = 1; c <= H + kPrimeChunk < p
+        if (idx[o] >= p) idx[o] -= p;
+      }
+      for (int sI = 1; sI <= H; ++sI) {
+        float2 x = base[sI * m], y = base[(p - sI) * m];
+        if (INV && m > 1) {
+          x = cmulc(x, __ldg(tw + j * sI * step));
+          y = cmulc(y, __ldg(tw + j * (p - sI) * step));
+        }
+        const float2 P = cadd(x, y), Q = csub(x, y);
+        X0 = cadd(X0, P);
 #pragma unroll
-      for (int o = 0; o < 4; ++o) {
-        const int c = lane + 32 * o;
-        if (c < p) {
-          float2 w = wp[idx[o]];
-          acc[o] = cadd(acc[o], INV ? cmulc(a, w) : cmul(a, w));
-          idx[o] += c;
-          if (idx[o] >= p) idx[o] -= p;
+        for (int o = 0; o < kPrimeChunk; ++o) {
+          const float2 w = cs[idx[o]];
+          A[o].x = fmaf(P.x, w.x, A[o].x);
+          A[o].y = fmaf(P.y, w.x, A[o].y);
+          B[o].x = fmaf(Q.x, w.y, B[o].x);
+          B[o].y = fmaf(Q.y, w.y, B[o].y);
+          idx[o] += c0 + o;
+          if (idx[o] >= p) idx[o] -= p;  // c0 + o <= H + kPrimeChunk - 1 < p, so one step is enough
         }
       }
     }
-    __syncwarp();
+    __syncthreads();
+    if (active) {
+      if (chunk == 0) base[0] = X0;
 #pragma unroll
-    for (int o = 0; o < 4; ++o) {
-      const int c = lane + 32 * o;
-      if (c < p) {
-        float2 r = acc[o];
-        if (!INV && m > 1) r = cmul(r, __ldg(tw + j * c * step));
-        base[c * m] = r;
+      for (int o = 0; o < kPrimeChunk; ++o) {
+        const int c = c0 + o;
+        if (c <= H) {
+          const float2 iB = mul_i(B[o]);
+          float2 xc = INV ? cadd(A[o], iB) : csub(A[o], iB);
+          float2 xq = INV ? csub(A[o], iB) : cadd(A[o], iB);
+          if (!INV && m > 1) {
+            xc = cmul(xc, __ldg(tw + j * c * step));
+            xq = cmul(xq, __ldg(tw + j * (p - c) * step));
+          }
+          base[c * m] = xc;
+          base[(p - c) * m] = xq;
+        }
       }
     }
+    __syncthreads();
   }
-  __syncthreads();
 }
 
 template <bool INV>
@@ -189,7 +231,7 @@ __device__ __forceinline__ void one_pass(float2* buf, int N, int ns, int r, cons
     case 4: pass_small<4, INV>(buf, N, ns, tw); break;
     case 5: pass_small<5, INV>(buf, N, ns, tw); break;
     case 7: pass_small<7, INV>(buf, N, ns, tw); break;
-    default: pass_generic<INV>(buf, N, ns, r, tw, wp); break;
+    default: pass_prime<INV>(buf, N, ns, r, tw, wp); break;
   }
 }
 
@@ -291,13 +333,16 @@ __device__ __forceinline__ double block_excl_scan(double v, double* red /* smem 
 
 __global__ void __launch_bounds__(kSssThreads, 1)
 sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict__ plans,
-           const float2* __restrict__ tables, const float* __restrict__ scores, float* __restrict__ smoothed,
-           int32_t* __restrict__ kstar_out, float2* __restrict__ scratch, int64_t scratch_per_block) {
+           const float2* __restrict__ tables, const float* scores, float* smoothed /* may alias scores */,
+           int32_t* __restrict__ kstar_out, float2* __restrict__ scratch, int64_t scratch_per_block,
+           const int32_t* __restrict__ budgets, const int32_t* __restrict__ cu_kept, int32_t* __restrict__ kept_idx,
+           int* __restrict__ status) {
   extern __shared__ __align__(16) float2 sbuf[];
   __shared__ FftPlan pl;
   __shared__ float2 wp[128];
   __shared__ double red[32];
   __shared__ int s_kstar;
+  __shared__ SelectSmem ssm;
 
   for (int u = blockIdx.x; u < sh.total_heads; u += gridDim.x) {
     const int r = u / sh.heads_per_req;
@@ -311,7 +356,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     const int n = pl.n, N = pl.N, Kb = n / 2;
     float2* buf = pl.in_smem ? sbuf : scratch + static_cast<int64_t>(blockIdx.x) * scratch_per_block;
     const float* x = scores + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P;
-    float* y = smoothed + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P;
+    float* y = smoothed ? smoothed + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P : nullptr;
 
     // 1. load (packed: z_m = x_2m + i x_2m+1)
     if (pl.packed) {
@@ -327,7 +372,8 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     else
       fft_dif(buf, pl.seq, tables, wp);
     const bool direct = !pl.bluestein;
-#define POS(k) (direct ? seq_pos(pl.seq, (k)) : (k))
+    const int* pos_tab = reinterpret_cast<const int*>(tables + pl.pos_offset);  // where the forward pass left each bin
+#define POS(k) (direct ? __ldg(pos_tab + (k)) : (k))
 
     // 3. packed: turn Z into the real sequence's spectrum F, pairwise in place.
     //    Slot of bin 0 holds (F_0, F_N), both real.
@@ -427,17 +473,48 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
       fft_dit_inv(buf, pl.seq, tables, wp);
 #undef POS
 
-    // 7. residual mix
+    // 7. residual mix. `smoothed` (optional) gets the result; when budgets are given the result
+    //    also stays in the work buffer, as order-preserving keys, for the selection below.
     const float inv = 1.f / static_cast<float>(N), al = sh.alpha, om = 1.f - sh.alpha;
+    const bool sel = budgets != nullptr;
+    uint32_t* keys = reinterpret_cast<uint32_t*>(buf);
     if (pl.packed) {
       for (int m = threadIdx.x; m < N; m += kSssThreads) {
         float2 z = buf[m];
         const float x0 = x[2 * m], x1 = x[2 * m + 1];
-        y[2 * m] = fmaf(al, z.x * inv, om * x0);
-        y[2 * m + 1] = fmaf(al, z.y * inv, om * x1);
+        const float y0 = fmaf(al, z.x * inv, om * x0), y1 = fmaf(al, z.y * inv, om * x1);
+        if (y) {
+          y[2 * m] = y0;
+          y[2 * m + 1] = y1;
+        }
+        if (sel) *reinterpret_cast<uint2*>(keys + 2 * m) = make_uint2(score_key(y0), score_key(y1));
       }
     } else {
-      for (int m = threadIdx.x; m < N; m += kSssThreads) y[m] = fmaf(al, buf[m].x * inv, om * x[m]);
+      // key m lands in the slot of complex element m / 2: read a batch, then write it
+      for (int m0 = 0; m0 < N; m0 += kSssThreads) {
+        const int m = m0 + threadIdx.x;
+        float ym = 0.f;
+        if (m < N) {
+          ym = fmaf(al, buf[m].x * inv, om * x[m]);
+          if (y) y[m] = ym;
+        }
+        if (sel) {
+          __syncthreads();
+          if (m < N) keys[m] = score_key(ym);
+          __syncthreads();
+        }
+      }
+    }
+    if (sel) {
+      // 8. top-k of the smoothed scores, straight from the work buffer
+      const int P = rq.P, W = sh.window;
+      int k = budgets[u] - W;
+      if (k < 0 || k > P) {
+        if (threadIdx.x == 0) atomicExch(status, AUDIOKV_EDEVICE);
+        k = k < 0 ? 0 : P;
+      }
+      __syncthreads();
+      select_topk([&](int j) -> uint32_t { return keys[j]; }, P, W, k, kept_idx + cu_kept[u], &ssm, status);
     }
   }
 }
@@ -458,6 +535,10 @@ __global__ void fft_table_kernel(const FftPlan* __restrict__ plans, int n_plans,
       sincospi(2.0 * k / pl.n, &s, &c);
       tables[pl.post_offset + k] = make_float2(static_cast<float>(c), static_cast<float>(-s));
     }
+  }
+  if (!pl.bluestein) {
+    int* pos_tab = reinterpret_cast<int*>(tables + pl.pos_offset);
+    for (int k = gid; k < pl.N; k += gsz) pos_tab[k] = seq_pos(pl.seq, k);
   }
   if (pl.bluestein) {
     const int N = pl.N, M = pl.M;
@@ -505,12 +586,14 @@ cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_pl
 
 cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_plans, const float2* d_tables,
                        const float* scores, float* smoothed, int32_t* kstar, float2* scratch,
-                       int64_t scratch_per_block, int grid, size_t smem_bytes, Launch ln) {
+                       int64_t scratch_per_block, int grid, size_t smem_bytes, const int32_t* budgets,
+                       const int32_t* cu_kept, int32_t* kept_idx, int* status, Launch ln) {
   cudaError_t e = cudaFuncSetAttribute(sss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   if (e != cudaSuccess) return e;
   sss_kernel<<<grid, kSssThreads, smem_bytes, ln.stream>>>(sh, d_reqs, d_plans, d_tables, scores, smoothed, kstar,
-                                                           scratch, scratch_per_block);
-  ln.done("sss");
+                                                           scratch, scratch_per_block, budgets, cu_kept, kept_idx,
+                                                           status);
+  ln.done(budgets ? "sss_select" : "sss");
   return cudaGetLastError();
 }
 
