@@ -123,7 +123,8 @@ def run_cuda(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     spec = wl.config(1)
-    w = wl.generate(spec, seed=rank)          # every rank evicts its own request: no exchange step
+    w = wl.generate(spec, seed=rank, layers=args.layers)   # every rank evicts its own request: no exchange step
+    spec = w.spec
     L = spec.seq_lens[0]
     prob = B.Problem.from_workload(w)
     tb = [int(x) for x in w.total_budget]
@@ -319,6 +320,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline (profiling runs)")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="truncate the stack to its first LAYERS layers (small cases for profiler captures; not a bench line)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
 #include <string>
 #include <vector>
 
@@ -21,7 +22,7 @@ constexpr int kMaxHeadsPerReq = 2048;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {  // byte offsets inside the workspace
-  size_t status, reqs, plans, tables, stats, fft_scratch, scores, kstar, end;
+  size_t status, reqs, plans, tables, units, stats, fft_scratch, scores, kstar, end;
 };
 
 struct Plan {
@@ -32,6 +33,8 @@ struct Plan {
   Shape sh{};
   std::vector<ReqDesc> reqs;
   std::vector<FftPlan> fft;
+  std::vector<ScoreUnit> units;   // sweep 1 (all keys, ascending) then sweep 2 (prefix keys, descending)
+  int n_units1 = 0, n_units2 = 0;
   int64_t table_len = 0;        // float2 elements
   int64_t scores_len = 0;
   int max_L = 0, max_P = 0;
@@ -237,6 +240,38 @@ int build_plan(const audiokv_params* p, Plan* pl) {
     d.fft_plan = found;
   }
   pl->n_slab = (pl->max_L + kSlabKeys - 1) / kSlabKeys;
+  // Schedule of the tensor-core scoring: sweep 1 walks the heads in order; sweep 2 walks them backwards, since the
+  // heads sweep 1 touched last are the ones still in L2.
+  pl->units.clear();
+  for (int sweep = 1; sweep <= 2; ++sweep) {
+    const size_t first = pl->units.size();
+    for (int r = 0; r < p->n_req; ++r) {
+      const ReqDesc& d = pl->reqs[r];
+      const int range = sweep == 1 ? d.L : d.P;
+      const int slabs = (range + kSlabKeys - 1) / kSlabKeys;
+      for (int hr = 0; hr < sh.heads_per_req; ++hr)
+        for (int sl = 0; sl < slabs; ++sl) {
+          ScoreUnit un{};
+          un.u = d.head_base + hr;
+          un.r = r;
+          un.l = hr / p->n_kv_heads;
+          un.h = hr % p->n_kv_heads;
+          un.slab = sl;
+          un.kt0 = sl * kSlabKeys;
+          const int end = range < un.kt0 + kSlabKeys ? range : un.kt0 + kSlabKeys;
+          un.n_tiles = (end - un.kt0 + 127) / 128;
+          un.P = d.P;
+          un.score_base = d.score_offset + static_cast<int64_t>(hr) * d.P;
+          un.head_slabs = (d.L + kSlabKeys - 1) / kSlabKeys;
+          pl->units.push_back(un);
+        }
+    }
+    if (sweep == 1) pl->n_units1 = static_cast<int>(pl->units.size());
+    else {
+      pl->n_units2 = static_cast<int>(pl->units.size() - first);
+      std::reverse(pl->units.begin() + first, pl->units.end());
+    }
+  }
   pl->sss_grid = sh.total_heads < 148 ? sh.total_heads : 148;
   int smem_c = 2;
   pl->scratch_per_block = 0;
@@ -253,6 +288,7 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   L.reqs = off;        off = align_up(off + sizeof(ReqDesc) * AUDIOKV_MAX_REQ);
   L.plans = off;       off = align_up(off + sizeof(FftPlan) * kMaxPlans);
   L.tables = off;      off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->table_len));
+  L.units = off;       off = align_up(off + sizeof(ScoreUnit) * pl->units.size());
   L.stats = off;       off = align_up(off + sizeof(float2) * static_cast<size_t>(sh.total_heads) * pl->n_slab * sh.window * sh.group);
   L.fft_scratch = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->scratch_per_block) * pl->sss_grid);
   L.scores = off;      off = align_up(off + sizeof(float) * static_cast<size_t>(pl->scores_len));
@@ -289,6 +325,9 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
     if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.plans, pl.fft.data(), sizeof(FftPlan) * pl.fft.size(),
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess)
       return cuda_fail(ctx, e);
+    if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.units, pl.units.data(), sizeof(ScoreUnit) * pl.units.size(),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+      return cuda_fail(ctx, e);
     Launch ln{stream, &ctx->launches, &ctx->prof};
     e = launch_fft_tables(static_cast<int>(pl.fft.size()), reinterpret_cast<float2*>(ctx->ws + pl.lay.tables),
                           reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans), ln);
@@ -320,8 +359,11 @@ int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cuda
   float2* stats = reinterpret_cast<float2*>(ctx->ws + pl.lay.stats);
   cudaError_t e = cudaErrorNotSupported;
   if (score_umma_takes(pl.sh))
-    e = launch_score_umma(pl.sh, pl.reqs.data(), d_reqs(ctx), q, k, scores, stats, pl.n_slab, kSlabKeys,
-                          d_status(ctx), ln);
+  {
+    const ScoreUnit* units = reinterpret_cast<const ScoreUnit*>(ctx->ws + pl.lay.units);
+    e = launch_score_umma(pl.sh, pl.reqs.data(), units, pl.n_units1, units + pl.n_units1, pl.n_units2, q, k, scores,
+                          stats, pl.n_slab, kSlabKeys, d_status(ctx), ln);
+  }
   if (e == cudaErrorNotSupported)  // fp32 inputs, W * G above 256, or strides the copy engine cannot take
     e = launch_score_simt(pl.sh, d_reqs(ctx), q, k, scores, stats, pl.n_slab, kSlabKeys, ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);

@@ -96,14 +96,25 @@ struct Launch {
 cudaError_t launch_score_simt(const Shape& sh, const ReqDesc* d_reqs, const void* q, const void* k, float* scores,
                               float2* stats_ws, int n_slab, int slab_keys, Launch ln);
 
+// One unit of work of the tensor-core scoring kernel: one slab of one head. The schedule of each sweep is a
+// table of these, built on the host in processing order, so that no role of the kernel divides to find its work.
+struct ScoreUnit {
+  int32_t u, r, l, h;              // flat head, request, layer, KV head
+  int32_t slab, kt0, n_tiles, P;   // slab number, first key, K tiles of 128 keys, prefix length of the request
+  int64_t score_base;              // element offset of the head's scores in a packed score buffer
+  int32_t head_slabs;              // slabs of this head in the statistics buffer (all keys, window included)
+  int32_t pad;
+};
+
 // score_umma.cu: bf16 scoring on the tcgen05 tensor cores (same statistics buffer). score_umma_takes says
 // whether the shape fits the kernel; the launcher returns cudaErrorNotSupported when the strides
 // cannot be described to the copy engine, and the caller then scores with launch_score_simt.
 // h_reqs: host copy of the request table (the tensor maps are encoded on the host).
 bool score_umma_takes(const Shape& sh);
-cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ReqDesc* d_reqs, const void* q,
-                              const void* k, float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status,
-                              Launch ln);
+// units1 / units2: device tables of the two sweeps (build_score_units gives their host form).
+cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, int n_units1,
+                              const ScoreUnit* units2, int n_units2, const void* q, const void* k, float* scores,
+                              float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln);
 
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);

@@ -42,7 +42,7 @@ struct TmapPack {
 
 struct UmmaArgs {
   Shape sh;
-  const ReqDesc* reqs;
+  const ScoreUnit* units;  // this sweep's schedule, in processing order
   float2* stats;
   float* scores;
   int* status;
@@ -55,15 +55,15 @@ struct UmmaArgs {
 };
 
 struct Small {
-  alignas(16) float negc[2][2][256];  // sweep 2: -(max + log2 sum) per row; one copy per group and head parity (read as float4)
+  alignas(16) float negc[2][256];     // sweep 2: -(max + log2 sum) per row, by head parity (read 16 bytes at a time)
   alignas(16) float2 mrg[2][128];     // sweep 1, one row block: the second group's partial statistics
-  alignas(16) ReqDesc reqs[AUDIOKV_MAX_REQ];
+  alignas(16) float part[4][128];     // sweep 2: the second group's partial column sums, by tile number mod 4
   alignas(8) uint64_t k_full[kMaxStages];
   uint64_t k_empty[kMaxStages];
   uint64_t q_full, q_empty;
-  uint64_t acc_full[2], acc_empty[2];
-  uint64_t grp_bar[2];  // one per epilogue group (128 arrivals)
+  uint64_t acc_full[2][2], acc_empty[2][2];  // [group][buffer]: each epilogue group has its own accumulator stream
   uint64_t all_bar;     // both groups (256 arrivals)
+  uint64_t part_full[4];  // sweep 2: the second group's four warps have written part[i]
   uint64_t drain;       // stop path only: the MMAs still in flight
   uint32_t tmem_base;
   int abort;
@@ -165,100 +165,183 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 32 (16) consecutive fp32 columns of this thread's TMEM lane; returns when the data is in registers.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 32 (16) consecutive fp32 columns of this thread's TMEM lane. The load is asynchronous: the
+// registers hold the data only after tmem_wait on the same array (the first wait after a batch
+// of loads waits for all of them), so a thread issues every load of a tile up front.
+#define AKV_R8(r, o) "=r"(r[o]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
+#define AKV_RW8(r, o) "+r"(r[o]), "+r"(r[o + 1]), "+r"(r[o + 2]), "+r"(r[o + 3]), "+r"(r[o + 4]), "+r"(r[o + 5]), "+r"(r[o + 6]), "+r"(r[o + 7])
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
       "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
-      "tcgen05.wait::ld.sync.aligned;\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : AKV_R8(r, 0), AKV_R8(r, 8), AKV_R8(r, 16), AKV_R8(r, 24)
       : "r"(taddr)
       : "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-  uint32_t r[16];
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
-      "tcgen05.wait::ld.sync.aligned;\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : AKV_R8(r, 0), AKV_R8(r, 8)
       : "r"(taddr)
       : "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" : AKV_RW8(r, 0), AKV_RW8(r, 8), AKV_RW8(r, 16), AKV_RW8(r, 24)::"memory");
+}
+__device__ __forceinline__ void tmem_wait(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" : AKV_RW8(r, 0), AKV_RW8(r, 8)::"memory");
+}
+#undef AKV_R8
+#undef AKV_RW8
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-
-// ---- schedule ----------------------------------------------------------------------------
-// A unit is one slab of one head. Units are numbered request by request, head by head.
-struct Unit {
-  int u, r, l, h, slab, kt0, n_tiles, P;
-};
-template <int SWEEP>
-__device__ __forceinline__ Unit decode_unit(const Shape& sh, const ReqDesc* reqs, int idx, int slab_keys) {
-  Unit U{};
-  int base = 0;
-  for (int r = 0; r < sh.n_req; ++r) {
-    const int range = SWEEP == 1 ? reqs[r].L : reqs[r].P;  // sweep 2 needs the prefix keys only
-    const int slabs = (range + slab_keys - 1) / slab_keys;
-    const int cnt = slabs * sh.heads_per_req;
-    if (idx < base + cnt || r == sh.n_req - 1) {
-      const int local = idx - base;
-      const int hr = local / slabs;
-      U.slab = local - hr * slabs;
-      U.r = r;
-      U.u = reqs[r].head_base + hr;
-      U.l = hr / sh.n_kv_heads;
-      U.h = hr - U.l * sh.n_kv_heads;
-      U.kt0 = U.slab * slab_keys;
-      const int end = min(range, U.kt0 + slab_keys);
-      U.n_tiles = (end - U.kt0 + kTileKeys - 1) / kTileKeys;
-      U.P = reqs[r].P;
-      return U;
-    }
-    base += cnt;
-  }
-  return U;
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// Two fp32 values in one 64-bit register: the scale-and-shift before an exponential and the add after
+// it are issued once per pair (fma.rn.f32x2 / add.rn.f32x2), which leaves issue slots to the
+// special-function unit that bounds both sweeps.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 pack2(uint32_t a, uint32_t b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// exp2 of both halves
+__device__ __forceinline__ f32x2 ex2_2(f32x2 x) {
+  float a, b;
+  unpack2(x, a, b);
+  return pack2(ex2(a), ex2(b));
+}
+__device__ __forceinline__ float hsum(f32x2 a, f32x2 b, f32x2 c, f32x2 d) {
+  float x, y;
+  unpack2(add2(add2(a, b), add2(c, d)), x, y);
+  return x + y;
 }
 
-// Sweep 1, 32 logits of one row: running maximum (raw dot products) and sum of exp2.
-template <bool MASKED>
-__device__ __forceinline__ void stats_chunk(float (&z)[32], int col0, int last_col, float sl, float& m_run, float& Z) {
-  if (MASKED) {
+// Sweep 1: N = NH * 32 logits of this thread's row (columns col0 .. col0 + N - 1 of the tile). Updates the
+// row's running maximum (raw dot products) and its sum of exp2 relative to that maximum.
+template <int NH>
+__device__ __forceinline__ void stats_part(uint32_t (&r)[NH][32], bool masked, int col0, int last_col, float sl,
+                                           float& m_run, float& Z) {
+  constexpr int N = NH * 32;
+  if (masked) {
 #pragma unroll
-    for (int c = 0; c < 32; ++c)
-      if (col0 + c > last_col) z[c] = -INFINITY;
+    for (int i = 0; i < N; ++i)
+      if (col0 + i > last_col) r[i >> 5][i & 31] = 0xff800000u;  // -inf
   }
-  float cm = z[0];
+  float cm = __uint_as_float(r[0][0]);
 #pragma unroll
-  for (int c = 1; c < 32; ++c) cm = fmaxf(cm, z[c]);
-  if (MASKED && cm == -INFINITY) return;
+  for (int i = 1; i + 1 < N; i += 2)
+    cm = max3(cm, __uint_as_float(r[i >> 5][i & 31]), __uint_as_float(r[(i + 1) >> 5][(i + 1) & 31]));
+  cm = fmaxf(cm, __uint_as_float(r[NH - 1][31]));
+  if (cm == -INFINITY) return;  // fully masked: adds nothing
   const float m_new = fmaxf(m_run, cm);
-  Z *= ex2((m_run - m_new) * sl);  // first chunk: exp2(-inf) = 0
+  const float rescale = ex2((m_run - m_new) * sl);  // first time: exp2(-inf) = 0
   m_run = m_new;
   const float nb = -m_new * sl;
-  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  const f32x2 sl2 = pack2(sl, sl), nb2 = pack2(nb, nb);
+  f32x2 a0 = pack2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
 #pragma unroll
-  for (int c = 0; c < 32; c += 4) {
-    a0 += ex2(fmaf(z[c], sl, nb));
-    a1 += ex2(fmaf(z[c + 1], sl, nb));
-    a2 += ex2(fmaf(z[c + 2], sl, nb));
-    a3 += ex2(fmaf(z[c + 3], sl, nb));
+  for (int i = 0; i < N; i += 8) {
+    a0 = add2(a0, ex2_2(fma2(pack2(r[i >> 5][i & 31], r[i >> 5][(i & 31) + 1]), sl2, nb2)));
+    a1 = add2(a1, ex2_2(fma2(pack2(r[i >> 5][(i & 31) + 2], r[i >> 5][(i & 31) + 3]), sl2, nb2)));
+    a2 = add2(a2, ex2_2(fma2(pack2(r[i >> 5][(i & 31) + 4], r[i >> 5][(i & 31) + 5]), sl2, nb2)));
+    a3 = add2(a3, ex2_2(fma2(pack2(r[i >> 5][(i & 31) + 6], r[i >> 5][(i & 31) + 7]), sl2, nb2)));
   }
-  Z += (a0 + a1) + (a2 + a3);
+  Z = fmaf(Z, rescale, hsum(a0, a1, a2, a3));
+}
+// One tile of sweep 1, NCH chunks of 32 columns: the next chunk's TMEM load runs under the arithmetic of this one.
+template <int NCH>
+__device__ __forceinline__ void stats_tile(uint32_t taddr, bool live, bool masked, int col0, int last_col, float sl,
+                                           float& m_run, float& Z) {
+  uint32_t ra[1][32], rb[1][32];
+  tmem_ld32_issue(taddr, ra[0]);
+#pragma unroll
+  for (int c = 0; c < NCH; c += 2) {
+    tmem_wait(ra[0]);
+    if (c + 1 < NCH) tmem_ld32_issue(taddr + (c + 1) * 32, rb[0]);
+    if (live) stats_part<1>(ra, masked, col0 + c * 32, last_col, sl, m_run, Z);  // padding rows only take part in the loads
+    __syncwarp();  // a warp may hold live and padding rows: rejoin before the warp-wide TMEM instructions
+    if (c + 1 < NCH) {
+      tmem_wait(rb[0]);
+      if (c + 2 < NCH) tmem_ld32_issue(taddr + (c + 2) * 32, ra[0]);
+      if (live) stats_part<1>(rb, masked, col0 + (c + 1) * 32, last_col, sl, m_run, Z);
+      __syncwarp();
+    }
+  }
+}
+
+// Sweep 2: N logits of this thread's key against N query rows; nc = their -(max + log2 sum), 16-byte aligned.
+// Adds exp2(z * sl + nc[row]) into four pairs of partial sums.
+template <int N>
+__device__ __forceinline__ void colsum_part(const uint32_t (&r)[N], const float* __restrict__ nc, f32x2 sl2, f32x2& a0,
+                                            f32x2& a1, f32x2& a2, f32x2& a3) {
+  const ulonglong2* nc2 = reinterpret_cast<const ulonglong2*>(nc);
+#pragma unroll
+  for (int j = 0; j < N; j += 8) {
+    const ulonglong2 v = nc2[j >> 2], w = nc2[(j >> 2) + 1];
+    a0 = add2(a0, ex2_2(fma2(pack2(r[j], r[j + 1]), sl2, v.x)));
+    a1 = add2(a1, ex2_2(fma2(pack2(r[j + 2], r[j + 3]), sl2, v.y)));
+    a2 = add2(a2, ex2_2(fma2(pack2(r[j + 4], r[j + 5]), sl2, w.x)));
+    a3 = add2(a3, ex2_2(fma2(pack2(r[j + 6], r[j + 7]), sl2, w.y)));
+  }
+}
+// One tile of sweep 2: this group's n_u (<= 8) units of 16 TMEM columns starting at taddr; nc points at the
+// first of its query rows. Chunks of 32 columns (and a last one of 16), each loaded under the arithmetic of
+// the one before.
+__device__ __forceinline__ float colsum_tile(uint32_t taddr, int n_u, const float* __restrict__ nc, float sl) {
+  const int n32 = n_u >> 1;
+  const bool tail = (n_u & 1) != 0;
+  uint32_t ra[32], rb[32], rt[16];
+  if (n32 > 0) tmem_ld32_issue(taddr, ra);
+  else if (tail) tmem_ld16_issue(taddr, rt);
+  const f32x2 sl2 = pack2(sl, sl);
+  f32x2 a0 = pack2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
+#pragma unroll
+  for (int c = 0; c < 4; c += 2) {
+    if (c < n32) {
+      tmem_wait(ra);
+      if (c + 1 < n32) tmem_ld32_issue(taddr + (c + 1) * 32, rb);
+      else if (tail) tmem_ld16_issue(taddr + n32 * 32, rt);
+      colsum_part<32>(ra, nc + c * 32, sl2, a0, a1, a2, a3);
+    }
+    if (c + 1 < n32) {
+      tmem_wait(rb);
+      if (c + 2 < n32) tmem_ld32_issue(taddr + (c + 2) * 32, ra);
+      else if (tail) tmem_ld16_issue(taddr + n32 * 32, rt);
+      colsum_part<32>(rb, nc + (c + 1) * 32, sl2, a0, a1, a2, a3);
+    }
+  }
+  if (tail) {
+    tmem_wait(rt);
+    colsum_part<16>(rt, nc + n32 * 32, sl2, a0, a1, a2, a3);
+  }
+  return hsum(a0, a1, a2, a3);
 }
 
 template <int SWEEP, int D>
@@ -289,17 +372,18 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
     }
     mbar_init(smem_u32(&sm->q_full), 1);
     mbar_init(smem_u32(&sm->q_empty), 1);
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&sm->acc_full[b]), 1);
-      mbar_init(smem_u32(&sm->acc_empty[b]), both ? 8 : 4);
-      mbar_init(smem_u32(&sm->grp_bar[b]), 128);
+    for (int g = 0; g < 2; ++g) {
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(smem_u32(&sm->acc_full[g][b]), 1);
+        mbar_init(smem_u32(&sm->acc_empty[g][b]), 4);
+      }
     }
     mbar_init(smem_u32(&sm->all_bar), 256);
+    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sm->part_full[i]), 4);
     mbar_init(smem_u32(&sm->drain), 1);
     sm->abort = 0;
     fence_barrier_init();
   }
-  for (int r = threadIdx.x; r < sh.n_req; r += kThreads) sm->reqs[r] = a.reqs[r];
   {  // rows of the Q tile that no copy ever writes must read as zero
     uint4* qz = reinterpret_cast<uint4*>(q_s);
     const int n16 = KB * q_blk / 16;
@@ -316,20 +400,30 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = sm->tmem_base;
-  const ReqDesc* reqs = sm->reqs;
 
   const int unit_begin = static_cast<int>(static_cast<int64_t>(blockIdx.x) * a.n_units / gridDim.x);
   const int unit_end = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * a.n_units / gridDim.x);
-  // Sweep 2 walks the units backwards: the heads sweep 1 touched last are the ones still in L2.
-  auto unit_index = [&](int n) { return SWEEP == 2 ? a.n_units - 1 - n : n; };
+
+  // Every tile is split between the two epilogue groups, and each group gets its share through its own
+  // pair of accumulator buffers (TMEM columns (2 b + g) * 128 ..), filled by its own MMAs: the groups
+  // then run half a tile apart instead of in step, and one group's exponentials cover the other's
+  // loads and maxima.
+  //   sweep 1, two row blocks: group g = row block g, all 128 keys;
+  //   sweep 1, one row block:  group g = keys 64 g .. 64 g + 63 of every row;
+  //   sweep 2: group 0 = the first half of the query rows (in units of 16), group 1 = the rest.
+  const int n16 = a.r_pad >> 4, u_split = (n16 + 1) >> 1;
+  auto share_units = [&](int g) { return g == 0 ? u_split : n16 - u_split; };  // sweep 2: units of 16 rows
 
   if (warp == kProducerWarp) {
     if (lane == 0) {
       // ---- TMA producer ----
-      int it = 0, heads = 0, prev_u = -1;
+      int it = 0, heads = 0, prev_u = -1, s = 0;  // s, ph: slot of the K ring and its phase
+      uint32_t ph = 0;
       bool ok = true;
+      ScoreUnit Unext = a.units[unit_begin < unit_end ? unit_begin : 0];
       for (int n = unit_begin; n < unit_end && ok; ++n) {
-        const Unit U = decode_unit<SWEEP>(sh, reqs, unit_index(n), a.slab_keys);
+        const ScoreUnit U = Unext;
+        if (n + 1 < unit_end) Unext = a.units[n + 1];  // the next descriptor arrives under this unit's work
         if (U.u != prev_u) {
           if (heads > 0) ok = mbar_wait(smem_u32(&sm->q_empty), (heads - 1) & 1, abort);  // MMAs on the old Q are done
           if (!ok) break;
@@ -341,8 +435,6 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
           ++heads;
         }
         for (int t = 0; t < U.n_tiles; ++t, ++it) {
-          const int s = it % S;
-          const uint32_t ph = (it / S) & 1;
           ok = mbar_wait(smem_u32(&sm->k_empty[s]), ph ^ 1, abort);
           if (!ok) break;
           const uint32_t bar = smem_u32(&sm->k_full[s]);
@@ -350,6 +442,10 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
           for (int kb = 0; kb < KB; ++kb)
             tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r], bar, kb * 64, U.kt0 + t * kTileKeys, U.h,
                         U.l);
+          if (++s == S) {
+            s = 0;
+            ph ^= 1;
+          }
         }
       }
       if (*abort) {  // let the copies still in flight land before the CTA goes away
@@ -362,12 +458,14 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
   } else if (warp == kMmaWarp) {
     if (lane == 0) {
       // ---- MMA issuer ----
-      int it = 0, heads = 0, prev_u = -1;
+      int it = 0, heads = 0, prev_u = -1, s = 0;
+      uint32_t ph = 0;
       bool ok = true;
-      const int n_blk = both ? 2 : 1;
-      const uint32_t idesc = SWEEP == 1 ? umma_idesc(128, kTileKeys) : umma_idesc(kTileKeys, a.r_pad);
+      const uint32_t idesc1 = both ? umma_idesc(128, kTileKeys) : umma_idesc(128, kTileKeys / 2);
+      ScoreUnit Unext = a.units[unit_begin < unit_end ? unit_begin : 0];
       for (int n = unit_begin; n < unit_end && ok; ++n) {
-        const Unit U = decode_unit<SWEEP>(sh, reqs, unit_index(n), a.slab_keys);
+        const ScoreUnit U = Unext;
+        if (n + 1 < unit_end) Unext = a.units[n + 1];  // the next descriptor arrives under this unit's work
         if (U.u != prev_u) {
           if (prev_u != -1) umma_commit(smem_u32(&sm->q_empty));
           ok = mbar_wait(smem_u32(&sm->q_full), heads & 1, abort);
@@ -376,31 +474,39 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
           prev_u = U.u;
           ++heads;
         }
-        for (int t = 0; t < U.n_tiles; ++t, ++it) {
-          const int s = it % S;
-          ok = mbar_wait(smem_u32(&sm->k_full[s]), (it / S) & 1, abort);
+        for (int t = 0; t < U.n_tiles && ok; ++t, ++it) {
+          ok = mbar_wait(smem_u32(&sm->k_full[s]), ph, abort);
           if (!ok) break;
           const int b = it & 1;
-          ok = mbar_wait(smem_u32(&sm->acc_empty[b]), ((it >> 1) & 1) ^ 1, abort);
-          if (!ok) break;
-          tc_fence_after();
           const uint32_t k_addr = smem_u32(k_s + s * kKStage);
           const uint32_t q_addr = smem_u32(q_s);
-          for (int blk = 0; blk < n_blk; ++blk) {
-            const uint32_t d_tmem = tmem_base + b * kAccCols + blk * 128;
+          for (int g = 0; g < 2; ++g) {
+            if (SWEEP == 2 && share_units(g) == 0) continue;
+            ok = mbar_wait(smem_u32(&sm->acc_empty[g][b]), ((it >> 1) & 1) ^ 1, abort);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (2 * b + g) * 128;
+            // byte offsets of the group's share inside the Q tile / the K tile (multiples of 1024: whole 8-row groups)
+            const uint32_t q_off = SWEEP == 1 ? (both ? g * (128 * 128) : 0) : (g == 0 ? 0 : u_split * 16 * 128);
+            const uint32_t k_off = SWEEP == 1 && !both ? g * (64 * 128) : 0;
+            const uint32_t idesc = SWEEP == 1 ? idesc1 : umma_idesc(kTileKeys, share_units(g) * 16);
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
 #pragma unroll
               for (int ks = 0; ks < 4; ++ks) {
-                const uint64_t dq = umma_desc(q_addr + kb * q_blk + blk * (128 * 128) + ks * 32);
-                const uint64_t dk = umma_desc(k_addr + kb * kKBlk + ks * 32);
+                const uint64_t dq = umma_desc(q_addr + kb * q_blk + q_off + ks * 32);
+                const uint64_t dk = umma_desc(k_addr + kb * kKBlk + k_off + ks * 32);
                 if (SWEEP == 1) umma_bf16(d_tmem, dq, dk, idesc, (kb | ks) != 0);
                 else umma_bf16(d_tmem, dk, dq, idesc, (kb | ks) != 0);
               }
             }
+            umma_commit(smem_u32(&sm->acc_full[g][b]));
           }
           umma_commit(smem_u32(&sm->k_empty[s]));
-          umma_commit(smem_u32(&sm->acc_full[b]));
+          if (++s == S) {
+            s = 0;
+            ph ^= 1;
+          }
         }
       }
       if (*abort) {  // TMEM must not be released under MMAs that are still running
@@ -410,112 +516,116 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
     }
   } else {
     // ---- epilogue: two groups of four warps; warp w reads TMEM lanes 32 (w % 4) .. +31 ----
+    // Both groups work on every tile, so that the MMAs of the next tile (other accumulator buffer)
+    // run under the arithmetic of this one:
+    //   sweep 1, two row blocks: group g owns row block g (128 key columns per thread);
+    //   sweep 1, one row block:  group g owns key columns 64 g .. 64 g + 63 of every row;
+    //   sweep 2: group 0 sums over the first half of the query rows, group 1 over the rest and hands
+    //            its partial sums to group 0 through shared memory.
     const int g = warp >> 2, quarter = warp & 3;
     const int gl = quarter * 32 + lane;  // thread index inside the group = TMEM lane
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     const float sl = sh.scale_log2e;
     int it = 0, prev_u = -1, n_done = 0, heads = 0;
-    uint32_t grp_phase = 0, all_phase = 0;
+    uint32_t all_phase = 0;
     bool ok = true;
+    const int row = (both ? g * 128 : 0) + gl;   // sweep 1: this thread's query row
+    const int col0 = both ? 0 : g * 64;          // sweep 1: first key column of its share
+    const int win_i = row / G;                   // window row of that query row
+    const bool live = row < R;
+    const int u0 = g == 0 ? 0 : u_split, n_u = share_units(g);  // sweep 2: this group's units of 16 query rows
+    ScoreUnit Unext = a.units[unit_begin < unit_end ? unit_begin : 0];
     for (int n = unit_begin; n < unit_end && ok; ++n, ++n_done) {
-      const Unit U = decode_unit<SWEEP>(sh, reqs, unit_index(n), a.slab_keys);
+      const ScoreUnit U = Unext;
+      if (n + 1 < unit_end) Unext = a.units[n + 1];
       if (SWEEP == 2 && U.u != prev_u) {
-        // merge the slabs' statistics of this head: negc[row] = -(max + log2 sum); +/-inf rows give 0
-        const int slabs = (reqs[U.r].L + a.slab_keys - 1) / a.slab_keys;
-        const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.n_slab * R;
-        for (int row = gl; row < 256; row += 128) {
-          float c = -INFINITY;
-          if (row < R) {
-            float M = -INFINITY;
-            for (int s = 0; s < slabs; ++s) M = fmaxf(M, hs[static_cast<int64_t>(s) * R + row].x);
-            float Zt = 0.f;
-            for (int s = 0; s < slabs; ++s) {
-              const float2 st = hs[static_cast<int64_t>(s) * R + row];
-              if (st.y > 0.f) Zt += st.y * exp2f(st.x - M);
+        // Merge the slabs' statistics of this head: negc[row] = -(max + log2 sum); padding rows get -inf.
+        // One row per epilogue thread, eight independent loads in flight at a time.
+        const int slabs = U.head_slabs;
+        const int rr = g * 128 + gl;
+        float c = -INFINITY;
+        if (rr < R) {
+          const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.n_slab * R + rr;
+          float M = -INFINITY, Zt = 0.f;
+          for (int s0 = 0; s0 < slabs; s0 += 8) {
+            float2 st[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              st[i] = s0 + i < slabs ? __ldg(hs + static_cast<int64_t>(s0 + i) * R) : make_float2(-INFINITY, 0.f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              if (st[i].y > 0.f) {
+                const float m_new = fmaxf(M, st[i].x);
+                Zt = Zt * exp2f(M - m_new) + st[i].y * exp2f(st[i].x - m_new);  // first: 0 * exp2(-inf) = 0
+                M = m_new;
+              }
             }
-            c = -(M + log2f(Zt));
           }
-          // two copies by head parity: a slower warp of the group may still read the previous head's
-          sm->negc[g][heads & 1][row] = c;
+          c = -(M + log2f(Zt));
         }
+        // two copies by head parity: a slower warp may still read the previous head's
+        sm->negc[heads & 1][rr] = c;
         ++heads;
-        mbar_arrive(smem_u32(&sm->grp_bar[g]));
-        ok = mbar_wait(smem_u32(&sm->grp_bar[g]), grp_phase, abort);
-        grp_phase ^= 1;
+        mbar_arrive(smem_u32(&sm->all_bar));
+        ok = mbar_wait(smem_u32(&sm->all_bar), all_phase, abort);
+        all_phase ^= 1;
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
       prev_u = U.u;
-      float m_run = -INFINITY, Z = 0.f;  // sweep 1: this thread's row
-      const int row = (both ? g * 128 : 0) + gl;
-      const int win_i = row / G;         // window row of this query row
+      float m_run = -INFINITY, Z = 0.f;  // sweep 1: this thread's row (its share of the columns)
       for (int t = 0; t < U.n_tiles; ++t, ++it) {
         const int b = it & 1;
-        if (!both && b != g) continue;   // tiles alternate between the groups
-        ok = mbar_wait(smem_u32(&sm->acc_full[b]), (it >> 1) & 1, abort);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after();
+        const bool has_share = SWEEP == 1 || n_u > 0;
+        if (has_share) {
+          ok = mbar_wait(smem_u32(&sm->acc_full[g][b]), (it >> 1) & 1, abort);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+        }
         const int kt = U.kt0 + t * kTileKeys;
+        const uint32_t taddr = lane_addr + (2 * b + g) * 128;
         if (SWEEP == 1) {
-          const uint32_t taddr = lane_addr + b * kAccCols + (both ? g * 128 : 0);
           const bool masked = kt + kTileKeys - 1 > U.P;  // the tile reaches into the window: causal mask, end of request
           const int last_col = U.P + win_i - kt;         // last visible key of this row, relative to the tile
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            float z[32];
-            tmem_ld32(taddr + c * 32, z);
-            if (row < R) {
-              if (masked) stats_chunk<true>(z, c * 32, last_col, sl, m_run, Z);
-              else stats_chunk<false>(z, c * 32, last_col, sl, m_run, Z);
-            }
-          }
+          if (both) stats_tile<4>(taddr, live, masked, col0, last_col, sl, m_run, Z);
+          else stats_tile<2>(taddr, live, masked, col0, last_col, sl, m_run, Z);
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[g][b]));
         } else {
-          const uint32_t taddr = lane_addr + b * kAccCols;
-          const float* nc = sm->negc[g][(heads - 1) & 1];
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-          const int n32 = a.r_pad >> 5;
-#pragma unroll 1
-          for (int c = 0; c < n32; ++c) {
-            float z[32];
-            tmem_ld32(taddr + c * 32, z);
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              const float4 v = *reinterpret_cast<const float4*>(nc + c * 32 + i);
-              a0 += ex2(fmaf(z[i], sl, v.x));
-              a1 += ex2(fmaf(z[i + 1], sl, v.y));
-              a2 += ex2(fmaf(z[i + 2], sl, v.z));
-              a3 += ex2(fmaf(z[i + 3], sl, v.w));
-            }
+          float acc = 0.f;
+          if (has_share) {
+            acc = colsum_tile(taddr, n_u, sm->negc[(heads - 1) & 1] + u0 * 16, sl);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[g][b]));
           }
-          if (a.r_pad & 16) {
-            float z[16];
-            tmem_ld16(taddr + n32 * 32, z);
-#pragma unroll
-            for (int i = 0; i < 16; i += 4) {
-              const float4 v = *reinterpret_cast<const float4*>(nc + n32 * 32 + i);
-              a0 += ex2(fmaf(z[i], sl, v.x));
-              a1 += ex2(fmaf(z[i + 1], sl, v.y));
-              a2 += ex2(fmaf(z[i + 2], sl, v.z));
-              a3 += ex2(fmaf(z[i + 3], sl, v.w));
-            }
+          const int slot = it & 3;
+          if (g == 1) {
+            sm->part[slot][gl] = acc;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm->part_full[slot]));
+          } else {
+            // Slot it & 3 is written again four tiles on. By then the MMAs of tile it + 4 have been issued,
+            // so this group has released the buffer of tile it + 2, which it does after the read below.
+            ok = mbar_wait(smem_u32(&sm->part_full[slot]), (it >> 2) & 1, abort);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const int key = kt + gl;
+            if (key < U.P)
+              a.scores[U.score_base + key] =
+                  acc + sm->part[slot][gl];
           }
-          const int key = kt + gl;
-          if (key < U.P)
-            a.scores[reqs[U.r].score_offset + static_cast<int64_t>(U.u - reqs[U.r].head_base) * U.P + key] =
-                (a0 + a1) + (a2 + a3);
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[b]));
       }
       if (!ok) break;
       if (SWEEP == 1) {
         float2* out = a.stats + (static_cast<int64_t>(U.u) * a.n_slab + U.slab) * R;
         if (both) {
-          if (row < R) out[row] = make_float2(m_run * sl, Z);
+          if (live) out[row] = make_float2(m_run * sl, Z);
         } else {
-          // one row block: both groups hold partial statistics of the same rows
+          // one row block: the two groups hold the statistics of the two column halves of the same rows
           float2* mg = sm->mrg[n_done & 1];
           if (g == 1) mg[gl] = make_float2(m_run, Z);
           mbar_arrive(smem_u32(&sm->all_bar));
@@ -523,7 +633,7 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
           all_phase ^= 1;
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          if (g == 0 && row < R) {
+          if (g == 0 && live) {
             const float2 o = mg[gl];
             const float M = fmaxf(m_run, o.x);
             float Zt = 0.f;
@@ -596,9 +706,9 @@ bool score_umma_takes(const Shape& sh) {
   return room >= 2 * stage;
 }
 
-cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ReqDesc* d_reqs, const void* q,
-                              const void* k, float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status,
-                              Launch ln) {
+cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, int n_units1,
+                              const ScoreUnit* units2, int n_units2, const void* q, const void* k, float* scores,
+                              float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln) {
   if (!score_umma_takes(sh) || slab_keys % kTileKeys) return cudaErrorNotSupported;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
@@ -621,7 +731,6 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ReqD
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorNotSupported;
   }
-  int n_units1 = 0, n_units2 = 0;
   for (int r = 0; r < sh.n_req; ++r) {
     const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(h_reqs[r].L),
                                 static_cast<cuuint64_t>(sh.n_kv_heads), static_cast<cuuint64_t>(sh.n_layers)};
@@ -635,13 +744,10 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ReqD
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorNotSupported;
-    n_units1 += sh.heads_per_req * ((h_reqs[r].L + slab_keys - 1) / slab_keys);
-    n_units2 += sh.heads_per_req * ((h_reqs[r].P + slab_keys - 1) / slab_keys);
   }
 
   UmmaArgs args{};
   args.sh = sh;
-  args.reqs = d_reqs;
   args.stats = stats_ws;
   args.scores = scores;
   args.status = status;
@@ -661,6 +767,7 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ReqD
 
 #define AKV_SWEEP(SW, DD, UNITS)                                                           \
   args.n_units = (UNITS);                                                                  \
+  args.units = SW == 1 ? units1 : units2;                                                  \
   e = launch_sweep<SW, DD>(tm, args, (UNITS) < n_sm ? (UNITS) : n_sm, smem, ln.stream);     \
   if (e != cudaSuccess) return e;                                                          \
   ln.done(SW == 1 ? "score_umma_stats" : "score_umma_colsum")
