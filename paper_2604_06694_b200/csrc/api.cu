@@ -140,6 +140,12 @@ bool factor_len(int N, FftSeq* sq) {
   return true;
 }
 
+// float2 slots of shared memory a plan's block needs: the work buffer, and with tables N (W_N) + N/2 + 1 (post) + N/4 + 1 (positions)
+int sss_smem_complex(const FftPlan& fp, bool with_tables) {
+  const int len = fp.bluestein ? fp.M : fp.N;
+  return len + (with_tables ? fp.N + fp.N / 2 + 1 + fp.N / 4 + 1 : 0);
+}
+
 void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
   memset(fp, 0, sizeof(*fp));
   fp->n = n;
@@ -159,6 +165,8 @@ void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
     buf_len = M;
   }
   fp->in_smem = buf_len <= kSssSmemComplex ? 1 : 0;
+  // a direct transform also keeps its tables on chip when buffer + W_N + post-twiddles + uint16 positions fit
+  fp->tabs_smem = (!fp->bluestein && fp->in_smem && N < 65536 && sss_smem_complex(*fp, true) <= kSssSmemComplex) ? 1 : 0;
   fp->seq.tw_offset = *table_len;
   *table_len += fp->seq.N;
   if (fp->packed) {
@@ -277,7 +285,10 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   pl->scratch_per_block = 0;
   for (const FftPlan& fp : pl->fft) {
     const int len = fp.bluestein ? fp.M : fp.N;
-    if (fp.in_smem) smem_c = len > smem_c ? len : smem_c;
+    if (fp.in_smem) {
+      const int need = sss_smem_complex(fp, fp.tabs_smem != 0);
+      smem_c = need > smem_c ? need : smem_c;
+    }
     else pl->scratch_per_block = len > pl->scratch_per_block ? len : pl->scratch_per_block;
   }
   pl->sss_smem = static_cast<size_t>(smem_c) * sizeof(float2);

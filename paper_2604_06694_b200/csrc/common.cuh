@@ -58,6 +58,8 @@ struct FftPlan {
   int32_t bluestein; // 1: N goes through a chirp-z convolution of length M (a power of two)
   int32_t M;         // convolution length (bluestein only)
   int32_t in_smem;   // 1: the work buffer fits in shared memory
+  int32_t tabs_smem; // 1: twiddles, post-twiddles and bin positions are staged in shared memory after the buffer
+  int32_t pad_;
   FftSeq seq;        // passes for length N (direct) or M (bluestein)
   int64_t chirp_offset;   // float2 index of c_j = exp(-i pi j^2 / N), j in [0, N)      (bluestein)
   int64_t filter_offset;  // float2 index of FFT_M of the wrapped conjugate chirp / M    (bluestein)
@@ -91,6 +93,28 @@ struct Launch {
     }
   }
 };
+
+// Programmatic dependent launch: a kernel launched with launch_chained may be set up on the SMs while the
+// kernel before it on the stream is still draining. Such a kernel calls chain_wait() before it touches global
+// memory (it returns once every earlier kernel has finished and its writes are visible), and every kernel
+// calls chain_release() at its start so that its successor may be brought in early.
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                           Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
 
 // score_simt.cu: fp32-FMA scoring for any dtype. stats_ws: float2 [total_heads][n_slab][rows].
 cudaError_t launch_score_simt(const Shape& sh, const ReqDesc* d_reqs, const void* q, const void* k, float* scores,

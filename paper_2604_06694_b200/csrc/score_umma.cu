@@ -365,6 +365,7 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
   const int S = a.n_stages;
 
   // ---- set-up ----
+  chain_release();
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(smem_u32(&sm->k_full[s]), 1);
@@ -399,6 +400,7 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  chain_wait();  // everything above is local to the CTA; from here on it reads what earlier kernels wrote
   const uint32_t tmem_base = sm->tmem_base;
 
   const int unit_begin = static_cast<int>(static_cast<int64_t>(blockIdx.x) * a.n_units / gridDim.x);
@@ -690,8 +692,7 @@ cudaError_t launch_sweep(const TmapPack& tm, const UmmaArgs& args, int grid, siz
   auto kern = score_umma_kernel<SWEEP, D>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  kern<<<grid, kThreads, smem, stream>>>(tm, args);
-  return cudaGetLastError();
+  return launch_chained(kern, dim3(grid), dim3(kThreads), smem, stream, tm, args);
 }
 
 }  // namespace

@@ -42,6 +42,8 @@ __global__ void __launch_bounds__(256)
 gather_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const int32_t* __restrict__ cu_kept,
               const int32_t* __restrict__ kept_idx, const uint4* __restrict__ k, const uint4* __restrict__ v,
               uint4* __restrict__ k_out, uint4* __restrict__ v_out, int chunks_per_row, int elems_per_chunk) {
+  chain_release();
+  chain_wait();  // kept_idx and cu_kept come from the kernels before
   const int64_t total_rows = cu_kept[sh.total_heads];
   const int64_t n_items = total_rows * chunks_per_row;
   for (int64_t it = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; it < n_items;
@@ -88,10 +90,11 @@ cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t*
   const int esize = sh.dtype == AUDIOKV_F32 ? 4 : 2;
   const int elems_per_chunk = 16 / esize;
   const int chunks_per_row = sh.head_dim / elems_per_chunk;
-  gather_kernel<<<148 * 8, 256, 0, ln.stream>>>(sh, d_reqs, cu_kept, kept_idx, (const uint4*)k, (const uint4*)v,
-                                                 (uint4*)k_out, (uint4*)v_out, chunks_per_row, elems_per_chunk);
+  cudaError_t e = launch_chained(gather_kernel, dim3(148 * 8), dim3(256), 0, ln.stream, sh, d_reqs, cu_kept, kept_idx,
+                                 (const uint4*)k, (const uint4*)v, (uint4*)k_out, (uint4*)v_out, chunks_per_row,
+                                 elems_per_chunk);
   ln.done("gather");
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace akv

@@ -2,8 +2,8 @@
 //
 // A real sequence of even length n is packed into a complex one of length N = n/2
 // (odd n: length N = n with zero imaginary part). The complex transform is an in-place
-// mixed-radix decimation-in-frequency FFT (radices 4, 2, 3, 5, 7 per thread, larger primes up
-// to 127 as paired O(p^2) sums split over warps); its output is left in digit-reversed order and addressed through
+// mixed-radix decimation-in-frequency FFT (radices 2 to 19 one butterfly per thread, larger primes up
+// to 127 as paired O(p^2) sums, one output pair of one butterfly per task); its output is left in digit-reversed order and addressed through
 // pos(k), and the inverse is the matching decimation-in-time chain, so no reordering pass
 // and no second buffer is needed. Lengths with a larger prime factor go through a chirp-z
 // (Bluestein) convolution of power-of-two length M >= 2N - 1 built from the same passes.
@@ -107,7 +107,7 @@ __device__ __forceinline__ void dft_small(float2* v) {
 // Forward (decimation in frequency): DFT_R, then multiply output c by W_ns^{j c}.
 // Inverse (decimation in time): multiply input c by W_ns^{-j c}, then inverse DFT_R.
 template <int R, bool INV>
-__device__ __forceinline__ void pass_small(float2* buf, int N, int ns, const float2* __restrict__ tw) {
+__device__ __forceinline__ void pass_small(float2* buf, int N, int ns, const float2* tw) {
   const int m = ns / R, step = N / ns, nb = N / R;
   for (int t = threadIdx.x; t < nb; t += kSssThreads) {
     const int b = t / m, j = t - b * m;
@@ -119,12 +119,12 @@ __device__ __forceinline__ void pass_small(float2* buf, int N, int ns, const flo
       dft_small<R, false>(v);
       if (m > 1) {
 #pragma unroll
-        for (int c = 1; c < R; ++c) v[c] = cmul(v[c], __ldg(tw + j * c * step));
+        for (int c = 1; c < R; ++c) v[c] = cmul(v[c], tw[j * c * step]);
       }
     } else {
       if (m > 1) {
 #pragma unroll
-        for (int c = 1; c < R; ++c) v[c] = cmulc(v[c], __ldg(tw + j * c * step));
+        for (int c = 1; c < R; ++c) v[c] = cmulc(v[c], tw[j * c * step]);
       }
       dft_small<R, true>(v);
     }
@@ -134,85 +134,297 @@ __device__ __forceinline__ void pass_small(float2* buf, int N, int ns, const flo
   __syncthreads();
 }
 
-// The same pass for an odd prime radix p, 11 <= p <= 127. A length-p DFT is O(p^2); pairing
-// inputs s and p - s (P = a_s + a_{p-s}, Q = a_s - a_{p-s}) gives outputs c and p - c from the
-// same real-by-complex products: X_c = A -/+ iB, A = a_0 + sum_s P_s cos(2 pi s c / p),
-// B = sum_s Q_s sin(2 pi s c / p). Work is split into warp tasks: 32 consecutive butterflies
-// (one per lane) times a chunk of kPrimeChunk output pairs, so the cos/sin reads are
-// broadcasts. A round holds whole butterfly groups only: results stay in registers until
-// every task of the round has read its inputs, then overwrite them.
-constexpr int kPrimeChunk = 6;
+// cos / sin of 2 pi t / R for the odd radices handled by one thread per butterfly with streamed outputs.
+template <int R>
+__device__ __forceinline__ float ocos(int t) {
+  if (R == 11) {
+    switch (t) {
+      case 0: return 1.0f;
+      case 1: return 0.84125353283118121f;
+      case 2: return 0.41541501300188644f;
+      case 3: return -0.142314838273285f;
+      case 4: return -0.65486073394528499f;
+      case 5: return -0.95949297361449737f;
+      case 6: return -0.95949297361449748f;
+      case 7: return -0.65486073394528521f;
+      case 8: return -0.14231483827328523f;
+      case 9: return 0.41541501300188605f;
+      case 10: return 0.84125353283118121f;
+    }
+  }
+  if (R == 13) {
+    switch (t) {
+      case 0: return 1.0f;
+      case 1: return 0.88545602565320991f;
+      case 2: return 0.56806474673115592f;
+      case 3: return 0.12053668025532301f;
+      case 4: return -0.35460488704253545f;
+      case 5: return -0.74851074817110119f;
+      case 6: return -0.97094181742605201f;
+      case 7: return -0.97094181742605212f;
+      case 8: return -0.7485107481711013f;
+      case 9: return -0.3546048870425359f;
+      case 10: return 0.1205366802553232f;
+      case 11: return 0.56806474673115481f;
+      case 12: return 0.88545602565321002f;
+    }
+  }
+  if (R == 17) {
+    switch (t) {
+      case 0: return 1.0f;
+      case 1: return 0.93247222940435581f;
+      case 2: return 0.73900891722065909f;
+      case 3: return 0.44573835577653831f;
+      case 4: return 0.092268359463302016f;
+      case 5: return -0.27366299007208289f;
+      case 6: return -0.60263463637925629f;
+      case 7: return -0.85021713572961399f;
+      case 8: return -0.98297309968390179f;
+      case 9: return -0.98297309968390179f;
+      case 10: return -0.8502171357296141f;
+      case 11: return -0.60263463637925718f;
+      case 12: return -0.27366299007208311f;
+      case 13: return 0.092268359463302432f;
+      case 14: return 0.4457383557765377f;
+      case 15: return 0.73900891722065853f;
+      case 16: return 0.93247222940435581f;
+    }
+  }
+  if (R == 19) {
+    switch (t) {
+      case 0: return 1.0f;
+      case 1: return 0.94581724170063464f;
+      case 2: return 0.78914050939639357f;
+      case 3: return 0.54694815812242692f;
+      case 4: return 0.24548548714079924f;
+      case 5: return -0.082579345472332269f;
+      case 6: return -0.40169542465296942f;
+      case 7: return -0.67728157162574087f;
+      case 8: return -0.87947375120648896f;
+      case 9: return -0.98636130340272232f;
+      case 10: return -0.98636130340272243f;
+      case 11: return -0.8794737512064893f;
+      case 12: return -0.6772815716257411f;
+      case 13: return -0.40169542465296904f;
+      case 14: return -0.082579345472332741f;
+      case 15: return 0.24548548714079879f;
+      case 16: return 0.54694815812242659f;
+      case 17: return 0.78914050939639391f;
+      case 18: return 0.94581724170063464f;
+    }
+  }
+  return 0.f;
+}
+template <int R>
+__device__ __forceinline__ float osin(int t) {
+  if (R == 11) {
+    switch (t) {
+      case 0: return 0.0f;
+      case 1: return 0.54064081745559756f;
+      case 2: return 0.90963199535451833f;
+      case 3: return 0.9898214418809328f;
+      case 4: return 0.75574957435425827f;
+      case 5: return 0.28173255684142967f;
+      case 6: return -0.28173255684142939f;
+      case 7: return -0.75574957435425816f;
+      case 8: return -0.98982144188093268f;
+      case 9: return -0.90963199535451855f;
+      case 10: return -0.54064081745559744f;
+    }
+  }
+  if (R == 13) {
+    switch (t) {
+      case 0: return 0.0f;
+      case 1: return 0.46472317204376851f;
+      case 2: return 0.82298386589365635f;
+      case 3: return 0.99270887409805397f;
+      case 4: return 0.93501624268541483f;
+      case 5: return 0.66312265824079519f;
+      case 6: return 0.23931566428755768f;
+      case 7: return -0.23931566428755743f;
+      case 8: return -0.66312265824079497f;
+      case 9: return -0.93501624268541472f;
+      case 10: return -0.99270887409805397f;
+      case 11: return -0.82298386589365702f;
+      case 12: return -0.4647231720437684f;
+    }
+  }
+  if (R == 17) {
+    switch (t) {
+      case 0: return 0.0f;
+      case 1: return 0.36124166618715292f;
+      case 2: return 0.67369564364655721f;
+      case 3: return 0.89516329135506234f;
+      case 4: return 0.99573417629503447f;
+      case 5: return 0.96182564317281904f;
+      case 6: return 0.7980172272802396f;
+      case 7: return 0.52643216287735606f;
+      case 8: return 0.18374951781657037f;
+      case 9: return -0.18374951781657012f;
+      case 10: return -0.52643216287735584f;
+      case 11: return -0.79801722728023894f;
+      case 12: return -0.96182564317281904f;
+      case 13: return -0.99573417629503447f;
+      case 14: return -0.89516329135506256f;
+      case 15: return -0.67369564364655776f;
+      case 16: return -0.36124166618715303f;
+    }
+  }
+  if (R == 19) {
+    switch (t) {
+      case 0: return 0.0f;
+      case 1: return 0.32469946920468346f;
+      case 2: return 0.61421271268966782f;
+      case 3: return 0.83716647826252855f;
+      case 4: return 0.96940026593933037f;
+      case 5: return 0.99658449300666985f;
+      case 6: return 0.9157733266550574f;
+      case 7: return 0.73572391067313181f;
+      case 8: return 0.47594739303707367f;
+      case 9: return 0.16459459028073403f;
+      case 10: return -0.16459459028073378f;
+      case 11: return -0.47594739303707312f;
+      case 12: return -0.73572391067313159f;
+      case 13: return -0.91577332665505762f;
+      case 14: return -0.99658449300666985f;
+      case 15: return -0.96940026593933049f;
+      case 16: return -0.83716647826252877f;
+      case 17: return -0.61421271268966737f;
+      case 18: return -0.32469946920468373f;
+    }
+  }
+  return 0.f;
+}
 
-template <bool INV>
-__device__ __noinline__ void pass_prime(float2* buf, int N, int ns, int p, const float2* __restrict__ tw,
-                                           float2* cs /* smem [128]: (cos, sin) of 2 pi t / p */) {
-  __syncthreads();
-  for (int t = threadIdx.x; t < p; t += kSssThreads) {
-    const float2 w = __ldg(tw + t * (N / p));
-    cs[t] = make_float2(w.x, -w.y);
+// One in-place pass of an odd radix R in {11, 13, 17, 19}: one thread per butterfly. The inputs are folded into
+// P_s = a_s + a_{R-s}, Q_s = a_s - a_{R-s} (kept in registers); outputs c and R - c come from the same
+// real-by-complex products, X_c = A -/+ iB with A = a_0 + sum_s P_s cos(2 pi s c / R), B = sum_s Q_s sin(2 pi s c / R),
+// and are written back as soon as they are complete.
+template <int R, bool INV>
+__device__ __noinline__ void pass_odd(float2* buf, int N, int ns, const float2* tw) {
+  constexpr int H = (R - 1) / 2;
+  const int m = ns / R, step = N / ns, nb = N / R;
+  for (int t = threadIdx.x; t < nb; t += kSssThreads) {
+    const int b = t / m, j = t - b * m;
+    float2* p = buf + b * ns + j;
+    const float2 v0 = p[0];
+    float2 P[H], Q[H];
+    float2 sum = v0;
+#pragma unroll
+    for (int sI = 1; sI <= H; ++sI) {
+      float2 x = p[sI * m], y = p[(R - sI) * m];
+      if (INV && m > 1) {
+        x = cmulc(x, tw[j * sI * step]);
+        y = cmulc(y, tw[j * (R - sI) * step]);
+      }
+      P[sI - 1] = cadd(x, y);
+      Q[sI - 1] = csub(x, y);
+      sum = cadd(sum, P[sI - 1]);
+    }
+    p[0] = sum;
+#pragma unroll
+    for (int c = 1; c <= H; ++c) {
+      float2 A = v0, B = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int sI = 1; sI <= H; ++sI) {
+        const float cc = ocos<R>((sI * c) % R), ss = osin<R>((sI * c) % R);
+        A.x = fmaf(P[sI - 1].x, cc, A.x);
+        A.y = fmaf(P[sI - 1].y, cc, A.y);
+        B.x = fmaf(Q[sI - 1].x, ss, B.x);
+        B.y = fmaf(Q[sI - 1].y, ss, B.y);
+      }
+      const float2 iB = mul_i(B);
+      float2 xc = INV ? cadd(A, iB) : csub(A, iB);
+      float2 xq = INV ? csub(A, iB) : cadd(A, iB);
+      if (!INV && m > 1) {
+        xc = cmul(xc, tw[j * c * step]);
+        xq = cmul(xq, tw[j * (R - c) * step]);
+      }
+      p[c * m] = xc;
+      p[(R - c) * m] = xq;
+    }
   }
   __syncthreads();
+}
+
+// The same pass for an odd prime radix p, 23 <= p <= 127 (11 to 19 have pass_odd). A length-p DFT is O(p^2); pairing
+// inputs s and p - s (P = a_s + a_{p-s}, Q = a_s - a_{p-s}) gives outputs c and p - c from the
+// same real-by-complex products: X_c = A -/+ iB, A = a_0 + sum_s P_s cos(2 pi s c / p),
+// B = sum_s Q_s sin(2 pi s c / p); c = 0 is the plain sum. One task = one butterfly and one c in
+// [0, (p-1)/2]; consecutive threads take consecutive butterflies of the same c, so the data
+// reads are contiguous and the cos/sin reads are broadcasts. A thread keeps the results of its
+// (at most kPrimeTasks) tasks in registers until every task of the round has read its inputs.
+// The pass twiddles are applied in a sweep of their own (inverse: before, forward: with the
+// write-back).
+constexpr int kPrimeTasks = 6;
+
+template <bool INV>
+__device__ __noinline__ void pass_prime(float2* buf, int N, int ns, int p, const float2* tw,
+                                        float2* cs /* smem [128]: (cos, sin) of 2 pi t / p */) {
+  __syncthreads();
+  for (int t = threadIdx.x; t < p; t += kSssThreads) {
+    const float2 w = tw[t * (N / p)];
+    cs[t] = make_float2(w.x, -w.y);
+  }
   const int m = ns / p, step = N / ns, nb = N / p, H = (p - 1) / 2;
-  const int n_chunks = (H + kPrimeChunk - 1) / kPrimeChunk;
-  const int gpr = 32 / n_chunks;  // butterfly groups per round (n_chunks <= 11)
-  const int n_groups = (nb + 31) / 32;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int chunk = warp % n_chunks, c0 = 1 + chunk * kPrimeChunk;
-  for (int g0 = 0; g0 < n_groups; g0 += gpr) {
-    const int grp = g0 + warp / n_chunks;
-    const int t = grp * 32 + lane;
-    const bool active = warp < gpr * n_chunks && grp < n_groups && t < nb;
-    float2 A[kPrimeChunk], B[kPrimeChunk];
-    float2 X0 = make_float2(0.f, 0.f);
-    float2* base = buf;
-    int j = 0;
-    if (active) {
-      const int b = t / m;
-      j = t - b * m;
-      base = buf + b * ns + j;
-      const float2 a0 = base[0];
-      X0 = a0;
-      int idx[kPrimeChunk];
+  if (INV && m > 1) {
+    // element e = b ns + s m + j gets W_ns^{-j s}
+    for (int e = threadIdx.x; e < N; e += kSssThreads) {
+      const int r = e % ns, sI = r / m, j = r - sI * m;
+      if (sI > 0 && j > 0) buf[e] = cmulc(buf[e], tw[j * sI * step]);
+    }
+  }
+  __syncthreads();
+  const int per_round = max(1, (kPrimeTasks * kSssThreads) / (H + 1));  // butterflies per round
+  for (int b0 = 0; b0 < nb; b0 += per_round) {
+    const int nbr = min(per_round, nb - b0);
+    const int n_task = nbr * (H + 1);
+    float2 A[kPrimeTasks], B[kPrimeTasks];
 #pragma unroll
-      for (int o = 0; o < kPrimeChunk; ++o) {
-        A[o] = a0;
-        B[o] = make_float2(0.f, 0.f);
-        idx[o] = c0 + o;  // (s * c) mod p at s = 1; c <= H + kPrimeChunk < p
-        if (idx[o] >= p) idx[o] -= p;
-      }
-      for (int sI = 1; sI <= H; ++sI) {
-        float2 x = base[sI * m], y = base[(p - sI) * m];
-        if (INV && m > 1) {
-          x = cmulc(x, __ldg(tw + j * sI * step));
-          y = cmulc(y, __ldg(tw + j * (p - sI) * step));
+    for (int i = 0; i < kPrimeTasks; ++i) {
+      const int q = threadIdx.x + kSssThreads * i;
+      A[i] = make_float2(0.f, 0.f);
+      B[i] = make_float2(0.f, 0.f);
+      if (q < n_task) {
+        const int c = q / nbr;
+        const int t = b0 + q - c * nbr;
+        const int b = t / m, j = t - b * m;
+        const float2* base = buf + b * ns + j;
+        float2 a = base[0], bb = make_float2(0.f, 0.f);
+        int idx = c;
+        for (int sI = 1; sI <= H; ++sI) {
+          const float2 x = base[sI * m], y = base[(p - sI) * m];
+          const float2 P = cadd(x, y), Q = csub(x, y);
+          const float2 w = cs[idx];
+          a.x = fmaf(P.x, w.x, a.x);
+          a.y = fmaf(P.y, w.x, a.y);
+          bb.x = fmaf(Q.x, w.y, bb.x);
+          bb.y = fmaf(Q.y, w.y, bb.y);
+          idx += c;
+          if (idx >= p) idx -= p;
         }
-        const float2 P = cadd(x, y), Q = csub(x, y);
-        X0 = cadd(X0, P);
-#pragma unroll
-        for (int o = 0; o < kPrimeChunk; ++o) {
-          const float2 w = cs[idx[o]];
-          A[o].x = fmaf(P.x, w.x, A[o].x);
-          A[o].y = fmaf(P.y, w.x, A[o].y);
-          B[o].x = fmaf(Q.x, w.y, B[o].x);
-          B[o].y = fmaf(Q.y, w.y, B[o].y);
-          idx[o] += c0 + o;
-          if (idx[o] >= p) idx[o] -= p;  // c0 + o <= H + kPrimeChunk - 1 < p, so one step is enough
-        }
+        A[i] = a;
+        B[i] = bb;
       }
     }
     __syncthreads();
-    if (active) {
-      if (chunk == 0) base[0] = X0;
 #pragma unroll
-      for (int o = 0; o < kPrimeChunk; ++o) {
-        const int c = c0 + o;
-        if (c <= H) {
-          const float2 iB = mul_i(B[o]);
-          float2 xc = INV ? cadd(A[o], iB) : csub(A[o], iB);
-          float2 xq = INV ? csub(A[o], iB) : cadd(A[o], iB);
+    for (int i = 0; i < kPrimeTasks; ++i) {
+      const int q = threadIdx.x + kSssThreads * i;
+      if (q < n_task) {
+        const int c = q / nbr;
+        const int t = b0 + q - c * nbr;
+        const int b = t / m, j = t - b * m;
+        float2* base = buf + b * ns + j;
+        if (c == 0) {
+          base[0] = A[i];
+        } else {
+          const float2 iB = mul_i(B[i]);
+          float2 xc = INV ? cadd(A[i], iB) : csub(A[i], iB);
+          float2 xq = INV ? csub(A[i], iB) : cadd(A[i], iB);
           if (!INV && m > 1) {
-            xc = cmul(xc, __ldg(tw + j * c * step));
-            xq = cmul(xq, __ldg(tw + j * (p - c) * step));
+            xc = cmul(xc, tw[j * c * step]);
+            xq = cmul(xq, tw[j * (p - c) * step]);
           }
           base[c * m] = xc;
           base[(p - c) * m] = xq;
@@ -231,13 +443,17 @@ __device__ __forceinline__ void one_pass(float2* buf, int N, int ns, int r, cons
     case 4: pass_small<4, INV>(buf, N, ns, tw); break;
     case 5: pass_small<5, INV>(buf, N, ns, tw); break;
     case 7: pass_small<7, INV>(buf, N, ns, tw); break;
+    case 11: pass_odd<11, INV>(buf, N, ns, tw); break;
+    case 13: pass_odd<13, INV>(buf, N, ns, tw); break;
+    case 17: pass_odd<17, INV>(buf, N, ns, tw); break;
+    case 19: pass_odd<19, INV>(buf, N, ns, tw); break;
     default: pass_prime<INV>(buf, N, ns, r, tw, wp); break;
   }
 }
 
 // Forward transform, natural order in, digit-reversed order out (see seq_pos).
-__device__ __forceinline__ void fft_dif(float2* buf, const FftSeq& sq, const float2* tables, float2* wp) {
-  const float2* tw = tables + sq.tw_offset;
+// tw: W_N^t = exp(-2 pi i t / N), t in [0, N); in shared or global memory.
+__device__ __forceinline__ void fft_dif(float2* buf, const FftSeq& sq, const float2* tw, float2* wp) {
   int ns = sq.N;
   for (int i = 0; i < sq.n_pass; ++i) {
     one_pass<false>(buf, sq.N, ns, sq.radix[i], tw, wp);
@@ -245,8 +461,7 @@ __device__ __forceinline__ void fft_dif(float2* buf, const FftSeq& sq, const flo
   }
 }
 // Inverse (unnormalised, sign +), digit-reversed order in, natural order out.
-__device__ __forceinline__ void fft_dit_inv(float2* buf, const FftSeq& sq, const float2* tables, float2* wp) {
-  const float2* tw = tables + sq.tw_offset;
+__device__ __forceinline__ void fft_dit_inv(float2* buf, const FftSeq& sq, const float2* tw, float2* wp) {
   int ns = 1;
   for (int i = sq.n_pass - 1; i >= 0; --i) {
     ns *= sq.radix[i];
@@ -284,10 +499,10 @@ __device__ __forceinline__ void bluestein(float2* buf, const FftPlan& pl, const 
     buf[j] = v;
   }
   __syncthreads();
-  fft_dif(buf, pl.seq, tables, wp);
+  fft_dif(buf, pl.seq, tables + pl.seq.tw_offset, wp);
   for (int j = threadIdx.x; j < M; j += kSssThreads) buf[j] = cmul(buf[j], __ldg(filt + j));
   __syncthreads();
-  fft_dit_inv(buf, pl.seq, tables, wp);
+  fft_dit_inv(buf, pl.seq, tables + pl.seq.tw_offset, wp);
   for (int j = threadIdx.x; j < N; j += kSssThreads) {
     float2 v = cmul(buf[j], __ldg(chirp + j));
     buf[j] = CONJ ? cconj(v) : v;
@@ -343,7 +558,10 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
   __shared__ double red[32];
   __shared__ int s_kstar;
   __shared__ SelectSmem ssm;
+  chain_release();
+  chain_wait();
 
+  int loaded_plan = -1;  // plan whose tables sit in shared memory
   for (int u = blockIdx.x; u < sh.total_heads; u += gridDim.x) {
     const int r = u / sh.heads_per_req;
     const ReqDesc rq = reqs[r];
@@ -355,6 +573,31 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     __syncthreads();
     const int n = pl.n, N = pl.N, Kb = n / 2;
     float2* buf = pl.in_smem ? sbuf : scratch + static_cast<int64_t>(blockIdx.x) * scratch_per_block;
+    // Tables of a direct transform that fit beside the work buffer are staged in shared memory once per plan:
+    // the passes read twiddles with data-dependent strides, which from global memory costs a round trip each.
+    const float2* tw = tables + pl.seq.tw_offset;
+    const float2* post = tables + pl.post_offset;
+    const int* pos_tab = reinterpret_cast<const int*>(tables + pl.pos_offset);  // where the forward pass left each bin
+    const uint16_t* s_pos = nullptr;
+    if (pl.tabs_smem) {
+      float2* s_tw = sbuf + N;
+      float2* s_post = s_tw + N;
+      uint16_t* sp = reinterpret_cast<uint16_t*>(s_post + N / 2 + 1);
+      if (loaded_plan != rq.fft_plan) {
+        for (int t = threadIdx.x; t < N; t += kSssThreads) {
+          s_tw[t] = __ldg(tw + t);
+          sp[t] = static_cast<uint16_t>(__ldg(pos_tab + t));
+        }
+        if (pl.packed)
+          for (int t = threadIdx.x; t <= N / 2; t += kSssThreads) s_post[t] = __ldg(post + t);
+        loaded_plan = rq.fft_plan;
+      }
+      tw = s_tw;
+      post = s_post;
+      s_pos = sp;
+    } else if (pl.in_smem) {
+      loaded_plan = -1;  // this head's work buffer may run over the staged tables
+    }
     const float* x = scores + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P;
     float* y = smoothed ? smoothed + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P : nullptr;
 
@@ -370,14 +613,12 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     if (pl.bluestein)
       bluestein<false>(buf, pl, tables, wp);
     else
-      fft_dif(buf, pl.seq, tables, wp);
+      fft_dif(buf, pl.seq, tw, wp);
     const bool direct = !pl.bluestein;
-    const int* pos_tab = reinterpret_cast<const int*>(tables + pl.pos_offset);  // where the forward pass left each bin
-#define POS(k) (direct ? __ldg(pos_tab + (k)) : (k))
+#define POS(k) (direct ? (s_pos ? static_cast<int>(s_pos[(k)]) : __ldg(pos_tab + (k))) : (k))
 
     // 3. packed: turn Z into the real sequence's spectrum F, pairwise in place.
     //    Slot of bin 0 holds (F_0, F_N), both real.
-    const float2* post = tables + pl.post_offset;
     if (pl.packed) {
       for (int k = threadIdx.x; k <= N / 2; k += kSssThreads) {
         if (k == 0) {
@@ -391,7 +632,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
           float2 zk = buf[pk], zq = cconj(buf[pq]);
           float2 E = cscale(cadd(zk, zq), 0.5f);
           float2 O = mul_mi(cscale(csub(zk, zq), 0.5f));
-          float2 T = cmul(O, __ldg(post + k));
+          float2 T = cmul(O, post[k]);
           buf[pk] = cadd(E, T);
           buf[pq] = cconj(csub(E, T));
         }
@@ -411,18 +652,36 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
       float2 f = buf[POS(k)];
       return static_cast<double>(f.x) * f.x + static_cast<double>(f.y) * f.y;
     };
+    // each thread owns `per` consecutive bins; up to 8 of their energies stay in registers for the second look
+    double ecache[8];
     double local = 0.0;
-    for (int k = k0; k < k1; ++k) local += energy(k);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      ecache[i] = k0 + i < k1 ? energy(k0 + i) : 0.0;
+      local += ecache[i];
+    }
+    for (int k = k0 + 8; k < k1; ++k) local += energy(k);
     const double before = block_excl_scan(local, red);
     const double total = block_sum(local, red);
     const double thr = static_cast<double>(sh.rho) * total;
     {
       double run = before;
-      for (int k = k0; k < k1; ++k) {
+      bool found = false;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (!found && k0 + i < k1) {
+          run += ecache[i];
+          if (run >= thr) {
+            atomicMin(&s_kstar, k0 + i);
+            found = true;
+          }
+        }
+      }
+      for (int k = k0 + 8; k < k1 && !found; ++k) {
         run += energy(k);
         if (run >= thr) {
           atomicMin(&s_kstar, k);
-          break;
+          found = true;
         }
       }
     }
@@ -451,7 +710,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
           float2 fk = cscale(buf[pk], weight(k)), fq = cconj(cscale(buf[pq], weight(N - k)));
           float2 E = cscale(cadd(fk, fq), 0.5f);
           float2 Tt = cscale(csub(fk, fq), 0.5f);
-          float2 O = cmulc(Tt, __ldg(post + k));
+          float2 O = cmulc(Tt, post[k]);
           float2 iO = mul_i(O);
           buf[pk] = cadd(E, iO);
           buf[pq] = cconj(csub(E, iO));
@@ -470,7 +729,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     if (pl.bluestein)
       bluestein<true>(buf, pl, tables, wp);
     else
-      fft_dit_inv(buf, pl.seq, tables, wp);
+      fft_dit_inv(buf, pl.seq, tw, wp);
 #undef POS
 
     // 7. residual mix. `smoothed` (optional) gets the result; when budgets are given the result
@@ -569,7 +828,7 @@ fft_filter_kernel(const FftPlan* __restrict__ plans, float2* __restrict__ tables
   __syncthreads();
   if (!pl.bluestein) return;
   float2* f = tables + pl.filter_offset;
-  fft_dif(f, pl.seq, tables, wp);
+  fft_dif(f, pl.seq, tables + pl.seq.tw_offset, wp);
   const float inv = 1.f / static_cast<float>(pl.M);
   for (int j = threadIdx.x; j < pl.M; j += kSssThreads) f[j] = cscale(f[j], inv);
 }
