@@ -113,6 +113,38 @@ def kernel_algorithmic_bytes(name, spec, w):
     return 0
 
 
+def kernel_algorithmic_exps(name, spec, w):
+    """exp2 evaluations the softmax of each scoring sweep needs per launch: one per (window row, query head,
+    visible key) in the statistics sweep, one per (window row, query head, prefix key) in the column-sum sweep."""
+    NL, W, Hq = spec.n_layers, spec.window, spec.n_q_heads
+    n = 0
+    for L in spec.seq_lens:
+        P = L - W
+        if "stats" in name:
+            n += NL * Hq * sum(P + i + 1 for i in range(W))
+        else:
+            n += NL * Hq * W * P
+    return n
+
+
+def kernel_roofline(name, ms, spec, w, peaks, sm_max_mhz):
+    """Roofline entry of one kernel: the scoring sweeps are bound by the special-function units (16 exp2 per clock
+    and SM, 148 SMs, at the maximum SM clock), everything else by HBM (measured copy bandwidth)."""
+    nbytes = kernel_algorithmic_bytes(name, spec, w)
+    hbm = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+    if name.startswith("score_umma"):
+        peak = 148 * 16 * (sm_max_mhz or 1965.0) * 1e6 / 1e9      # Gexp2/s
+        ach = kernel_algorithmic_exps(name, spec, w) / (ms * 1e-3) / 1e9
+        return {"kernel": name, "bound": "alu", "achieved": round(ach, 1), "peak": round(peak, 1), "unit": "Gexp2/s",
+                "frac": round(ach / peak, 4), "peak_kind": "148 SMs x 16 exp2/clk x max SM clock",
+                "algorithmic_exp2": kernel_algorithmic_exps(name, spec, w), "algorithmic_bytes": nbytes,
+                "hbm_gbs": round(hbm, 1), "hbm_frac_of_measured": round(hbm / peaks["hbm_gbs"], 4),
+                "traffic": NCU_TRAFFIC_BYTES.get(name)}
+    return {"kernel": name, "bound": "hbm", "achieved": round(hbm, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": round(hbm / peaks["hbm_gbs"], 4), "algorithmic_bytes": nbytes,
+            "traffic": NCU_TRAFFIC_BYTES.get(name)}
+
+
 def run_cuda(args):
     from paper_2604_06694_b200 import binding as B
     rank = int(os.environ.get("RANK", "0"))
@@ -155,6 +187,8 @@ def run_cuda(args):
     stream = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        time.sleep(0.3)                       # nvidia-smi needs a moment to start; the GPU idles meanwhile
     n0 = ctx.launch_count()
     e0.record(stream)
     for _ in range(args.steps):
@@ -167,13 +201,27 @@ def run_cuda(args):
     if world > 1:
         torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
     ms_step = float(t.item()) / args.steps
-    clocks = sampler.stop() if sampler else None
+    clocks = None
+    if sampler:
+        # nvidia-smi delivers a sample every 200 ms: when the timed region was shorter than about a second the
+        # same step loop goes on (untimed) until the sampler has seen a second of this load
+        t_load = ms_total * 1e-3
+        extra = 0
+        while t_load < 1.2:
+            for _ in range(200):
+                step()
+            torch.cuda.synchronize()
+            extra += 200
+            t_load += 200 * ms_step * 1e-3
+        clocks = sampler.stop()
+        clocks["window"] = ("timed region" if extra == 0 else
+                            f"timed region ({args.steps} steps) + {extra} more untimed steps of the same loop")
     assert ctx.last_device_status() == 0
 
     # per-kernel durations: the same loop again with an event after every kernel
     ctx.profile_enable(True)
     per_kernel = {}
-    for _ in range(args.steps):
+    for _ in range(min(args.steps, 200)):
         step()
         for name, ms in ctx.profile_read():
             per_kernel.setdefault(name, []).append(ms)
@@ -232,8 +280,10 @@ def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_m
     kern = {n: statistics.mean(v) for n, v in per_kernel.items()}
     tot = sum(kern.values()) or 1.0
     dom = max(kern, key=kern.get)
-    dom_bytes = kernel_algorithmic_bytes(dom, spec, w)
-    achieved = dom_bytes / (kern[dom] * 1e-3) / 1e9
+    sm_max = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz")
+    per_kernel_roofline = [kernel_roofline(n, v, spec, w, peaks, sm_max) for n, v in kern.items() if n != "allocate"]
+    roof = dict(next(r for r in per_kernel_roofline if r["kernel"] == dom))
+    roof["peak_source"] = peak_kind
     line = {
         "metric": METRIC, "value": round(us_layer, 4), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "higher_is_better": False,
@@ -250,9 +300,8 @@ def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_m
         "gpu_launches": int(launches),
         "kernels_ms": {n: round(v, 5) for n, v in kern.items()},
         "kernel_share": {n: round(v / tot, 4) for n, v in kern.items()},
-        "roofline": {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4), "peak_kind": peak_kind,
-                     "algorithmic_bytes": dom_bytes, "traffic": NCU_TRAFFIC_BYTES.get(dom)},
+        "roofline": roof,
+        "kernel_rooflines": per_kernel_roofline,
         "e2e": None if e2e_ms is None else
                {"value": round(e2e_ms * 1e3 / (NL * world), 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
@@ -315,7 +364,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline (profiling runs)")
