@@ -36,37 +36,57 @@ select_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restric
   }
 }
 
-// Copies the kept rows. One 16-byte chunk of a K row and of the matching V row per thread
-// and step; the head of an output row is found by bisection in cu_kept.
+// Copies the kept rows. A warp takes eight output rows at a time: lanes 0-7 look up the head of one row each
+// (bisection in cu_kept) and its source row; then all lanes copy 16-byte chunks, K chunks first, V chunks after,
+// eight independent loads in flight per lane before the stores. log2_chunks: log2 of the chunks per row.
+constexpr int kGatherRows = 8;
+
 __global__ void __launch_bounds__(256)
 gather_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const int32_t* __restrict__ cu_kept,
               const int32_t* __restrict__ kept_idx, const uint4* __restrict__ k, const uint4* __restrict__ v,
-              uint4* __restrict__ k_out, uint4* __restrict__ v_out, int chunks_per_row, int elems_per_chunk) {
+              uint4* __restrict__ k_out, uint4* __restrict__ v_out, int log2_chunks, int elems_per_chunk) {
   chain_release();
   chain_wait();  // kept_idx and cu_kept come from the kernels before
   const int64_t total_rows = cu_kept[sh.total_heads];
-  const int64_t n_items = total_rows * chunks_per_row;
-  for (int64_t it = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; it < n_items;
-       it += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-    const int64_t row = it / chunks_per_row;
-    const int c = static_cast<int>(it - row * chunks_per_row);
-    int lo = 0, hi = sh.total_heads;  // largest u with cu_kept[u] <= row
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (cu_kept[mid] <= row) lo = mid; else hi = mid;
+  const int64_t n_batches = (total_rows + kGatherRows - 1) / kGatherRows;
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = (blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x) >> 5;
+  const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+  const int chunks = 1 << log2_chunks;
+  for (int64_t bt = warp0; bt < n_batches; bt += n_warps) {
+    const int64_t row0 = bt * kGatherRows;
+    int64_t my_src = 0;  // lane i < 8: first 16-byte chunk of the source row of output row row0 + i
+    if (lane < kGatherRows && row0 + lane < total_rows) {
+      const int64_t row = row0 + lane;
+      int lo = 0, hi = sh.total_heads;  // largest u with cu_kept[u] <= row
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(cu_kept + mid) <= row) lo = mid; else hi = mid;
+      }
+      const int u = lo;
+      const ReqDesc rq = reqs[u / sh.heads_per_req];
+      const int lh = u - rq.head_base;
+      const int l = lh / sh.n_kv_heads, h = lh - l * sh.n_kv_heads;
+      const int tok = __ldg(kept_idx + row);
+      my_src = (rq.kv_offset + l * sh.kv_stride_layer + h * sh.kv_stride_head + tok * sh.kv_stride_tok) / elems_per_chunk;
     }
-    const int u = lo;
-    const int r = u / sh.heads_per_req;
-    const ReqDesc rq = reqs[r];
-    const int lh = u - rq.head_base;
-    const int l = lh / sh.n_kv_heads, h = lh - l * sh.n_kv_heads;
-    const int tok = kept_idx[row];
-    const int64_t src_elem = rq.kv_offset + l * sh.kv_stride_layer + h * sh.kv_stride_head + tok * sh.kv_stride_tok;
-    const int64_t src = src_elem / elems_per_chunk + c;
-    const uint4 kv = __ldg(k + src);
-    const uint4 vv = __ldg(v + src);
-    k_out[it] = kv;
-    v_out[it] = vv;
+    const int n_rows = static_cast<int>(min(static_cast<int64_t>(kGatherRows), total_rows - row0));
+    int64_t so[kGatherRows];  // every lane gets the eight source rows (all lanes take part in the shuffles)
+#pragma unroll
+    for (int i = 0; i < kGatherRows; ++i) so[i] = __shfl_sync(0xffffffffu, my_src, i);
+    for (int c0 = lane; c0 < 2 * chunks; c0 += 32) {
+      const bool is_v = c0 >= chunks;
+      const int c = c0 & (chunks - 1);
+      const uint4* src = is_v ? v : k;
+      uint4* dst = (is_v ? v_out : k_out) + (row0 << log2_chunks) + c;
+      uint4 val[kGatherRows];
+#pragma unroll
+      for (int i = 0; i < kGatherRows; ++i)
+        if (i < n_rows) val[i] = __ldg(src + so[i] + c);
+#pragma unroll
+      for (int i = 0; i < kGatherRows; ++i)
+        if (i < n_rows) dst[static_cast<int64_t>(i) << log2_chunks] = val[i];
+    }
   }
 }
 
@@ -89,9 +109,11 @@ cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t*
                           const void* k, const void* v, void* k_out, void* v_out, Launch ln) {
   const int esize = sh.dtype == AUDIOKV_F32 ? 4 : 2;
   const int elems_per_chunk = 16 / esize;
-  const int chunks_per_row = sh.head_dim / elems_per_chunk;
+  const int chunks_per_row = sh.head_dim / elems_per_chunk;  // 8 .. 64: head_dim is 64, 128 or 256
+  int log2_chunks = 0;
+  while ((1 << log2_chunks) < chunks_per_row) ++log2_chunks;
   cudaError_t e = launch_chained(gather_kernel, dim3(148 * 8), dim3(256), 0, ln.stream, sh, d_reqs, cu_kept, kept_idx,
-                                 (const uint4*)k, (const uint4*)v, (uint4*)k_out, (uint4*)v_out, chunks_per_row,
+                                 (const uint4*)k, (const uint4*)v, (uint4*)k_out, (uint4*)v_out, log2_chunks,
                                  elems_per_chunk);
   ln.done("gather");
   return e;
