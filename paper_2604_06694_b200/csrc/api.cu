@@ -142,7 +142,7 @@ bool factor_len(int N, FftSeq* sq) {
 
 // float2 slots of shared memory a plan's block needs: the work buffer, and with tables N (W_N) + N/2 + 1 (post) + N/4 + 1 (positions)
 int sss_smem_complex(const FftPlan& fp, bool with_tables) {
-  const int len = fp.bluestein ? fp.M : fp.N;
+  const int len = sss_padded(fp.bluestein ? fp.M : fp.N);
   return len + (with_tables ? fp.N + fp.N / 2 + 1 + fp.N / 4 + 1 : 0);
 }
 
@@ -164,7 +164,7 @@ void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
     factor_len(M, &fp->seq);
     buf_len = M;
   }
-  fp->in_smem = buf_len <= kSssSmemComplex ? 1 : 0;
+  fp->in_smem = sss_padded(buf_len) <= kSssSmemComplex ? 1 : 0;
   // a direct transform also keeps its tables on chip when buffer + W_N + post-twiddles + uint16 positions fit
   fp->tabs_smem = (!fp->bluestein && fp->in_smem && N < 65536 && sss_smem_complex(*fp, true) <= kSssSmemComplex) ? 1 : 0;
   fp->seq.tw_offset = *table_len;

@@ -69,6 +69,9 @@ struct FftPlan {
 
 constexpr int kMaxPlans = AUDIOKV_MAX_REQ;
 
+// float2 slots of a shared-memory work buffer of `len` elements: element i sits at i + (i >> 4) (see SkewBuf in sss.cu)
+__host__ __device__ inline int sss_padded(int len) { return len + (len >> 4) + 1; }
+
 // ---- launchers (one per source file) ---------------------------------------------------
 // Optional per-kernel timing: an event after every kernel launch of one call.
 struct Profiler {

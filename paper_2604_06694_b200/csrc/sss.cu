@@ -29,6 +29,21 @@ __device__ __forceinline__ float2 cscale(float2 a, float s) { return make_float2
 __device__ __forceinline__ float2 mul_i(float2 a) { return make_float2(-a.y, a.x); }    // i * a
 __device__ __forceinline__ float2 mul_mi(float2 a) { return make_float2(a.y, -a.x); }   // -i * a
 
+// The work buffer of a transform. In shared memory element i lives at i + (i >> 4): the passes of an in-place
+// transform read with power-of-two strides (and the late ones with strides of a few elements between
+// neighbouring threads), which without the skew puts many lanes on the same banks. sh = 31 switches the skew
+// off (global scratch, tables).
+struct SkewBuf {
+  float2* p;
+  int sh;
+  int off;
+  __device__ __forceinline__ float2& operator[](int i) const {
+    const int e = off + i;
+    return p[e + (e >> sh)];
+  }
+  __device__ __forceinline__ SkewBuf operator+(int d) const { return SkewBuf{p, sh, off + d}; }
+};
+
 // cos / sin of 2 pi t / R for the odd radices handled per thread.
 template <int R>
 __device__ __forceinline__ float rcos(int t) {
@@ -107,11 +122,11 @@ __device__ __forceinline__ void dft_small(float2* v) {
 // Forward (decimation in frequency): DFT_R, then multiply output c by W_ns^{j c}.
 // Inverse (decimation in time): multiply input c by W_ns^{-j c}, then inverse DFT_R.
 template <int R, bool INV>
-__device__ __forceinline__ void pass_small(float2* buf, int N, int ns, const float2* tw) {
+__device__ __forceinline__ void pass_small(SkewBuf buf, int N, int ns, const float2* tw) {
   const int m = ns / R, step = N / ns, nb = N / R;
   for (int t = threadIdx.x; t < nb; t += kSssThreads) {
     const int b = t / m, j = t - b * m;
-    float2* p = buf + b * ns + j;
+    const SkewBuf p = buf + (b * ns + j);
     float2 v[R];
 #pragma unroll
     for (int s = 0; s < R; ++s) v[s] = p[s * m];
@@ -301,12 +316,12 @@ __device__ __forceinline__ float osin(int t) {
 // real-by-complex products, X_c = A -/+ iB with A = a_0 + sum_s P_s cos(2 pi s c / R), B = sum_s Q_s sin(2 pi s c / R),
 // and are written back as soon as they are complete.
 template <int R, bool INV>
-__device__ __noinline__ void pass_odd(float2* buf, int N, int ns, const float2* tw) {
+__device__ __noinline__ void pass_odd(SkewBuf buf, int N, int ns, const float2* tw) {
   constexpr int H = (R - 1) / 2;
   const int m = ns / R, step = N / ns, nb = N / R;
   for (int t = threadIdx.x; t < nb; t += kSssThreads) {
     const int b = t / m, j = t - b * m;
-    float2* p = buf + b * ns + j;
+    const SkewBuf p = buf + (b * ns + j);
     const float2 v0 = p[0];
     float2 P[H], Q[H];
     float2 sum = v0;
@@ -359,7 +374,7 @@ __device__ __noinline__ void pass_odd(float2* buf, int N, int ns, const float2* 
 constexpr int kPrimeTasks = 6;
 
 template <bool INV>
-__device__ __noinline__ void pass_prime(float2* buf, int N, int ns, int p, const float2* tw,
+__device__ __noinline__ void pass_prime(SkewBuf buf, int N, int ns, int p, const float2* tw,
                                         float2* cs /* smem [128]: (cos, sin) of 2 pi t / p */) {
   __syncthreads();
   for (int t = threadIdx.x; t < p; t += kSssThreads) {
@@ -389,7 +404,7 @@ __device__ __noinline__ void pass_prime(float2* buf, int N, int ns, int p, const
         const int c = q / nbr;
         const int t = b0 + q - c * nbr;
         const int b = t / m, j = t - b * m;
-        const float2* base = buf + b * ns + j;
+        const SkewBuf base = buf + (b * ns + j);
         float2 a = base[0], bb = make_float2(0.f, 0.f);
         int idx = c;
         for (int sI = 1; sI <= H; ++sI) {
@@ -415,7 +430,7 @@ __device__ __noinline__ void pass_prime(float2* buf, int N, int ns, int p, const
         const int c = q / nbr;
         const int t = b0 + q - c * nbr;
         const int b = t / m, j = t - b * m;
-        float2* base = buf + b * ns + j;
+        const SkewBuf base = buf + (b * ns + j);
         if (c == 0) {
           base[0] = A[i];
         } else {
@@ -436,7 +451,7 @@ __device__ __noinline__ void pass_prime(float2* buf, int N, int ns, int p, const
 }
 
 template <bool INV>
-__device__ __forceinline__ void one_pass(float2* buf, int N, int ns, int r, const float2* tw, float2* wp) {
+__device__ __forceinline__ void one_pass(SkewBuf buf, int N, int ns, int r, const float2* tw, float2* wp) {
   switch (r) {
     case 2: pass_small<2, INV>(buf, N, ns, tw); break;
     case 3: pass_small<3, INV>(buf, N, ns, tw); break;
@@ -453,7 +468,7 @@ __device__ __forceinline__ void one_pass(float2* buf, int N, int ns, int r, cons
 
 // Forward transform, natural order in, digit-reversed order out (see seq_pos).
 // tw: W_N^t = exp(-2 pi i t / N), t in [0, N); in shared or global memory.
-__device__ __forceinline__ void fft_dif(float2* buf, const FftSeq& sq, const float2* tw, float2* wp) {
+__device__ __forceinline__ void fft_dif(SkewBuf buf, const FftSeq& sq, const float2* tw, float2* wp) {
   int ns = sq.N;
   for (int i = 0; i < sq.n_pass; ++i) {
     one_pass<false>(buf, sq.N, ns, sq.radix[i], tw, wp);
@@ -461,7 +476,7 @@ __device__ __forceinline__ void fft_dif(float2* buf, const FftSeq& sq, const flo
   }
 }
 // Inverse (unnormalised, sign +), digit-reversed order in, natural order out.
-__device__ __forceinline__ void fft_dit_inv(float2* buf, const FftSeq& sq, const float2* tw, float2* wp) {
+__device__ __forceinline__ void fft_dit_inv(SkewBuf buf, const FftSeq& sq, const float2* tw, float2* wp) {
   int ns = 1;
   for (int i = sq.n_pass - 1; i >= 0; --i) {
     ns *= sq.radix[i];
@@ -485,7 +500,7 @@ __device__ __forceinline__ int seq_pos(const FftSeq& sq, int k) {
 // CONJ: conjugate on the way in and out, which turns the forward transform into the
 // unnormalised inverse.
 template <bool CONJ>
-__device__ __forceinline__ void bluestein(float2* buf, const FftPlan& pl, const float2* tables, float2* wp) {
+__device__ __forceinline__ void bluestein(SkewBuf buf, const FftPlan& pl, const float2* tables, float2* wp) {
   const float2* chirp = tables + pl.chirp_offset;
   const float2* filt = tables + pl.filter_offset;
   const int N = pl.N, M = pl.M;
@@ -572,7 +587,8 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     }
     __syncthreads();
     const int n = pl.n, N = pl.N, Kb = n / 2;
-    float2* buf = pl.in_smem ? sbuf : scratch + static_cast<int64_t>(blockIdx.x) * scratch_per_block;
+    const SkewBuf buf = pl.in_smem ? SkewBuf{sbuf, 4, 0}
+                                   : SkewBuf{scratch + static_cast<int64_t>(blockIdx.x) * scratch_per_block, 31, 0};
     // Tables of a direct transform that fit beside the work buffer are staged in shared memory once per plan:
     // the passes read twiddles with data-dependent strides, which from global memory costs a round trip each.
     const float2* tw = tables + pl.seq.tw_offset;
@@ -580,7 +596,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     const int* pos_tab = reinterpret_cast<const int*>(tables + pl.pos_offset);  // where the forward pass left each bin
     const uint16_t* s_pos = nullptr;
     if (pl.tabs_smem) {
-      float2* s_tw = sbuf + N;
+      float2* s_tw = sbuf + sss_padded(N);
       float2* s_post = s_tw + N;
       uint16_t* sp = reinterpret_cast<uint16_t*>(s_post + N / 2 + 1);
       if (loaded_plan != rq.fft_plan) {
@@ -736,7 +752,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     //    also stays in the work buffer, as order-preserving keys, for the selection below.
     const float inv = 1.f / static_cast<float>(N), al = sh.alpha, om = 1.f - sh.alpha;
     const bool sel = budgets != nullptr;
-    uint32_t* keys = reinterpret_cast<uint32_t*>(buf);
+    // packed: the keys of tokens 2m and 2m+1 replace element m; otherwise the key of token m goes to the real part of element m
     if (pl.packed) {
       for (int m = threadIdx.x; m < N; m += kSssThreads) {
         float2 z = buf[m];
@@ -746,22 +762,13 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
           y[2 * m] = y0;
           y[2 * m + 1] = y1;
         }
-        if (sel) *reinterpret_cast<uint2*>(keys + 2 * m) = make_uint2(score_key(y0), score_key(y1));
+        if (sel) buf[m] = make_float2(__uint_as_float(score_key(y0)), __uint_as_float(score_key(y1)));
       }
     } else {
-      // key m lands in the slot of complex element m / 2: read a batch, then write it
-      for (int m0 = 0; m0 < N; m0 += kSssThreads) {
-        const int m = m0 + threadIdx.x;
-        float ym = 0.f;
-        if (m < N) {
-          ym = fmaf(al, buf[m].x * inv, om * x[m]);
-          if (y) y[m] = ym;
-        }
-        if (sel) {
-          __syncthreads();
-          if (m < N) keys[m] = score_key(ym);
-          __syncthreads();
-        }
+      for (int m = threadIdx.x; m < N; m += kSssThreads) {
+        const float ym = fmaf(al, buf[m].x * inv, om * x[m]);
+        if (y) y[m] = ym;
+        if (sel) buf[m].x = __uint_as_float(score_key(ym));
       }
     }
     if (sel) {
@@ -773,7 +780,11 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
         k = k < 0 ? 0 : P;
       }
       __syncthreads();
-      select_topk([&](int j) -> uint32_t { return keys[j]; }, P, W, k, kept_idx + cu_kept[u], &ssm, status);
+      if (pl.packed)
+        select_topk([&](int j) -> uint32_t { const float2 e = buf[j >> 1]; return __float_as_uint((j & 1) ? e.y : e.x); }, P, W, k,
+                    kept_idx + cu_kept[u], &ssm, status);
+      else
+        select_topk([&](int j) -> uint32_t { return __float_as_uint(buf[j].x); }, P, W, k, kept_idx + cu_kept[u], &ssm, status);
     }
   }
 }
@@ -828,7 +839,7 @@ fft_filter_kernel(const FftPlan* __restrict__ plans, float2* __restrict__ tables
   __syncthreads();
   if (!pl.bluestein) return;
   float2* f = tables + pl.filter_offset;
-  fft_dif(f, pl.seq, tables + pl.seq.tw_offset, wp);
+  fft_dif(SkewBuf{f, 31, 0}, pl.seq, tables + pl.seq.tw_offset, wp);
   const float inv = 1.f / static_cast<float>(pl.M);
   for (int j = threadIdx.x; j < pl.M; j += kSssThreads) f[j] = cscale(f[j], inv);
 }
