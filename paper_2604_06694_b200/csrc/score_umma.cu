@@ -9,9 +9,9 @@
 //   sweep 2  D[key][row]  = K Q^T  (keys on the TMEM lanes): every thread owns one key
 //            and adds exp2(z - max - log2 sum) over the rows; no cross-thread reduction.
 // Both sweeps are one persistent kernel (one CTA per SM) with three roles:
-//   warp 8    TMA producer: the Q tile of a head once, K tiles of 128 keys through a ring;
-//   warp 9    MMA issuer: tcgen05.mma, bf16 x bf16 -> fp32 in TMEM, two accumulator buffers;
-//   warps 0-7 two groups of 128 threads that read the accumulators (tcgen05.ld) and do the
+//   warp 16   TMA producer: the Q tile of a head once, K tiles of 128 keys through a ring;
+//   warp 17   MMA issuer: tcgen05.mma, bf16 x bf16 -> fp32 in TMEM, two accumulator buffers;
+//   warps 0-15 four groups of 128 threads that read the accumulators (tcgen05.ld) and do the
 //             softmax arithmetic.
 // Q and K tiles are K-major with the 128-byte swizzle, so the same shared-memory tile is
 // the A operand of one sweep and the B operand of the other.
@@ -26,9 +26,10 @@ namespace akv {
 namespace {
 
 constexpr int kTileKeys = 128;    // keys per K tile (UMMA M in sweep 2, N in sweep 1)
-constexpr int kProducerWarp = 8;
-constexpr int kMmaWarp = 9;
-constexpr int kThreads = 320;
+constexpr int kEpiWarps = 16;      // four epilogue groups of four warps (one warp per TMEM lane quarter)
+constexpr int kProducerWarp = kEpiWarps;
+constexpr int kMmaWarp = kEpiWarps + 1;
+constexpr int kThreads = (kEpiWarps + 2) * 32;
 constexpr int kAccCols = 256;     // TMEM columns of one accumulator buffer
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxStages = 8;
@@ -56,14 +57,14 @@ struct UmmaArgs {
 
 struct Small {
   alignas(16) float negc[2][256];     // sweep 2: -(max + log2 sum) per row, by head parity (read 16 bytes at a time)
-  alignas(16) float2 mrg[2][128];     // sweep 1, one row block: the second group's partial statistics
-  alignas(16) float part[4][128];     // sweep 2: the second group's partial column sums, by tile number mod 4
+  alignas(16) float2 mrg[2][3][128];  // sweep 1: partial statistics of the groups that share a row, by unit parity
+  alignas(16) float part[4][3][128];  // sweep 2: partial column sums of groups 1-3, by tile number mod 4
   alignas(8) uint64_t k_full[kMaxStages];
   uint64_t k_empty[kMaxStages];
   uint64_t q_full, q_empty;
   uint64_t acc_full[2][2], acc_empty[2][2];  // [group][buffer]: each epilogue group has its own accumulator stream
-  uint64_t all_bar;     // both groups (256 arrivals)
-  uint64_t part_full[4];  // sweep 2: the second group's four warps have written part[i]
+  uint64_t all_bar;     // all epilogue threads (512 arrivals)
+  uint64_t part_full[4];  // sweep 2: the twelve warps of groups 1-3 have written part[i]
   uint64_t drain;       // stop path only: the MMAs still in flight
   uint32_t tmem_base;
   int abort;
@@ -311,30 +312,22 @@ __device__ __forceinline__ void colsum_part(const uint32_t (&r)[N], const float*
     a3 = add2(a3, ex2_2(fma2(pack2(r[j + 6], r[j + 7]), sl2, w.y)));
   }
 }
-// One tile of sweep 2: this group's n_u (<= 8) units of 16 TMEM columns starting at taddr; nc points at the
-// first of its query rows. Chunks of 32 columns (and a last one of 16), each loaded under the arithmetic of
-// the one before.
+// One tile of sweep 2: this group's n_u (<= 4) units of 16 TMEM columns starting at taddr; nc points at the
+// first of its query rows. Chunks of 32 columns and a last one of 16; the other warps of the scheduler cover
+// the load latency.
 __device__ __forceinline__ float colsum_tile(uint32_t taddr, int n_u, const float* __restrict__ nc, float sl) {
   const int n32 = n_u >> 1;
   const bool tail = (n_u & 1) != 0;
-  uint32_t ra[32], rb[32], rt[16];
-  if (n32 > 0) tmem_ld32_issue(taddr, ra);
-  else if (tail) tmem_ld16_issue(taddr, rt);
+  uint32_t ra[32], rt[16];
+  if (tail) tmem_ld16_issue(taddr + n32 * 32, rt);
   const f32x2 sl2 = pack2(sl, sl);
   f32x2 a0 = pack2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
 #pragma unroll
-  for (int c = 0; c < 4; c += 2) {
+  for (int c = 0; c < 2; ++c) {
     if (c < n32) {
+      tmem_ld32_issue(taddr + c * 32, ra);
       tmem_wait(ra);
-      if (c + 1 < n32) tmem_ld32_issue(taddr + (c + 1) * 32, rb);
-      else if (tail) tmem_ld16_issue(taddr + n32 * 32, rt);
       colsum_part<32>(ra, nc + c * 32, sl2, a0, a1, a2, a3);
-    }
-    if (c + 1 < n32) {
-      tmem_wait(rb);
-      if (c + 2 < n32) tmem_ld32_issue(taddr + (c + 2) * 32, ra);
-      else if (tail) tmem_ld16_issue(taddr + n32 * 32, rt);
-      colsum_part<32>(rb, nc + (c + 1) * 32, sl2, a0, a1, a2, a3);
     }
   }
   if (tail) {
@@ -376,11 +369,11 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
     for (int g = 0; g < 2; ++g) {
       for (int b = 0; b < 2; ++b) {
         mbar_init(smem_u32(&sm->acc_full[g][b]), 1);
-        mbar_init(smem_u32(&sm->acc_empty[g][b]), 4);
+        mbar_init(smem_u32(&sm->acc_empty[g][b]), 8);  // the two epilogue groups that share the stream
       }
     }
-    mbar_init(smem_u32(&sm->all_bar), 256);
-    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sm->part_full[i]), 4);
+    mbar_init(smem_u32(&sm->all_bar), kEpiWarps * 32);
+    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sm->part_full[i]), 12);
     mbar_init(smem_u32(&sm->drain), 1);
     sm->abort = 0;
     fence_barrier_init();
@@ -517,56 +510,63 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
       }
     }
   } else {
-    // ---- epilogue: two groups of four warps; warp w reads TMEM lanes 32 (w % 4) .. +31 ----
-    // Both groups work on every tile, so that the MMAs of the next tile (other accumulator buffer)
-    // run under the arithmetic of this one:
-    //   sweep 1, two row blocks: group g owns row block g (128 key columns per thread);
-    //   sweep 1, one row block:  group g owns key columns 64 g .. 64 g + 63 of every row;
-    //   sweep 2: group 0 sums over the first half of the query rows, group 1 over the rest and hands
-    //            its partial sums to group 0 through shared memory.
-    const int g = warp >> 2, quarter = warp & 3;
+    // ---- epilogue: four groups of four warps; warp w reads TMEM lanes 32 (w % 4) .. +31 ----
+    // Groups 2 st and 2 st + 1 share accumulator stream st and split its columns in two:
+    //   sweep 1, two row blocks: stream = row block, group = 64 of its 128 key columns;
+    //   sweep 1, one row block:  stream = 64 key columns, group = 32 of them;
+    //   sweep 2: stream = half of the query rows (units of 16), group = half of those; groups 1-3 hand their
+    //            partial column sums to group 0 through shared memory.
+    // Four warps per scheduler keep the special-function unit fed while others load, reduce or wait.
+    const int g4 = warp >> 2, quarter = warp & 3;
+    const int st = g4 >> 1, sub = g4 & 1;
     const int gl = quarter * 32 + lane;  // thread index inside the group = TMEM lane
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     const float sl = sh.scale_log2e;
     int it = 0, prev_u = -1, n_done = 0, heads = 0;
     uint32_t all_phase = 0;
     bool ok = true;
-    const int row = (both ? g * 128 : 0) + gl;   // sweep 1: this thread's query row
-    const int col0 = both ? 0 : g * 64;          // sweep 1: first key column of its share
-    const int win_i = row / G;                   // window row of that query row
+    const int row = (both ? st * 128 : 0) + gl;                // sweep 1: this thread's query row
+    const int col0 = both ? sub * 64 : st * 64 + sub * 32;     // sweep 1: first key column (of the tile) of its share
+    const int tcol1 = both ? sub * 64 : sub * 32;              // ... and that column inside the stream's accumulator
+    const int win_i = row / G;                                 // window row of that query row
     const bool live = row < R;
-    const int u0 = g == 0 ? 0 : u_split, n_u = share_units(g);  // sweep 2: this group's units of 16 query rows
+    // sweep 2: the stream's units of 16 query rows, and this group's part of them
+    const int st_u0 = st == 0 ? 0 : u_split, st_n = share_units(st);
+    const int half_n = (st_n + 1) >> 1;
+    const int my_u0 = sub == 0 ? 0 : half_n, my_n = sub == 0 ? half_n : st_n - half_n;
     ScoreUnit Unext = a.units[unit_begin < unit_end ? unit_begin : 0];
     for (int n = unit_begin; n < unit_end && ok; ++n, ++n_done) {
       const ScoreUnit U = Unext;
       if (n + 1 < unit_end) Unext = a.units[n + 1];
       if (SWEEP == 2 && U.u != prev_u) {
         // Merge the slabs' statistics of this head: negc[row] = -(max + log2 sum); padding rows get -inf.
-        // One row per epilogue thread, eight independent loads in flight at a time.
+        // One row per thread of the first two groups, eight independent loads in flight at a time.
         const int slabs = U.head_slabs;
-        const int rr = g * 128 + gl;
-        float c = -INFINITY;
-        if (rr < R) {
-          const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.n_slab * R + rr;
-          float M = -INFINITY, Zt = 0.f;
-          for (int s0 = 0; s0 < slabs; s0 += 8) {
-            float2 st[8];
+        const int rr = g4 * 128 + gl;
+        if (rr < 256) {
+          float c = -INFINITY;
+          if (rr < R) {
+            const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.n_slab * R + rr;
+            float M = -INFINITY, Zt = 0.f;
+            for (int s0 = 0; s0 < slabs; s0 += 8) {
+              float2 sv[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              st[i] = s0 + i < slabs ? __ldg(hs + static_cast<int64_t>(s0 + i) * R) : make_float2(-INFINITY, 0.f);
+              for (int i = 0; i < 8; ++i)
+                sv[i] = s0 + i < slabs ? __ldg(hs + static_cast<int64_t>(s0 + i) * R) : make_float2(-INFINITY, 0.f);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              if (st[i].y > 0.f) {
-                const float m_new = fmaxf(M, st[i].x);
-                Zt = Zt * exp2f(M - m_new) + st[i].y * exp2f(st[i].x - m_new);  // first: 0 * exp2(-inf) = 0
-                M = m_new;
+              for (int i = 0; i < 8; ++i) {
+                if (sv[i].y > 0.f) {
+                  const float m_new = fmaxf(M, sv[i].x);
+                  Zt = Zt * exp2f(M - m_new) + sv[i].y * exp2f(sv[i].x - m_new);  // first: 0 * exp2(-inf) = 0
+                  M = m_new;
+                }
               }
             }
+            c = -(M + log2f(Zt));
           }
-          c = -(M + log2f(Zt));
+          // two copies by head parity: a slower warp may still read the previous head's
+          sm->negc[heads & 1][rr] = c;
         }
-        // two copies by head parity: a slower warp may still read the previous head's
-        sm->negc[heads & 1][rr] = c;
         ++heads;
         mbar_arrive(smem_u32(&sm->all_bar));
         ok = mbar_wait(smem_u32(&sm->all_bar), all_phase, abort);
@@ -578,34 +578,34 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
       float m_run = -INFINITY, Z = 0.f;  // sweep 1: this thread's row (its share of the columns)
       for (int t = 0; t < U.n_tiles; ++t, ++it) {
         const int b = it & 1;
-        const bool has_share = SWEEP == 1 || n_u > 0;
-        if (has_share) {
-          ok = mbar_wait(smem_u32(&sm->acc_full[g][b]), (it >> 1) & 1, abort);
+        const bool stream_on = SWEEP == 1 || st_n > 0;  // the MMA thread skips a stream without rows
+        if (stream_on) {
+          ok = mbar_wait(smem_u32(&sm->acc_full[st][b]), (it >> 1) & 1, abort);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
         }
         const int kt = U.kt0 + t * kTileKeys;
-        const uint32_t taddr = lane_addr + (2 * b + g) * 128;
+        const uint32_t taddr = lane_addr + (2 * b + st) * 128;
         if (SWEEP == 1) {
           const bool masked = kt + kTileKeys - 1 > U.P;  // the tile reaches into the window: causal mask, end of request
           const int last_col = U.P + win_i - kt;         // last visible key of this row, relative to the tile
-          if (both) stats_tile<4>(taddr, live, masked, col0, last_col, sl, m_run, Z);
-          else stats_tile<2>(taddr, live, masked, col0, last_col, sl, m_run, Z);
+          if (both) stats_tile<2>(taddr + tcol1, live, masked, col0, last_col, sl, m_run, Z);
+          else stats_tile<1>(taddr + tcol1, live, masked, col0, last_col, sl, m_run, Z);
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[g][b]));
+          if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[st][b]));
         } else {
           float acc = 0.f;
-          if (has_share) {
-            acc = colsum_tile(taddr, n_u, sm->negc[(heads - 1) & 1] + u0 * 16, sl);
+          if (stream_on) {
+            if (my_n > 0) acc = colsum_tile(taddr + my_u0 * 16, my_n, sm->negc[(heads - 1) & 1] + (st_u0 + my_u0) * 16, sl);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[g][b]));
+            if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[st][b]));
           }
           const int slot = it & 3;
-          if (g == 1) {
-            sm->part[slot][gl] = acc;
+          if (g4 != 0) {
+            sm->part[slot][g4 - 1][gl] = acc;
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sm->part_full[slot]));
           } else {
@@ -616,33 +616,32 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
             if (!ok) break;
             const int key = kt + gl;
             if (key < U.P)
-              a.scores[U.score_base + key] =
-                  acc + sm->part[slot][gl];
+              a.scores[U.score_base + key] = (acc + sm->part[slot][0][gl]) + (sm->part[slot][1][gl] + sm->part[slot][2][gl]);
           }
         }
       }
       if (!ok) break;
       if (SWEEP == 1) {
+        // the groups that share a row hand their statistics to the first of them
         float2* out = a.stats + (static_cast<int64_t>(U.u) * a.n_slab + U.slab) * R;
-        if (both) {
-          if (live) out[row] = make_float2(m_run * sl, Z);
-        } else {
-          // one row block: the two groups hold the statistics of the two column halves of the same rows
-          float2* mg = sm->mrg[n_done & 1];
-          if (g == 1) mg[gl] = make_float2(m_run, Z);
-          mbar_arrive(smem_u32(&sm->all_bar));
-          ok = mbar_wait(smem_u32(&sm->all_bar), all_phase, abort);
-          all_phase ^= 1;
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          if (g == 0 && live) {
-            const float2 o = mg[gl];
-            const float M = fmaxf(m_run, o.x);
-            float Zt = 0.f;
-            if (Z > 0.f) Zt += Z * ex2((m_run - M) * sl);
-            if (o.y > 0.f) Zt += o.y * ex2((o.x - M) * sl);
-            out[row] = make_float2(M * sl, Zt);
+        float2(*mg)[128] = sm->mrg[n_done & 1];
+        const bool writer = both ? sub == 0 : g4 == 0;
+        if (!writer) mg[both ? st : g4 - 1][gl] = make_float2(m_run, Z);
+        mbar_arrive(smem_u32(&sm->all_bar));
+        ok = mbar_wait(smem_u32(&sm->all_bar), all_phase, abort);
+        all_phase ^= 1;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (writer && live) {
+          const int s0 = both ? st : 0, ns_ = both ? 1 : 3;
+          float M = m_run;
+          for (int o = 0; o < ns_; ++o) M = fmaxf(M, mg[s0 + o][gl].x);
+          float Zt = Z > 0.f ? Z * ex2((m_run - M) * sl) : 0.f;
+          for (int o = 0; o < ns_; ++o) {
+            const float2 pz = mg[s0 + o][gl];
+            if (pz.y > 0.f) Zt += pz.y * ex2((pz.x - M) * sl);
           }
+          out[row] = make_float2(M * sl, Zt);
         }
       }
     }
