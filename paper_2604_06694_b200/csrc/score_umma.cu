@@ -358,7 +358,6 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
   const int S = a.n_stages;
 
   // ---- set-up ----
-  chain_release();
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(smem_u32(&sm->k_full[s]), 1);
@@ -393,7 +392,12 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  chain_wait();  // everything above is local to the CTA; from here on it reads what earlier kernels wrote
+  // Everything above is local to the CTA. Sweep 1 now waits for the kernels before it (they may have written K
+  // and Q) and only then lets sweep 2 be brought in. A CTA of sweep 2 therefore starts on inputs that are
+  // final: its copies and MMAs begin as soon as a CTA of sweep 1 has left the SM, and only its epilogue waits
+  // (below) for sweep 1 to finish, since only the statistics come from there.
+  if (SWEEP == 1) chain_wait();
+  chain_release();
   const uint32_t tmem_base = sm->tmem_base;
 
   const int unit_begin = static_cast<int>(static_cast<int64_t>(blockIdx.x) * a.n_units / gridDim.x);
@@ -534,6 +538,7 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
     const int st_u0 = st == 0 ? 0 : u_split, st_n = share_units(st);
     const int half_n = (st_n + 1) >> 1;
     const int my_u0 = sub == 0 ? 0 : half_n, my_n = sub == 0 ? half_n : st_n - half_n;
+    if (SWEEP == 2) chain_wait();  // the statistics of sweep 1 are complete and visible
     ScoreUnit Unext = a.units[unit_begin < unit_end ? unit_begin : 0];
     for (int n = unit_begin; n < unit_end && ok; ++n, ++n_done) {
       const ScoreUnit U = Unext;

@@ -222,3 +222,34 @@ def test_select_gather_parity(B, dtype, d):
                 rows_v = w.v[l, h, int(w.cu_seqlen[r]):int(w.cu_seqlen[r]) + L][idx]
                 assert np.array_equal(ko[cu[u]:cu[u + 1]], rows_k) and np.array_equal(vo[cu[u]:cu[u + 1]], rows_v)
                 u += 1
+
+
+def test_score_and_gather_token_major_cache(B):
+    """K and V stored [layer][token][head][d] (head stride below token stride): same scores, same kept rows."""
+    w = wl.generate(wl.config(1), layers=2)
+    s = w.spec
+    L, Hkv, d = s.seq_lens[0], s.n_kv_heads, s.head_dim
+    prob = B.Problem.from_workload(w)
+    prob_t = B.Problem.from_workload(w, kv_strides=(L * Hkv * d, Hkv * d, d))
+    q, k, v = to_dev(w, w.q), to_dev(w, w.k), to_dev(w, w.v)
+    k_t, v_t = k.permute(0, 2, 1, 3).contiguous(), v.permute(0, 2, 1, 3).contiguous()
+    out = []
+    for pb, kk, vv in ((prob, k, v), (prob_t, k_t, v_t)):
+        ctx = B.Context(pb)
+        scores = torch.empty(B.audiokv_scores_len(pb), device="cuda")
+        B.audiokv_score(ctx, pb, q, kk, scores)
+        TH, rows = pb.total_heads, int(w.total_budget.sum())
+        ko = torch.zeros((rows, d), dtype=torch.bfloat16, device="cuda")
+        vo = torch.zeros_like(ko)
+        kept = torch.zeros(rows, dtype=torch.int32, device="cuda")
+        bud = torch.zeros(TH, dtype=torch.int32, device="cuda")
+        cu = torch.zeros(TH + 1, dtype=torch.int32, device="cuda")
+        B.audiokv_evict(ctx, pb, q, kk, vv, torch.from_numpy(w.head_scores).cuda(), [int(x) for x in w.total_budget],
+                        ko, vo, kept, bud, cu)
+        torch.cuda.synchronize()
+        assert ctx.last_device_status() == 0
+        out.append((scores.cpu(), ko.cpu().view(torch.int16), vo.cpu().view(torch.int16), kept.cpu(), bud.cpu()))
+    for a, b in zip(*out):
+        assert torch.equal(a, b)
+    o, _ = oracle_scores(w, 0)
+    assert rel_err(out[1][0].numpy().reshape(o.shape)[1, 2], o[1, 2]) <= REL_TOL
