@@ -468,7 +468,7 @@ __device__ __forceinline__ void one_pass(SkewBuf buf, int N, int ns, int r, cons
 
 // Forward transform, natural order in, digit-reversed order out (see seq_pos).
 // tw: W_N^t = exp(-2 pi i t / N), t in [0, N); in shared or global memory.
-__device__ __forceinline__ void fft_dif(SkewBuf buf, const FftSeq& sq, const float2* tw, float2* wp) {
+__device__ __noinline__ void fft_dif(SkewBuf buf, const FftSeq& sq, const float2* tw, float2* wp) {
   int ns = sq.N;
   for (int i = 0; i < sq.n_pass; ++i) {
     one_pass<false>(buf, sq.N, ns, sq.radix[i], tw, wp);
@@ -476,7 +476,7 @@ __device__ __forceinline__ void fft_dif(SkewBuf buf, const FftSeq& sq, const flo
   }
 }
 // Inverse (unnormalised, sign +), digit-reversed order in, natural order out.
-__device__ __forceinline__ void fft_dit_inv(SkewBuf buf, const FftSeq& sq, const float2* tw, float2* wp) {
+__device__ __noinline__ void fft_dit_inv(SkewBuf buf, const FftSeq& sq, const float2* tw, float2* wp) {
   int ns = 1;
   for (int i = sq.n_pass - 1; i >= 0; --i) {
     ns *= sq.radix[i];
