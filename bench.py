@@ -154,7 +154,7 @@ def run_cuda(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    spec = wl.config(1)
+    spec = wl.config(args.config)
     w = wl.generate(spec, seed=rank, layers=args.layers)   # every rank evicts its own request: no exchange step
     spec = w.spec
     L = spec.seq_lens[0]
@@ -369,6 +369,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the CPU-oracle baseline (profiling runs)")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--config", type=int, default=1,
+                    help="workload index (1 = the benchmark workload; others are for exploration, not bench lines)")
     ap.add_argument("--layers", type=int, default=None,
                     help="truncate the stack to its first LAYERS layers (small cases for profiler captures; not a bench line)")
     args = ap.parse_args()

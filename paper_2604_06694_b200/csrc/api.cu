@@ -22,7 +22,7 @@ constexpr int kMaxHeadsPerReq = 2048;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {  // byte offsets inside the workspace
-  size_t status, reqs, plans, tables, units, stats, fft_scratch, scores, kstar, end;
+  size_t status, reqs, plans, tables, units, order, stats, fft_scratch, scores, kstar, end;
 };
 
 struct Plan {
@@ -35,6 +35,7 @@ struct Plan {
   std::vector<FftPlan> fft;
   std::vector<ScoreUnit> units;   // sweep 1 (all keys, ascending) then sweep 2 (prefix keys, descending)
   int n_units1 = 0, n_units2 = 0;
+  std::vector<int32_t> sss_order;  // heads in the order the smoothing blocks take them (see build_plan); -1 = none
   int64_t table_len = 0;        // float2 elements
   int64_t scores_len = 0;
   int max_L = 0, max_P = 0;
@@ -158,8 +159,17 @@ void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
     fp->M = 0;
   } else {
     fp->bluestein = 1;
-    int M = 1;
-    while (M < 2 * N - 1) M *= 2;
+    // convolution length: the smallest 2^a 3^b 5^c 7^d (a >= 2) that holds 2N - 1 points; close to 2N - 1
+    // instead of up to twice that for a power of two, which also keeps more transforms in shared memory
+    int M = 0;
+    for (int64_t p7 = 1; p7 < 4LL * N; p7 *= 7)
+      for (int64_t p5 = p7; p5 < 4LL * N; p5 *= 5)
+        for (int64_t p3 = p5; p3 < 4LL * N; p3 *= 3)
+          for (int64_t p2 = p3 * 4; p2 < 8LL * N; p2 *= 2)
+            if (p2 >= 2LL * N - 1) {
+              if (M == 0 || p2 < M) M = static_cast<int>(p2);
+              break;
+            }
     fp->M = M;
     factor_len(M, &fp->seq);
     buf_len = M;
@@ -281,6 +291,28 @@ int build_plan(const audiokv_params* p, Plan* pl) {
     }
   }
   pl->sss_grid = sh.total_heads < 148 ? sh.total_heads : 148;
+  {
+    // Block b of the smoothing kernel takes entries b, b + grid, b + 2 grid, ... of this list. Heads are sorted by an
+    // estimate of their transform's cost and dealt out in a snake (left to right, then right to left), so that
+    // a ragged batch with a few expensive lengths (chirp-z in global scratch) does not leave them to one block.
+    auto cost = [&](int u) -> double {
+      const FftPlan& fp = pl->fft[pl->reqs[u / sh.heads_per_req].fft_plan];
+      const double len = fp.bluestein ? fp.M : fp.N;
+      double c = len * (fp.bluestein ? 4.0 : 1.0) * (fp.in_smem ? 1.0 : 6.0);
+      for (int i = 0; i < fp.seq.n_pass; ++i)
+        if (fp.seq.radix[i] > 19) c += static_cast<double>(fp.seq.N) * fp.seq.radix[i] / 8.0;  // O(p N) prime pass
+      return c;
+    };
+    std::vector<int32_t> by_cost(sh.total_heads);
+    for (int u = 0; u < sh.total_heads; ++u) by_cost[u] = u;
+    std::stable_sort(by_cost.begin(), by_cost.end(), [&](int a, int b) { return cost(a) > cost(b); });
+    const int g = pl->sss_grid, tiers = (sh.total_heads + g - 1) / g;
+    pl->sss_order.assign(static_cast<size_t>(tiers) * g, -1);
+    for (int i = 0; i < sh.total_heads; ++i) {
+      const int tier = i / g, j = i - tier * g;
+      pl->sss_order[static_cast<size_t>(tier) * g + ((tier & 1) ? g - 1 - j : j)] = by_cost[i];
+    }
+  }
   int smem_c = 2;
   pl->scratch_per_block = 0;
   for (const FftPlan& fp : pl->fft) {
@@ -300,6 +332,7 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   L.plans = off;       off = align_up(off + sizeof(FftPlan) * kMaxPlans);
   L.tables = off;      off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->table_len));
   L.units = off;       off = align_up(off + sizeof(ScoreUnit) * pl->units.size());
+  L.order = off;       off = align_up(off + sizeof(int32_t) * pl->sss_order.size());
   L.stats = off;       off = align_up(off + sizeof(float2) * static_cast<size_t>(sh.total_heads) * pl->n_slab * sh.window * sh.group);
   L.fft_scratch = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->scratch_per_block) * pl->sss_grid);
   L.scores = off;      off = align_up(off + sizeof(float) * static_cast<size_t>(pl->scores_len));
@@ -337,6 +370,9 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess)
       return cuda_fail(ctx, e);
     if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.units, pl.units.data(), sizeof(ScoreUnit) * pl.units.size(),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+      return cuda_fail(ctx, e);
+    if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.order, pl.sss_order.data(), sizeof(int32_t) * pl.sss_order.size(),
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess)
       return cuda_fail(ctx, e);
     Launch ln{stream, &ctx->launches, &ctx->prof};
@@ -388,7 +424,8 @@ int do_smooth(audiokv_ctx* ctx, const float* scores, float* smoothed, int32_t* k
   cudaError_t e = launch_sss(pl.sh, d_reqs(ctx), reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans),
                              reinterpret_cast<const float2*>(ctx->ws + pl.lay.tables), scores, smoothed, kstar,
                              reinterpret_cast<float2*>(ctx->ws + pl.lay.fft_scratch), pl.scratch_per_block,
-                             pl.sss_grid, pl.sss_smem, budgets, cu_kept, kept_idx, d_status(ctx), ln);
+                             pl.sss_grid, pl.sss_smem, reinterpret_cast<const int32_t*>(ctx->ws + pl.lay.order),
+                             static_cast<int>(pl.sss_order.size()), budgets, cu_kept, kept_idx, d_status(ctx), ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 

@@ -145,12 +145,12 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
 
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);
-// smoothed may be null when budgets, cu_kept and kept_idx are given: the kernel then goes on to the
+// order: n_order head indices (or -1); block b takes entries b, b + grid, ... . smoothed may be null when budgets, cu_kept and kept_idx are given: the kernel then goes on to the
 // top-k selection of each head from the smoothed scores it holds on chip (step 4a of the pass).
 cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_plans, const float2* d_tables,
                        const float* scores, float* smoothed, int32_t* kstar, float2* scratch,
-                       int64_t scratch_per_block, int grid, size_t smem_bytes, const int32_t* budgets,
-                       const int32_t* cu_kept, int32_t* kept_idx, int* status, Launch ln);
+                       int64_t scratch_per_block, int grid, size_t smem_bytes, const int32_t* order, int n_order,
+                       const int32_t* budgets, const int32_t* cu_kept, int32_t* kept_idx, int* status, Launch ln);
 
 // allocate.cu (h_total_budget: host array [n_req])
 cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float* head_scores,
