@@ -145,6 +145,26 @@ def kernel_roofline(name, ms, spec, w, peaks, sm_max_mhz):
             "traffic": NCU_TRAFFIC_BYTES.get(name)}
 
 
+def rank_seed(rank: int) -> int:
+    """Every rank evicts a request of its own (weak scaling, no exchange step): rank r draws the workload with seed r."""
+    return rank
+
+
+def max_over_ranks(x: float, world: int, device="cpu") -> float:
+    """The slowest rank's time: all-reduce MAX over the default process group (identity when there is one rank)."""
+    if world <= 1:
+        return float(x)
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_us_per_layer(ms_step_max: float, n_layers: int, world: int) -> float:
+    """All ranks run n_layers layers each in ms_step_max: microseconds per layer of the whole job."""
+    return ms_step_max * 1e3 / (n_layers * world)
+
+
 def run_cuda(args):
     from paper_2604_06694_b200 import binding as B
     rank = int(os.environ.get("RANK", "0"))
@@ -155,7 +175,7 @@ def run_cuda(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     spec = wl.config(args.config)
-    w = wl.generate(spec, seed=rank, layers=args.layers)   # every rank evicts its own request: no exchange step
+    w = wl.generate(spec, seed=rank_seed(rank), layers=args.layers)   # every rank evicts its own request: no exchange step
     spec = w.spec
     L = spec.seq_lens[0]
     prob = B.Problem.from_workload(w)
@@ -197,10 +217,7 @@ def run_cuda(args):
     barrier()
     launches = ctx.launch_count() - n0
     ms_total = e0.elapsed_time(e1)
-    t = torch.tensor([ms_total], device="cuda")
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
     clocks = None
     if sampler:
         # nvidia-smi delivers a sample every 200 ms: when the timed region was shorter than about a second the
@@ -261,11 +278,7 @@ def run_e2e(B, ctx, prob, w, spec, tb, rows, TH, es, barrier, world, args):
     for _ in range(n_e2e):
         step_host()
     barrier()
-    e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
-    t = torch.tensor([e2e_ms], device="cuda")
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / n_e2e, world, "cuda")
     h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv, hS))
     d2h = sum(x.numel() * x.element_size() for x in (hko, hvo, hkept, hb, hcu))
     return e2e_ms, h2d, d2h
@@ -274,7 +287,7 @@ def run_e2e(B, ctx, prob, w, spec, tb, rows, TH, es, barrier, world, args):
 def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_ms, h2d, d2h):
     NL = spec.n_layers
     peaks, peak_kind = measured_peaks()
-    us_layer = ms_step * 1e3 / (NL * world)
+    us_layer = whole_job_us_per_layer(ms_step, NL, world)
     cbytes = contract_bytes_per_layer(spec, L)
     hbm_gbs = cbytes * NL * world / (ms_step * 1e-3) / 1e9
     kern = {n: statistics.mean(v) for n, v in per_kernel.items()}
@@ -346,13 +359,17 @@ def run_reference(args):
     w = wl.generate(spec, seed=0, layers=sample_layers)
     for _ in range(max(args.warmup, 1)):
         oracle_pass(w, spec, sample_layers)
-    ts = [oracle_pass(w, spec, sample_layers) for _ in range(args.steps)]
+    ts, t_begin = [], time.perf_counter()
+    for _ in range(args.steps):
+        ts.append(oracle_pass(w, spec, sample_layers))
+        if time.perf_counter() - t_begin > 120.0:     # a large --steps (the CUDA arm's default) stops after two minutes
+            break
     sec = sum(ts) / len(ts)
     us_layer = sec * 1e6 / sample_layers
     cores = os.cpu_count() or 1
     sample = f"each step = the first {sample_layers} of {spec.n_layers} layers (all four steps of the pass)"
     line = {"impl": "reference", "metric": METRIC, "value": round(us_layer, 1), "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": round(sec * 1e3, 3),
+            "steps": len(ts), "warmup": max(args.warmup, 1), "ms_per_step": round(sec * 1e3, 3),
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": spec.name, "layers": spec.n_layers, "L": spec.seq_lens[0], "window": spec.window,
                        "keep": spec.keep, "sample": sample},
