@@ -16,8 +16,10 @@ __device__ __forceinline__ uint32_t score_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+constexpr int kSelBins = 2048;  // 11-bit digits: three passes (11 + 11 + 10 bits) cover the 32-bit key
+
 struct SelectSmem {
-  int hist[256];
+  int hist[kSelBins];
   int wsum[32];
   uint32_t prefix;
   int want;
@@ -46,8 +48,8 @@ __device__ __forceinline__ int block_excl_scan_int(int v, int* wsum, int* total)
 
 // Writes to `out` the k prefix tokens (of P) with the largest keys, ties to the lower index, in
 // ascending token order, then the W window tokens P .. P+W-1. key_at(j) gives the key of token j.
-// Every thread of the block calls this with the same arguments. Four 8-bit radix passes find the
-// k-th largest key; the bin that holds it is located by a block-wide scan over the 256 counts.
+// Every thread of the block calls this with the same arguments. Three radix passes (11, 11 and 10 bits) find
+// the k-th largest key; the bin that holds it is located by a block-wide scan over the counts.
 template <typename KeyAt>
 __device__ __forceinline__ void select_topk(KeyAt key_at, int P, int W, int k, int32_t* __restrict__ out,
                                             SelectSmem* sm, int* __restrict__ status) {
@@ -59,26 +61,31 @@ __device__ __forceinline__ void select_topk(KeyAt key_at, int P, int W, int k, i
       sm->prefix = 0u;
       sm->want = k;
     }
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      for (int b = threadIdx.x; b < 256; b += kSelThreads) sm->hist[b] = 0;
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 21 : pass == 1 ? 10 : 0;
+      const int bits = pass == 2 ? 10 : 11;
+      const uint32_t dmask = (1u << bits) - 1u;
+      for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) sm->hist[b] = 0;
       __syncthreads();
       const uint32_t prefix = sm->prefix;
       const int want = sm->want;
-      const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + bits));
       for (int j = threadIdx.x; j < P; j += kSelThreads) {
         const uint32_t key = key_at(j);
-        if ((key & pmask) == prefix) atomicAdd(&sm->hist[(key >> shift) & 255u], 1);
+        if ((key & pmask) == prefix) atomicAdd(&sm->hist[(key >> shift) & dmask], 1);
       }
       __syncthreads();
-      // thread t < 256 owns bin 255 - t: `above` counts the keys in higher bins
-      const int bin = 255 - static_cast<int>(threadIdx.x);
-      const int cnt = threadIdx.x < 256 ? sm->hist[bin] : 0;
+      // thread t owns bins 2047 - 2t and 2046 - 2t (descending): `above` counts the keys in higher bins
+      const int b_hi = kSelBins - 1 - 2 * static_cast<int>(threadIdx.x), b_lo = b_hi - 1;
+      const int c_hi = sm->hist[b_hi], c_lo = sm->hist[b_lo];
       int tot;
-      const int above = block_excl_scan_int(cnt, sm->wsum, &tot);
-      if (threadIdx.x < 256 && above < want && want <= above + cnt) {
-        sm->prefix = prefix | (static_cast<uint32_t>(bin) << shift);
+      const int above = block_excl_scan_int(c_hi + c_lo, sm->wsum, &tot);
+      if (above < want && want <= above + c_hi) {
+        sm->prefix = prefix | (static_cast<uint32_t>(b_hi) << shift);
         sm->want = want - above;
+      } else if (above + c_hi < want && want <= above + c_hi + c_lo) {
+        sm->prefix = prefix | (static_cast<uint32_t>(b_lo) << shift);
+        sm->want = want - above - c_hi;
       }
       __syncthreads();
     }
