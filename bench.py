@@ -36,9 +36,11 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
 
 
-# DRAM bytes per launch (read + write) of each kernel at this workload, from the ncu captures summarised
-# under profiles/ (see the file named there); None where no capture has been taken yet.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on the benchmark workload, from
+# the ncu capture summarised in profiles/score_umma_c2.md and profiles/sss_select_gather_c2.md (ncu flushes the
+# caches before each kernel, so the column-sum sweep's K re-read counts in full). Only valid for config 1, all layers.
+NCU_TRAFFIC_BYTES = {"score_umma_stats": 254889728, "score_umma_colsum": 263040512, "sss_select": 3843072,
+                     "gather": 330574336}
 
 
 class ClockSampler:
@@ -131,6 +133,7 @@ def kernel_roofline(name, ms, spec, w, peaks, sm_max_mhz):
     """Roofline entry of one kernel: the scoring sweeps are bound by the special-function units (16 exp2 per clock
     and SM, 148 SMs, at the maximum SM clock), everything else by HBM (measured copy bandwidth)."""
     nbytes = kernel_algorithmic_bytes(name, spec, w)
+    traffic = NCU_TRAFFIC_BYTES.get(name) if (spec.name.startswith("c2_") and spec.n_layers == 28) else None
     hbm = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
     if name.startswith("score_umma"):
         peak = 148 * 16 * (sm_max_mhz or 1965.0) * 1e6 / 1e9      # Gexp2/s
@@ -139,10 +142,10 @@ def kernel_roofline(name, ms, spec, w, peaks, sm_max_mhz):
                 "frac": round(ach / peak, 4), "peak_kind": "148 SMs x 16 exp2/clk x max SM clock",
                 "algorithmic_exp2": kernel_algorithmic_exps(name, spec, w), "algorithmic_bytes": nbytes,
                 "hbm_gbs": round(hbm, 1), "hbm_frac_of_measured": round(hbm / peaks["hbm_gbs"], 4),
-                "traffic": NCU_TRAFFIC_BYTES.get(name)}
+                "traffic": traffic}
     return {"kernel": name, "bound": "hbm", "achieved": round(hbm, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": round(hbm / peaks["hbm_gbs"], 4), "algorithmic_bytes": nbytes,
-            "traffic": NCU_TRAFFIC_BYTES.get(name)}
+            "traffic": traffic}
 
 
 def rank_seed(rank: int) -> int:
