@@ -365,13 +365,14 @@ __device__ __noinline__ void pass_odd(SkewBuf buf, int N, int ns, const float2* 
 // The same pass for an odd prime radix p, 23 <= p <= 127 (11 to 19 have pass_odd). A length-p DFT is O(p^2); pairing
 // inputs s and p - s (P = a_s + a_{p-s}, Q = a_s - a_{p-s}) gives outputs c and p - c from the
 // same real-by-complex products: X_c = A -/+ iB, A = a_0 + sum_s P_s cos(2 pi s c / p),
-// B = sum_s Q_s sin(2 pi s c / p); c = 0 is the plain sum. One task = one butterfly and one c in
-// [0, (p-1)/2]; consecutive threads take consecutive butterflies of the same c, so the data
-// reads are contiguous and the cos/sin reads are broadcasts. A thread keeps the results of its
-// (at most kPrimeTasks) tasks in registers until every task of the round has read its inputs.
+// B = sum_s Q_s sin(2 pi s c / p); c = 0 is the plain sum. One task = one butterfly and kPrimeOut
+// consecutive c in [0, (p-1)/2]; consecutive threads take consecutive butterflies of the same c, so
+// the data reads are contiguous and the cos/sin reads are broadcasts. A thread keeps the results of
+// its (at most kPrimeTasks) tasks in registers until every task of the round has read its inputs.
 // The pass twiddles are applied in a sweep of their own (inverse: before, forward: with the
 // write-back).
-constexpr int kPrimeTasks = 6;
+constexpr int kPrimeTasks = 2;  // tasks per thread and round
+constexpr int kPrimeOut = 4;    // consecutive c per task: the folded inputs P_s, Q_s are formed once for all of them
 
 template <bool INV>
 __device__ __noinline__ void pass_prime(SkewBuf buf, int N, int ns, int p, const float2* tw,
@@ -390,36 +391,43 @@ __device__ __noinline__ void pass_prime(SkewBuf buf, int N, int ns, int p, const
     }
   }
   __syncthreads();
-  const int per_round = max(1, (kPrimeTasks * kSssThreads) / (H + 1));  // butterflies per round
+  const int n_chunks = (H + kPrimeOut) / kPrimeOut;  // chunks of c over [0, H]
+  const int per_round = max(1, (kPrimeTasks * kSssThreads) / n_chunks);  // butterflies per round
   for (int b0 = 0; b0 < nb; b0 += per_round) {
     const int nbr = min(per_round, nb - b0);
-    const int n_task = nbr * (H + 1);
-    float2 A[kPrimeTasks], B[kPrimeTasks];
+    const int n_task = nbr * n_chunks;
+    float2 A[kPrimeTasks][kPrimeOut], B[kPrimeTasks][kPrimeOut];
 #pragma unroll
     for (int i = 0; i < kPrimeTasks; ++i) {
       const int q = threadIdx.x + kSssThreads * i;
-      A[i] = make_float2(0.f, 0.f);
-      B[i] = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int o = 0; o < kPrimeOut; ++o) A[i][o] = B[i][o] = make_float2(0.f, 0.f);
       if (q < n_task) {
-        const int c = q / nbr;
-        const int t = b0 + q - c * nbr;
+        const int chunk = q / nbr;
+        const int t = b0 + q - chunk * nbr;
         const int b = t / m, j = t - b * m;
         const SkewBuf base = buf + (b * ns + j);
-        float2 a = base[0], bb = make_float2(0.f, 0.f);
-        int idx = c;
+        const float2 a0 = base[0];
+        int idx[kPrimeOut];
+#pragma unroll
+        for (int o = 0; o < kPrimeOut; ++o) {
+          A[i][o] = a0;
+          idx[o] = chunk * kPrimeOut + o;  // (s c) mod p at s = 1; c <= H + kPrimeOut - 1 < p
+        }
         for (int sI = 1; sI <= H; ++sI) {
           const float2 x = base[sI * m], y = base[(p - sI) * m];
           const float2 P = cadd(x, y), Q = csub(x, y);
-          const float2 w = cs[idx];
-          a.x = fmaf(P.x, w.x, a.x);
-          a.y = fmaf(P.y, w.x, a.y);
-          bb.x = fmaf(Q.x, w.y, bb.x);
-          bb.y = fmaf(Q.y, w.y, bb.y);
-          idx += c;
-          if (idx >= p) idx -= p;
+#pragma unroll
+          for (int o = 0; o < kPrimeOut; ++o) {
+            const float2 w = cs[idx[o]];
+            A[i][o].x = fmaf(P.x, w.x, A[i][o].x);
+            A[i][o].y = fmaf(P.y, w.x, A[i][o].y);
+            B[i][o].x = fmaf(Q.x, w.y, B[i][o].x);
+            B[i][o].y = fmaf(Q.y, w.y, B[i][o].y);
+            idx[o] += chunk * kPrimeOut + o;
+            if (idx[o] >= p) idx[o] -= p;
+          }
         }
-        A[i] = a;
-        B[i] = bb;
       }
     }
     __syncthreads();
@@ -427,22 +435,26 @@ __device__ __noinline__ void pass_prime(SkewBuf buf, int N, int ns, int p, const
     for (int i = 0; i < kPrimeTasks; ++i) {
       const int q = threadIdx.x + kSssThreads * i;
       if (q < n_task) {
-        const int c = q / nbr;
-        const int t = b0 + q - c * nbr;
+        const int chunk = q / nbr;
+        const int t = b0 + q - chunk * nbr;
         const int b = t / m, j = t - b * m;
         const SkewBuf base = buf + (b * ns + j);
-        if (c == 0) {
-          base[0] = A[i];
-        } else {
-          const float2 iB = mul_i(B[i]);
-          float2 xc = INV ? cadd(A[i], iB) : csub(A[i], iB);
-          float2 xq = INV ? csub(A[i], iB) : cadd(A[i], iB);
-          if (!INV && m > 1) {
-            xc = cmul(xc, tw[j * c * step]);
-            xq = cmul(xq, tw[j * (p - c) * step]);
+#pragma unroll
+        for (int o = 0; o < kPrimeOut; ++o) {
+          const int c = chunk * kPrimeOut + o;
+          if (c == 0) {
+            base[0] = A[i][o];
+          } else if (c <= H) {
+            const float2 iB = mul_i(B[i][o]);
+            float2 xc = INV ? cadd(A[i][o], iB) : csub(A[i][o], iB);
+            float2 xq = INV ? csub(A[i][o], iB) : cadd(A[i][o], iB);
+            if (!INV && m > 1) {
+              xc = cmul(xc, tw[j * c * step]);
+              xq = cmul(xq, tw[j * (p - c) * step]);
+            }
+            base[c * m] = xc;
+            base[(p - c) * m] = xq;
           }
-          base[c * m] = xc;
-          base[(p - c) * m] = xq;
         }
       }
     }
