@@ -175,6 +175,12 @@ void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
     buf_len = M;
   }
   fp->in_smem = sss_padded(buf_len) <= kSssSmemComplex ? 1 : 0;
+  fp->g_pass = 0;
+  if (!fp->in_smem) {
+    // leading passes on the global buffer until a block and its twiddles (padded(len) + len slots) fit on chip
+    int len = buf_len;
+    while (fp->g_pass < fp->seq.n_pass && sss_padded(len) + len > kSssSmemComplex) len /= fp->seq.radix[fp->g_pass++];
+  }
   // a direct transform also keeps its tables on chip when buffer + W_N + post-twiddles + uint16 positions fit
   fp->tabs_smem = (!fp->bluestein && fp->in_smem && N < 65536 && sss_smem_complex(*fp, true) <= kSssSmemComplex) ? 1 : 0;
   fp->seq.tw_offset = *table_len;
@@ -321,7 +327,13 @@ int build_plan(const audiokv_params* p, Plan* pl) {
       const int need = sss_smem_complex(fp, fp.tabs_smem != 0);
       smem_c = need > smem_c ? need : smem_c;
     }
-    else pl->scratch_per_block = len > pl->scratch_per_block ? len : pl->scratch_per_block;
+    else {
+      pl->scratch_per_block = len > pl->scratch_per_block ? len : pl->scratch_per_block;
+      int blk = len;
+      for (int i = 0; i < fp.g_pass; ++i) blk /= fp.seq.radix[i];
+      const int need = sss_padded(blk) + blk;
+      smem_c = need > smem_c ? need : smem_c;
+    }
   }
   pl->sss_smem = static_cast<size_t>(smem_c) * sizeof(float2);
 

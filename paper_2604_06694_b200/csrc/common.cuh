@@ -59,7 +59,7 @@ struct FftPlan {
   int32_t M;         // convolution length (bluestein only)
   int32_t in_smem;   // 1: the work buffer fits in shared memory
   int32_t tabs_smem; // 1: twiddles, post-twiddles and bin positions are staged in shared memory after the buffer
-  int32_t pad_;
+  int32_t g_pass;    // not in_smem: leading passes that run on the global buffer; the rest runs block by block in shared memory
   FftSeq seq;        // passes for length N (direct) or M (bluestein)
   int64_t chirp_offset;   // float2 index of c_j = exp(-i pi j^2 / N), j in [0, N)      (bluestein)
   int64_t filter_offset;  // float2 index of FFT_M of the wrapped conjugate chirp / M    (bluestein)

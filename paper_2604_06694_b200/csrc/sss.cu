@@ -495,6 +495,63 @@ __device__ __noinline__ void fft_dit_inv(SkewBuf buf, const FftSeq& sq, const fl
     one_pass<true>(buf, sq.N, ns, sq.radix[i], tw, wp);
   }
 }
+// The same two transforms for a buffer in global memory that is too long for shared memory. The first g passes
+// of the forward transform couple elements that lie far apart and run on the global buffer; after them the
+// transform falls apart into F = r_1 ... r_g contiguous blocks of length len = N / F, each of which is brought
+// into shared memory (with its own twiddles W_len^t = W_N^{t F}) for the remaining passes. The inverse runs the
+// steps backwards. Every element then makes g + 1 round trips to global memory instead of one per pass.
+__device__ __noinline__ void fft_dif_big(SkewBuf gbuf, const FftSeq& sq, int g, const float2* tw, float2* wp,
+                                         float2* sbuf) {
+  int ns = sq.N;
+  for (int i = 0; i < g; ++i) {
+    one_pass<false>(gbuf, sq.N, ns, sq.radix[i], tw, wp);
+    ns /= sq.radix[i];
+  }
+  const int len = ns, F = sq.N / len;
+  const SkewBuf sb{sbuf, 4, 0};
+  float2* s_tw = sbuf + sss_padded(len);
+  __syncthreads();
+  for (int t = threadIdx.x; t < len; t += kSssThreads) s_tw[t] = tw[t * F];
+  for (int blk = 0; blk < F; ++blk) {
+    __syncthreads();
+    for (int t = threadIdx.x; t < len; t += kSssThreads) sb[t] = gbuf[blk * len + t];
+    __syncthreads();
+    int ns2 = len;
+    for (int i = g; i < sq.n_pass; ++i) {
+      one_pass<false>(sb, len, ns2, sq.radix[i], s_tw, wp);
+      ns2 /= sq.radix[i];
+    }
+    for (int t = threadIdx.x; t < len; t += kSssThreads) gbuf[blk * len + t] = sb[t];
+  }
+  __syncthreads();
+}
+__device__ __noinline__ void fft_dit_inv_big(SkewBuf gbuf, const FftSeq& sq, int g, const float2* tw, float2* wp,
+                                             float2* sbuf) {
+  int len = sq.N;
+  for (int i = 0; i < g; ++i) len /= sq.radix[i];
+  const int F = sq.N / len;
+  const SkewBuf sb{sbuf, 4, 0};
+  float2* s_tw = sbuf + sss_padded(len);
+  __syncthreads();
+  for (int t = threadIdx.x; t < len; t += kSssThreads) s_tw[t] = tw[t * F];
+  for (int blk = 0; blk < F; ++blk) {
+    __syncthreads();
+    for (int t = threadIdx.x; t < len; t += kSssThreads) sb[t] = gbuf[blk * len + t];
+    __syncthreads();
+    int ns2 = 1;
+    for (int i = sq.n_pass - 1; i >= g; --i) {
+      ns2 *= sq.radix[i];
+      one_pass<true>(sb, len, ns2, sq.radix[i], s_tw, wp);
+    }
+    for (int t = threadIdx.x; t < len; t += kSssThreads) gbuf[blk * len + t] = sb[t];
+  }
+  __syncthreads();
+  int ns = len;
+  for (int i = g - 1; i >= 0; --i) {
+    ns *= sq.radix[i];
+    one_pass<true>(gbuf, sq.N, ns, sq.radix[i], tw, wp);
+  }
+}
 // Where the forward transform leaves bin k.
 __device__ __forceinline__ int seq_pos(const FftSeq& sq, int k) {
   int len = sq.N, p = 0;
@@ -512,7 +569,7 @@ __device__ __forceinline__ int seq_pos(const FftSeq& sq, int k) {
 // CONJ: conjugate on the way in and out, which turns the forward transform into the
 // unnormalised inverse.
 template <bool CONJ>
-__device__ __forceinline__ void bluestein(SkewBuf buf, const FftPlan& pl, const float2* tables, float2* wp) {
+__device__ __forceinline__ void bluestein(SkewBuf buf, const FftPlan& pl, const float2* tables, float2* wp, float2* sbuf) {
   const float2* chirp = tables + pl.chirp_offset;
   const float2* filt = tables + pl.filter_offset;
   const int N = pl.N, M = pl.M;
@@ -526,10 +583,12 @@ __device__ __forceinline__ void bluestein(SkewBuf buf, const FftPlan& pl, const 
     buf[j] = v;
   }
   __syncthreads();
-  fft_dif(buf, pl.seq, tables + pl.seq.tw_offset, wp);
+  if (pl.in_smem) fft_dif(buf, pl.seq, tables + pl.seq.tw_offset, wp);
+  else fft_dif_big(buf, pl.seq, pl.g_pass, tables + pl.seq.tw_offset, wp, sbuf);
   for (int j = threadIdx.x; j < M; j += kSssThreads) buf[j] = cmul(buf[j], __ldg(filt + j));
   __syncthreads();
-  fft_dit_inv(buf, pl.seq, tables + pl.seq.tw_offset, wp);
+  if (pl.in_smem) fft_dit_inv(buf, pl.seq, tables + pl.seq.tw_offset, wp);
+  else fft_dit_inv_big(buf, pl.seq, pl.g_pass, tables + pl.seq.tw_offset, wp, sbuf);
   for (int j = threadIdx.x; j < N; j += kSssThreads) {
     float2 v = cmul(buf[j], __ldg(chirp + j));
     buf[j] = CONJ ? cconj(v) : v;
@@ -625,8 +684,8 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
       tw = s_tw;
       post = s_post;
       s_pos = sp;
-    } else if (pl.in_smem) {
-      loaded_plan = -1;  // this head's work buffer may run over the staged tables
+    } else {
+      loaded_plan = -1;  // this head's work buffer (or its blocks) may run over the staged tables
     }
     const float* x = scores + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P;
     float* y = smoothed ? smoothed + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P : nullptr;
@@ -641,9 +700,11 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
 
     // 2. forward complex transform; bin k then sits at POS(k)
     if (pl.bluestein)
-      bluestein<false>(buf, pl, tables, wp);
-    else
+      bluestein<false>(buf, pl, tables, wp, sbuf);
+    else if (pl.in_smem)
       fft_dif(buf, pl.seq, tw, wp);
+    else
+      fft_dif_big(buf, pl.seq, pl.g_pass, tw, wp, sbuf);
     const bool direct = !pl.bluestein;
 #define POS(k) (direct ? (s_pos ? static_cast<int>(s_pos[(k)]) : __ldg(pos_tab + (k))) : (k))
 
@@ -757,9 +818,11 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
 
     // 6. inverse complex transform (unnormalised), natural order out
     if (pl.bluestein)
-      bluestein<true>(buf, pl, tables, wp);
-    else
+      bluestein<true>(buf, pl, tables, wp, sbuf);
+    else if (pl.in_smem)
       fft_dit_inv(buf, pl.seq, tw, wp);
+    else
+      fft_dit_inv_big(buf, pl.seq, pl.g_pass, tw, wp, sbuf);
 #undef POS
 
     // 7. residual mix. `smoothed` (optional) gets the result; when budgets are given the result
