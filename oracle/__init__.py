@@ -40,6 +40,8 @@ def _load():
         lib.akvo_rfft.argtypes = [vp, i32, i32, vp, vp]
         lib.akvo_irfft.argtypes = [vp, vp, i32, i32, vp]
         lib.akvo_sss.argtypes = [vp, i32, f64, f64, i32, i32, i32, vp, vp, vp, vp]
+        lib.akvo_smooth_variant.argtypes = [vp, i32, i32, f64, f64, i32, i32, i32, vp, vp]
+        lib.akvo_smooth_variant.restype = ctypes.c_int
         lib.akvo_allocate.argtypes = [vp, i32, i64, i32, i32, i32, vp]
         lib.akvo_select.argtypes = [vp, i32, i32, vp]
         lib.akvo_gather.argtypes = [vp, i32, i32, i64, vp, i32, vp]
@@ -118,6 +120,22 @@ def sss(x: np.ndarray, rho: float, alpha: float, T: int, force_kstar: int = -1, 
     if want_energy:
         return out, kstar.value, margin.value, E
     return out, kstar.value, margin.value
+
+
+FIXED_FRACTION, ENERGY_NO_MEAN, AVG_POOL, MAX_POOL = 1, 2, 3, 4
+
+
+def smooth_variant(x: np.ndarray, mode: int, param: float, alpha: float, T: int = 0, pool: int = 1, direct: bool = False):
+    """The smoothing variants for ablation-style runs (see akvo_smooth_variant). Returns (out, kstar)."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    n = x.shape[0]
+    out = np.zeros(n)
+    kstar = ctypes.c_int(0)
+    rc = _load().akvo_smooth_variant(_ptr(x), n, int(mode), float(param), float(alpha), int(T), int(pool), int(direct),
+                                     _ptr(out), ctypes.cast(ctypes.byref(kstar), ctypes.c_void_p))
+    if rc != 0:
+        raise ValueError("akvo_smooth_variant rejected its arguments")
+    return out, kstar.value
 
 
 def allocate(S: np.ndarray, B: int, w: int, r: int, L: int) -> np.ndarray:

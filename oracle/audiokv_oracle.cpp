@@ -286,6 +286,73 @@ int akvo_sss(const double* x, int n, double rho, double alpha, int T, int force_
 }
 
 // ---------------------------------------------------------------------------
+// Step 2, variants for ablation-style runs. The paper compares against SnapKV, whose local pooling of the
+// scores is what Spectral Score Smoothing replaces (Sections 3.3 and 4.3), and reports the sensitivity of the
+// cut-off over a range of values (Section 4.6), which can also be read as a cut-off at a fixed fraction of
+// the spectrum. None of these is the method itself; they share its residual mix out = (1 - alpha) x + alpha y.
+//   mode 1  fixed-fraction cut-off: k* = floor(param * (n/2)), param in [0, 1]; mask, inverse and mix as in
+//           akvo_sss (T = width of the cosine band).
+//   mode 2  energy cut-off with the mean left out: E'(k) = sum_{1<=i<=k} m_i^2 (E'(0) = 0), k* = the smallest k
+//           with E'(k) >= param * E'(n/2); bin 0 always passes. param = rho in (0, 1].
+//   mode 3  average pooling, window of `pool` (odd) tokens centred on j with zero padding:
+//           y_j = (1/pool) sum_{|i-j| <= pool/2, 0 <= i < n} x_i.
+//   mode 4  max pooling over the same window; padding never wins.
+// kstar_out: the cut-off of modes 1 and 2 (0 for the pooling modes).
+int akvo_smooth_variant(const double* x, int n, int mode, double param, double alpha, int T, int pool, int direct,
+                        double* out, int* kstar_out) {
+  if (n < 1 || T < 0 || mode < 1 || mode > 4) return -1;
+  std::vector<double> y(n);
+  int kstar = 0;
+  if (mode == 1 || mode == 2) {
+    const int Kb = n / 2;
+    std::vector<double> re(Kb + 1), im(Kb + 1);
+    akvo_rfft(x, n, direct, re.data(), im.data());
+    if (mode == 1) {
+      if (!(param >= 0.0 && param <= 1.0)) return -1;
+      kstar = static_cast<int>(std::floor(param * Kb));
+    } else {
+      std::vector<double> E(Kb + 1, 0.0);
+      double run = 0.0;
+      for (int k = 1; k <= Kb; ++k) {
+        run += re[k] * re[k] + im[k] * im[k];
+        E[k] = run;
+      }
+      const double thr = param * E[Kb];
+      kstar = Kb;
+      for (int k = 0; k <= Kb; ++k)
+        if (E[k] >= thr) {
+          kstar = k;
+          break;
+        }
+    }
+    const double pi = 3.14159265358979323846;
+    for (int i = 0; i <= Kb; ++i) {
+      double w = 0.0;
+      if (i <= kstar) w = 1.0;
+      else if (i <= kstar + T) w = 0.5 * (1.0 + std::cos(pi * (i - kstar) / (T + 1)));
+      re[i] *= w;
+      im[i] *= w;
+    }
+    akvo_irfft(re.data(), im.data(), n, direct, y.data());
+  } else {
+    if (pool < 1 || pool % 2 == 0) return -1;
+    const int h = pool / 2;
+    for (int j = 0; j < n; ++j) {
+      double acc = mode == 3 ? 0.0 : -INFINITY;
+      for (int i = j - h; i <= j + h; ++i) {
+        if (i < 0 || i >= n) continue;
+        if (mode == 3) acc += x[i];
+        else acc = std::max(acc, x[i]);
+      }
+      y[j] = mode == 3 ? acc / pool : acc;
+    }
+  }
+  if (kstar_out) *kstar_out = kstar;
+  for (int j = 0; j < n; ++j) out[j] = (1.0 - alpha) * x[j] + alpha * y[j];
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
 // Step 3: head-wise budgets (Section 3.1, the allocation equation
 //   b = w + r + B_score * S / sum S,
 // of which Section 3.2's floor(B * S_hit / sum S_hit) is the case w = r = 0).
