@@ -181,7 +181,8 @@ def run_cuda(args):
     w = wl.generate(spec, seed=rank_seed(rank), layers=args.layers)   # every rank evicts its own request: no exchange step
     spec = w.spec
     L = spec.seq_lens[0]
-    prob = B.Problem.from_workload(w)
+    prob = B.Problem.from_workload(w, smooth_mode=args.smooth_mode, smooth_kappa=args.kappa,
+                                   pool_kernel=args.pool_kernel)
     tb = [int(x) for x in w.total_budget]
     rows, TH = sum(tb), prob.total_heads
     es = w.torch_dtype()
@@ -307,7 +308,8 @@ def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_m
         "config": {"workload": spec.name, "layers": NL, "q_heads": spec.n_q_heads, "kv_heads": spec.n_kv_heads,
                    "head_dim": spec.head_dim, "L": L, "window": spec.window, "keep": spec.keep,
                    "requests_per_gpu": 1, "l2": "inputs larger than L2 (K+V of a step = %d MB)" % (2 * w.k.nbytes // 2**20),
-                   "parallelism": f"replicas x{world}, no collective"},
+                   "parallelism": f"replicas x{world}, no collective",
+                   "smooth_mode": args.smooth_mode},
         "tokens_heads_per_s": round(L * spec.n_kv_heads * NL * world / (ms_step * 1e-3), 1),
         "hbm_gbs": round(hbm_gbs, 1),
         "hbm_frac_of_nominal_8tbs": round(hbm_gbs / NOMINAL_HBM_GBS, 4),
@@ -391,6 +393,11 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--config", type=int, default=1,
                     help="workload index (1 = the benchmark workload; others are for exploration, not bench lines)")
+    ap.add_argument("--smooth-mode", type=int, default=0,
+                    help="0 = Spectral Score Smoothing (the benchmark); 1 fixed-fraction cut-off, 2 energy cut-off without "
+                         "the mean, 3 average pooling, 4 max pooling (variants for ablation-style runs, not bench lines)")
+    ap.add_argument("--kappa", type=float, default=0.5, help="cut-off fraction of --smooth-mode 1")
+    ap.add_argument("--pool-kernel", type=int, default=7, help="window of --smooth-mode 3 and 4 (odd)")
     ap.add_argument("--layers", type=int, default=None,
                     help="truncate the stack to its first LAYERS layers (small cases for profiler captures; not a bench line)")
     args = ap.parse_args()

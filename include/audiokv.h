@@ -43,6 +43,16 @@ extern "C" {
 
 enum { AUDIOKV_F32 = 0, AUDIOKV_BF16 = 1 };
 
+/* Step 2 as the paper defines it, and the variants used for ablation-style runs. */
+enum {
+  AUDIOKV_SMOOTH_SSS = 0,            /* Spectral Score Smoothing: energy cut-off rho (Section 3.3)              */
+  AUDIOKV_SMOOTH_FIXED_FRACTION = 1, /* same filter, cut-off at k* = floor(smooth_kappa * (n/2)): the other     */
+                                     /* reading of the cut-off range in the sensitivity study (Section 4.6)     */
+  AUDIOKV_SMOOTH_ENERGY_NO_MEAN = 2, /* energy cut-off with bin 0 left out of the energy (bin 0 always passes)  */
+  AUDIOKV_SMOOTH_AVG_POOL = 3,       /* local average pooling over pool_kernel tokens, zero padding: the local  */
+  AUDIOKV_SMOOTH_MAX_POOL = 4        /* pooling of the SnapKV lineage that SSS replaces (Sections 3.3, 4.3)     */
+};
+
 enum {
   AUDIOKV_OK = 0,
   AUDIOKV_EINVAL = -1,       /* an argument is out of range or inconsistent            */
@@ -77,6 +87,10 @@ typedef struct {
   float alpha;                   /* SSS mixing coefficient, in [0, 1]                            */
   int32_t transition_bins;       /* T >= 0: cosine band of T bins after the cut-off; 0 = binary mask */
   int32_t base_per_head;         /* r >= 0: uniform base allocation per head, in tokens          */
+  /* Smoothing variant (all zero = the paper's method). See audiokv_smooth.                            */
+  int32_t smooth_mode;           /* AUDIOKV_SMOOTH_*                                             */
+  float smooth_kappa;            /* AUDIOKV_SMOOTH_FIXED_FRACTION: cut-off fraction in [0, 1]    */
+  int32_t pool_kernel;           /* AUDIOKV_SMOOTH_*_POOL: odd window, 1 .. 1023 tokens          */
 } audiokv_params;
 
 #define AUDIOKV_MAX_REQ 64
@@ -148,7 +162,10 @@ int audiokv_score(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
  *   w_i = 1 (i <= k*), (1 + cos(pi (i-k*)/(T+1)))/2 (k* < i <= k*+T), 0 beyond;
  *   x~ = IRFFT(F .* w, n); smoothed = (1 - alpha) x + alpha x~.
  * Any n >= 1 (mixed radix for smooth lengths, chirp-z otherwise). `smoothed` may equal
- * `scores`. kstar_or_null: optional int32 [total heads] receiving k*. */
+ * `scores`. kstar_or_null: optional int32 [total heads] receiving k* (0 for the pooling modes).
+ * Variants (smooth_mode): FIXED_FRACTION and ENERGY_NO_MEAN change only how k* is chosen;
+ * AVG_POOL / MAX_POOL replace x~ by the pooled sequence y_j = mean (zero padding counted) or
+ * max of x over |i - j| <= pool_kernel / 2; the residual mix with alpha is the same. */
 int audiokv_smooth(audiokv_ctx* ctx, const audiokv_params* p, const float* scores, float* smoothed,
                    int32_t* kstar_or_null, audiokv_stream stream);
 

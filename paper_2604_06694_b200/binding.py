@@ -17,6 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libaudiokv.so")
 
 AUDIOKV_F32, AUDIOKV_BF16 = 0, 1
+(AUDIOKV_SMOOTH_SSS, AUDIOKV_SMOOTH_FIXED_FRACTION, AUDIOKV_SMOOTH_ENERGY_NO_MEAN, AUDIOKV_SMOOTH_AVG_POOL,
+ AUDIOKV_SMOOTH_MAX_POOL) = range(5)
 AUDIOKV_OK, AUDIOKV_EINVAL, AUDIOKV_EALIGN, AUDIOKV_EUNSUPPORTED = 0, -1, -2, -3
 AUDIOKV_EWORKSPACE, AUDIOKV_ECUDA, AUDIOKV_ETIMEOUT, AUDIOKV_EDEVICE = -4, -5, -6, -7
 
@@ -39,6 +41,7 @@ class audiokv_params(ctypes.Structure):
         ("kv_req_offset", ctypes.POINTER(ctypes.c_int64)),
         ("softmax_scale", ctypes.c_float), ("rho", ctypes.c_float), ("alpha", ctypes.c_float),
         ("transition_bins", ctypes.c_int32), ("base_per_head", ctypes.c_int32),
+        ("smooth_mode", ctypes.c_int32), ("smooth_kappa", ctypes.c_float), ("pool_kernel", ctypes.c_int32),
     ]
 
 
@@ -102,7 +105,8 @@ class Problem:
     def __init__(self, dtype: int, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
                  seq_lens: Sequence[int], window: int, q_strides: Sequence[int], kv_strides: Sequence[int],
                  kv_req_offset: Optional[Sequence[int]] = None, softmax_scale: float = 0.0, rho: float = 0.5,
-                 alpha: float = 0.5, transition_bins: int = 4, base_per_head: int = 0):
+                 alpha: float = 0.5, transition_bins: int = 4, base_per_head: int = 0, smooth_mode: int = 0,
+                 smooth_kappa: float = 0.0, pool_kernel: int = 1):
         n = len(seq_lens)
         self._seq = (ctypes.c_int32 * n)(*[int(x) for x in seq_lens])
         self._off = (ctypes.c_int64 * n)(*[int(x) for x in kv_req_offset]) if kv_req_offset is not None else None
@@ -115,6 +119,7 @@ class Problem:
         p.kv_req_offset = ctypes.cast(self._off, ctypes.POINTER(ctypes.c_int64)) if self._off is not None else None
         p.softmax_scale, p.rho, p.alpha = softmax_scale, rho, alpha
         p.transition_bins, p.base_per_head = transition_bins, base_per_head
+        p.smooth_mode, p.smooth_kappa, p.pool_kernel = smooth_mode, smooth_kappa, pool_kernel
         self.p = p
         self.seq_lens = [int(x) for x in seq_lens]
 

@@ -73,6 +73,11 @@ int check_params(const audiokv_params* p) {
   if (p->n_req < 1 || p->n_req > AUDIOKV_MAX_REQ || p->window < 1) return AUDIOKV_EINVAL;
   if (!(p->rho > 0.f && p->rho <= 1.f) || !(p->alpha >= 0.f && p->alpha <= 1.f)) return AUDIOKV_EINVAL;
   if (p->transition_bins < 0 || p->base_per_head < 0) return AUDIOKV_EINVAL;
+  if (p->smooth_mode < AUDIOKV_SMOOTH_SSS || p->smooth_mode > AUDIOKV_SMOOTH_MAX_POOL) return AUDIOKV_EINVAL;
+  if (p->smooth_mode == AUDIOKV_SMOOTH_FIXED_FRACTION && !(p->smooth_kappa >= 0.f && p->smooth_kappa <= 1.f))
+    return AUDIOKV_EINVAL;
+  if (p->smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL && (p->pool_kernel < 1 || p->pool_kernel > 1023 || p->pool_kernel % 2 == 0))
+    return AUDIOKV_EINVAL;
   for (int r = 0; r < p->n_req; ++r) {
     if (p->seq_len[r] <= p->window || p->seq_len[r] > AUDIOKV_MAX_SEQ_LEN) return AUDIOKV_EINVAL;
     if (p->kv_req_offset && p->kv_req_offset[r] < 0) return AUDIOKV_EINVAL;
@@ -105,7 +110,8 @@ bool same_plan(const Plan& pl, const audiokv_params* p) {
       a.q_stride_tok != p->q_stride_tok || a.q_stride_head != p->q_stride_head ||
       a.kv_stride_layer != p->kv_stride_layer || a.kv_stride_tok != p->kv_stride_tok ||
       a.kv_stride_head != p->kv_stride_head || a.softmax_scale != p->softmax_scale || a.rho != p->rho ||
-      a.alpha != p->alpha || a.transition_bins != p->transition_bins || a.base_per_head != p->base_per_head)
+      a.alpha != p->alpha || a.transition_bins != p->transition_bins || a.base_per_head != p->base_per_head ||
+      a.smooth_mode != p->smooth_mode || a.smooth_kappa != p->smooth_kappa || a.pool_kernel != p->pool_kernel)
     return false;
   for (int r = 0; r < p->n_req; ++r) {
     if (pl.seq_len[r] != p->seq_len[r]) return false;
@@ -235,6 +241,9 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   sh.alpha = p->alpha;
   sh.transition_bins = p->transition_bins;
   sh.base_per_head = p->base_per_head;
+  sh.smooth_mode = p->smooth_mode;
+  sh.smooth_kappa = p->smooth_kappa;
+  sh.pool_kernel = p->pool_kernel;
 
   pl->reqs.assign(p->n_req, ReqDesc{});
   pl->fft.clear();
@@ -690,7 +699,9 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
   }
   if (rc) return rc;
   if ((rc = do_score(ctx, q_win, k, ws_scores, s))) return rc;
-  if ((rc = do_smooth(ctx, ws_scores, nullptr, ws_kstar, budgets, cu_kept, kept_idx, s))) return rc;
+  // the pooling variants hand their result to the selection through the score buffer itself
+  float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
+  if ((rc = do_smooth(ctx, ws_scores, ws_smoothed, ws_kstar, budgets, cu_kept, kept_idx, s))) return rc;
   return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, s);
 }
 

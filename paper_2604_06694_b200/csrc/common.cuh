@@ -31,6 +31,8 @@ struct Shape {
   float softmax_scale;
   float rho, alpha;
   int32_t transition_bins, base_per_head;
+  int32_t smooth_mode, pool_kernel;  // AUDIOKV_SMOOTH_*; window of the pooling modes
+  float smooth_kappa;                // cut-off fraction of AUDIOKV_SMOOTH_FIXED_FRACTION
 };
 
 // Maps a flat head index to (request, layer, kv head). n_req is small: linear search.

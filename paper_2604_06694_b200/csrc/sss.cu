@@ -690,6 +690,39 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     const float* x = scores + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P;
     float* y = smoothed ? smoothed + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P : nullptr;
 
+    if (sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL) {
+      // Variant: local pooling instead of the spectral filter. The sequence is staged first (scores and smoothed
+      // may be the same array), pooled over |i - j| <= pool_kernel / 2 (average: zero padding counts in the
+      // divisor; maximum: padding never wins), mixed with alpha and written out; the selection then reads it back.
+      float* st = pl.in_smem ? reinterpret_cast<float*>(sbuf)
+                             : reinterpret_cast<float*>(scratch + static_cast<int64_t>(blockIdx.x) * scratch_per_block);
+      loaded_plan = -1;
+      for (int j = threadIdx.x; j < n; j += kSssThreads) st[j] = x[j];
+      __syncthreads();
+      const int hw = sh.pool_kernel / 2;
+      const bool is_max = sh.smooth_mode == AUDIOKV_SMOOTH_MAX_POOL;
+      const float inv_pool = 1.f / static_cast<float>(sh.pool_kernel), al = sh.alpha, om = 1.f - sh.alpha;
+      for (int j = threadIdx.x; j < n; j += kSssThreads) {
+        const int lo = max(0, j - hw), hi = min(n - 1, j + hw);
+        float acc = is_max ? -INFINITY : 0.f;
+        for (int i = lo; i <= hi; ++i) acc = is_max ? fmaxf(acc, st[i]) : acc + st[i];
+        const float pooled = is_max ? acc : acc * inv_pool;
+        if (y) y[j] = fmaf(al, pooled, om * st[j]);
+      }
+      if (threadIdx.x == 0 && kstar_out) kstar_out[u] = 0;
+      __syncthreads();
+      if (budgets != nullptr) {
+        const int P = rq.P, W = sh.window;
+        int k = budgets[u] - W;
+        if (k < 0 || k > P || y == nullptr) {
+          if (threadIdx.x == 0) atomicExch(status, AUDIOKV_EDEVICE);
+          k = k < 0 ? 0 : (k > P ? P : k);
+        }
+        if (y) select_topk([&](int j) -> uint32_t { return score_key(y[j]); }, P, W, k, kept_idx + cu_kept[u], &ssm, status);
+      }
+      continue;
+    }
+
     // 1. load (packed: z_m = x_2m + i x_2m+1)
     if (pl.packed) {
       for (int m = threadIdx.x; m < N; m += kSssThreads) buf[m] = make_float2(x[2 * m], x[2 * m + 1]);
@@ -735,7 +768,9 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     const int nbins = Kb + 1;
     const int per = (nbins + kSssThreads - 1) / kSssThreads;
     const int k0 = min(nbins, static_cast<int>(threadIdx.x) * per), k1 = min(nbins, k0 + per);
+    const bool no_mean = sh.smooth_mode == AUDIOKV_SMOOTH_ENERGY_NO_MEAN;  // variant: bin 0 adds no energy
     auto energy = [&](int k) -> double {
+      if (k == 0 && no_mean) return 0.0;
       if (pl.packed) {
         if (k == 0) return static_cast<double>(buf[0].x) * buf[0].x;
         if (k == N) return static_cast<double>(buf[0].y) * buf[0].y;
@@ -743,6 +778,10 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
       float2 f = buf[POS(k)];
       return static_cast<double>(f.x) * f.x + static_cast<double>(f.y) * f.y;
     };
+    if (sh.smooth_mode == AUDIOKV_SMOOTH_FIXED_FRACTION) {
+      // variant: the cut-off sits at a fixed fraction of the spectrum, no energies needed
+      if (threadIdx.x == 0) s_kstar = static_cast<int>(floor(static_cast<double>(sh.smooth_kappa) * Kb));
+    } else {
     // each thread owns `per` consecutive bins; up to 8 of their energies stay in registers for the second look
     double ecache[8];
     double local = 0.0;
@@ -775,6 +814,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
           found = true;
         }
       }
+    }
     }
     __syncthreads();
     const int kstar = min(s_kstar, Kb);
