@@ -42,6 +42,8 @@ def _load():
         lib.akvo_sss.argtypes = [vp, i32, f64, f64, i32, i32, i32, vp, vp, vp, vp]
         lib.akvo_smooth_variant.argtypes = [vp, i32, i32, f64, f64, i32, i32, i32, vp, vp]
         lib.akvo_smooth_variant.restype = ctypes.c_int
+        lib.akvo_hit_score.argtypes = [vp, i32, i32, ctypes.c_int64, vp, vp, i32, vp, vp]
+        lib.akvo_hit_score.restype = ctypes.c_int
         lib.akvo_allocate.argtypes = [vp, i32, i64, i32, i32, i32, vp]
         lib.akvo_select.argtypes = [vp, i32, i32, vp]
         lib.akvo_gather.argtypes = [vp, i32, i32, i64, vp, i32, vp]
@@ -136,6 +138,21 @@ def smooth_variant(x: np.ndarray, mode: int, param: float, alpha: float, T: int 
     if rc != 0:
         raise ValueError("akvo_smooth_variant rejected its arguments")
     return out, kstar.value
+
+
+def hit_score(attn: np.ndarray, row_len: np.ndarray, span: np.ndarray, K: int = 24):
+    """Offline head score: attn [n_steps][n_heads][row_stride], row_len [n_steps], span [n_steps][2] (inclusive).
+    Returns (s_hit float64 [n_heads], counts int64 [n_heads])."""
+    attn = np.ascontiguousarray(attn, dtype=np.float64)
+    T, H, stride = attn.shape
+    row_len = np.ascontiguousarray(row_len, dtype=np.int32)
+    span = np.ascontiguousarray(span, dtype=np.int32).reshape(T, 2)
+    counts = np.zeros(H, dtype=np.int64)
+    s = np.zeros(H)
+    rc = _load().akvo_hit_score(_ptr(attn), T, H, stride, _ptr(row_len), _ptr(span), int(K), _ptr(counts), _ptr(s))
+    if rc != 0:
+        raise ValueError("akvo_hit_score rejected its arguments")
+    return s, counts
 
 
 def allocate(S: np.ndarray, B: int, w: int, r: int, L: int) -> np.ndarray:

@@ -353,6 +353,40 @@ int akvo_smooth_variant(const double* x, int n, int mode, double param, double a
 }
 
 // ---------------------------------------------------------------------------
+// Offline head score (Section 3.2, "Collecting Attention Hits to Audio Spans" and "Head Importance Estimation").
+// For decode step t and head a, A_t^a is the attention row of the new token over the L_t previous tokens. With
+// S = TopK(A_t^a, K) (ties: the lower token index first) and the audio span [span_lo_t, span_hi_t] (inclusive) of
+// the word generated at step t:
+//     c = |S intersect span|,   r = c / K,   S_hit[a] = mean over the steps of r.
+// A row shorter than K contributes all its tokens. attn: [n_steps][n_heads][row_stride] double.
+// counts (optional): the integer hit totals sum_t c per head.
+int akvo_hit_score(const double* attn, int n_steps, int n_heads, int64_t row_stride, const int32_t* row_len,
+                   const int32_t* span, int K, int64_t* counts, double* s_hit) {
+  if (n_steps < 1 || n_heads < 1 || K < 1) return -1;
+  for (int a = 0; a < n_heads; ++a) {
+    int64_t total = 0;
+    double mean = 0.0;
+    for (int t = 0; t < n_steps; ++t) {
+      const int L = row_len[t];
+      if (L < 0 || L > row_stride) return -1;
+      const double* row = attn + (static_cast<int64_t>(t) * n_heads + a) * row_stride;
+      std::vector<int> idx(L);
+      std::iota(idx.begin(), idx.end(), 0);
+      std::stable_sort(idx.begin(), idx.end(), [&](int i, int j) { return row[i] > row[j]; });
+      const int k = std::min(K, L);
+      int c = 0;
+      for (int i = 0; i < k; ++i)
+        if (idx[i] >= span[2 * t] && idx[i] <= span[2 * t + 1]) ++c;
+      total += c;
+      mean += static_cast<double>(c) / K;
+    }
+    if (counts) counts[a] = total;
+    s_hit[a] = mean / n_steps;
+  }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
 // Step 3: head-wise budgets (Section 3.1, the allocation equation
 //   b = w + r + B_score * S / sum S,
 // of which Section 3.2's floor(B * S_hit / sum S_hit) is the case w = r = 0).

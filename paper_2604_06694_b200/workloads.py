@@ -175,3 +175,29 @@ def generate(spec: WorkloadSpec, seed: int = 0, layers: Optional[int] = None) ->
     B = np.array([kept_total(spec, L) for L in lens], dtype=np.int64)
     base = base_per_head(spec, min(lens))
     return Workload(spec, q, k, v, S, cu, B, base)
+
+
+def attention_rows(n_steps: int, n_heads: int, n_audio: int, n_text0: int = 16, seed: int = 0, word_tokens: int = 12):
+    """Synthetic decode-step attention rows for the offline head-score statistic (the paper records them with hooks
+    on a real model): step t attends over L_t = n_audio + n_text0 + t tokens; the word generated at step t spans
+    `word_tokens` audio tokens that advance with t (speech is read left to right); head a puts a share g_a of its
+    logit mass on that span (g ~ Beta(0.5, 2): few strongly audio-grounded heads) on top of i.i.d. noise and a sink
+    at token 0. Returns (attn float32 [n_steps][n_heads][Lmax] zero-padded, row_len int32, span int32 [n_steps][2],
+    grounding float64 [n_heads])."""
+    rng = np.random.Generator(np.random.Philox(key=[seed, 0xA77]))
+    Lmax = n_audio + n_text0 + n_steps
+    attn = np.zeros((n_steps, n_heads, Lmax), dtype=np.float32)
+    row_len = np.array([n_audio + n_text0 + t for t in range(n_steps)], dtype=np.int32)
+    span = np.zeros((n_steps, 2), dtype=np.int32)
+    g = rng.beta(0.5, 2.0, size=n_heads)
+    for t in range(n_steps):
+        lo = min(n_audio - word_tokens, int(t * (n_audio - word_tokens) / max(1, n_steps - 1)))
+        span[t] = (lo, lo + word_tokens - 1)
+        L = int(row_len[t])
+        z = rng.standard_normal(size=(n_heads, L))
+        z[:, 0] += 4.0
+        z[:, lo:lo + word_tokens] += 6.0 * g[:, None]
+        z -= z.max(axis=1, keepdims=True)
+        p = np.exp(z)
+        attn[t, :, :L] = (p / p.sum(axis=1, keepdims=True)).astype(np.float32)
+    return attn, row_len, span, g
