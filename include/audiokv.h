@@ -209,6 +209,20 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
 size_t audiokv_workspace_bytes_host(const audiokv_params* p, int64_t q_elems, int64_t kv_elems,
                                     const int64_t* total_budget);
 
+/* Offline head score (Section 3.2, "Collecting Attention Hits to Audio Spans" and "Head Importance
+ * Estimation"): the table S that audiokv_allocate consumes. For decode step t and head a, with
+ * S = TopK(attention row, top_k) (ties: lower token index) and the inclusive audio-token span
+ * [span[2t], span[2t+1]] of the word generated at step t:
+ *   c = |S intersect span|,  r = c / top_k,  s_hit[a] = mean over the steps of r.
+ * attn: device fp32 [n_steps][n_heads][row_stride], row t holds row_len[t] <= row_stride tokens (a row
+ * shorter than top_k contributes all of them). row_len: device int32 [n_steps]. span: device int32
+ * [n_steps][2]. top_k in 1..1024 (the paper uses 24). hit_counts: device int32 [n_heads], receives the
+ * integer totals sum_t c. s_hit: device fp32 [n_heads]. The paper records the rows with hooks on a real
+ * model and takes the spans from a word aligner; neither is part of this library. */
+int audiokv_hit_score(audiokv_ctx* ctx, const float* attn, int32_t n_steps, int32_t n_heads, int64_t row_stride,
+                      const int32_t* row_len, const int32_t* span, int32_t top_k, int32_t* hit_counts, float* s_hit,
+                      audiokv_stream stream);
+
 /* Step 1 for callers that cannot allocate device memory (the paper has no counterpart: this
  * is a deployment variant of audiokv_score, same arguments and same result).
  * Who needs it: code running under a memory pool or arena whose owner forbids cudaMalloc

@@ -90,6 +90,8 @@ def lib() -> ctypes.CDLL:
         L.audiokv_allocate.argtypes = [vp, pp, vp, ctypes.POINTER(i64), vp, vp, vp]
         L.audiokv_select_gather.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.audiokv_evict.argtypes = [vp, pp, vp, vp, vp, vp, ctypes.POINTER(i64), vp, vp, vp, vp, vp, vp]
+        L.audiokv_hit_score.argtypes = [vp, vp, i32, i32, i64, vp, vp, i32, vp, vp, vp]
+        L.audiokv_hit_score.restype = ctypes.c_int
         L.audiokv_evict_host.argtypes = [vp, pp, vp, i64, vp, vp, i64, vp, ctypes.POINTER(i64), vp, vp, vp, vp, vp, vp]
         for n in ("audiokv_create", "audiokv_destroy", "audiokv_last_device_status", "audiokv_score",
                   "audiokv_smooth", "audiokv_allocate", "audiokv_select_gather", "audiokv_evict",
@@ -270,6 +272,15 @@ def audiokv_evict(ctx: Context, prob: Problem, q_win, k, v, head_scores, total_b
                                    _dev(head_scores, "head_scores"), _budget_array(total_budget), _dev(k_out, "k_out"),
                                    _dev(v_out, "v_out"), _dev(kept_idx, "kept_idx"), _dev(budgets, "budgets"),
                                    _dev(cu_kept, "cu_kept"), _stream()), "audiokv_evict")
+
+
+def audiokv_hit_score(ctx: Context, attn: torch.Tensor, row_len: torch.Tensor, span: torch.Tensor, top_k: int,
+                      hit_counts: torch.Tensor, s_hit: torch.Tensor) -> None:
+    """attn: CUDA fp32 [n_steps][n_heads][row_stride] (contiguous); row_len int32 [n_steps]; span int32 [n_steps][2]."""
+    n_steps, n_heads, stride = attn.shape
+    ctx._check(lib().audiokv_hit_score(ctx.h, _dev(attn, "attn"), n_steps, n_heads, stride, _dev(row_len, "row_len"),
+                                       _dev(span, "span"), top_k, _dev(hit_counts, "hit_counts"), _dev(s_hit, "s_hit"),
+                                       _stream()), "audiokv_hit_score")
 
 
 def _host(t: torch.Tensor, name: str) -> ctypes.c_void_p:

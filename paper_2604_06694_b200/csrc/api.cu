@@ -558,6 +558,11 @@ int audiokv_create(audiokv_ctx** out, int device, size_t workspace_bytes) {
     return AUDIOKV_ECUDA;
   }
   c->ws_bytes = workspace_bytes;
+  if (workspace_bytes < 64 || cudaMemset(c->ws, 0, 64) != cudaSuccess) {  // the status word starts clean
+    cudaFree(c->ws);
+    delete c;
+    return workspace_bytes < 64 ? AUDIOKV_EINVAL : AUDIOKV_ECUDA;
+  }
   if (cudaEventCreateWithFlags(&c->plan_ready, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->join, cudaEventDisableTiming) != cudaSuccess ||
@@ -588,10 +593,10 @@ int audiokv_destroy(audiokv_ctx* ctx) {
 }
 
 int audiokv_last_device_status(audiokv_ctx* ctx, audiokv_stream stream) {
-  if (!ctx || !ctx->plan.valid) return AUDIOKV_EINVAL;
+  if (!ctx) return AUDIOKV_EINVAL;
   int st = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  cudaError_t e = cudaMemcpyAsync(&st, d_status(ctx), sizeof(int), cudaMemcpyDeviceToHost, s);
+  cudaError_t e = cudaMemcpyAsync(&st, ctx->ws, sizeof(int), cudaMemcpyDeviceToHost, s);  // first word of the workspace
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return st;
@@ -703,6 +708,22 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
   float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
   if ((rc = do_smooth(ctx, ws_scores, ws_smoothed, ws_kstar, budgets, cu_kept, kept_idx, s))) return rc;
   return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, s);
+}
+
+int audiokv_hit_score(audiokv_ctx* ctx, const float* attn, int32_t n_steps, int32_t n_heads, int64_t row_stride,
+                      const int32_t* row_len, const int32_t* span, int32_t top_k, int32_t* hit_counts, float* s_hit,
+                      audiokv_stream stream) {
+  if (!ctx || !attn || !row_len || !span || !hit_counts || !s_hit) return AUDIOKV_EINVAL;
+  if (n_steps < 1 || n_heads < 1 || row_stride < 1 || top_k < 1 || top_k > 1024) return AUDIOKV_EINVAL;
+  if (static_cast<int64_t>(n_steps) * n_heads > 0x7fffffffLL || ctx->ws_bytes < 64) return AUDIOKV_EINVAL;
+  cudaError_t e = cudaSetDevice(ctx->device);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  Launch ln{s, &ctx->launches, &ctx->prof};
+  // the status word is the first thing in the workspace, whatever plan the context holds
+  e = launch_hit_score(attn, n_steps, n_heads, row_stride, row_len, span, top_k, hit_counts, s_hit,
+                       reinterpret_cast<int*>(ctx->ws), ln);
+  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 
 int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, int64_t q_elems, const void* k,

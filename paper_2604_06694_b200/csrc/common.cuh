@@ -165,4 +165,8 @@ cudaError_t launch_select(const Shape& sh, const ReqDesc* d_reqs, const float* s
 cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t* cu_kept, const int32_t* kept_idx,
                           const void* k, const void* v, void* k_out, void* v_out, Launch ln);
 
+// hit_score.cu: offline head score. counts: int32 [n_heads] (cleared here, then the hit totals).
+cudaError_t launch_hit_score(const float* attn, int n_steps, int n_heads, int64_t row_stride, const int32_t* row_len,
+                             const int32_t* span, int top_k, int32_t* counts, float* s_hit, int* status, Launch ln);
+
 }  // namespace akv
