@@ -91,9 +91,11 @@ typedef struct {
   int32_t smooth_mode;           /* AUDIOKV_SMOOTH_*                                             */
   float smooth_kappa;            /* AUDIOKV_SMOOTH_FIXED_FRACTION: cut-off fraction in [0, 1]    */
   int32_t pool_kernel;           /* AUDIOKV_SMOOTH_*_POOL: odd window, 1 .. 1023 tokens          */
+  const int64_t* q_req_offset;   /* host [n_req], or NULL: element offset of request r's window queries,
+                                    replacing r*q_stride_req (which is then ignored)              */
 } audiokv_params;
 
-#define AUDIOKV_MAX_REQ 64
+#define AUDIOKV_MAX_REQ 8192
 #define AUDIOKV_MAX_SEQ_LEN 131072
 
 /* ---- host-side helpers (no GPU work) ------------------------------------------------ */
@@ -209,6 +211,30 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
 size_t audiokv_workspace_bytes_host(const audiokv_params* p, int64_t q_elems, int64_t kv_elems,
                                     const int64_t* total_budget);
 
+/* Decode-time re-eviction of an already compacted cache (Section 3.3: the importance
+ * sequence may also come from a sliding window of decoding steps; Fig. 3, decoding phase).
+ * After an eviction every head has its own length, so the cache is ragged per head: head
+ * u = (r*n_layers + l)*n_kv_heads + h holds rows [cu_cache[u], cu_cache[u+1]) of k_cache
+ * and v_cache (device, [rows][head_dim], row stride head_dim) in token order, the tokens
+ * decoded since the last eviction appended at the end; the last `window` rows are the
+ * tokens whose queries q_win holds (layout and strides as in audiokv_score). The call runs
+ * steps 1, 2 and 4 on every head with its own length n_u: scores of the first n_u - W rows,
+ * smoothing, the new_budgets[u] - W best of them plus the window, gathered.
+ *   p: dtype, n_layers, n_q_heads, n_kv_heads, head_dim, n_req, window, the q strides
+ *      (and q_req_offset), softmax_scale and the smoothing fields are read; seq_len, the kv
+ *      strides, kv_req_offset and base_per_head are ignored.
+ *   cu_cache: HOST int32 [total heads + 1], cu_cache[0] = 0, every n_u in (W, AUDIOKV_MAX_SEQ_LEN].
+ *   new_budgets: HOST int32 [total heads], W <= new_budgets[u] <= n_u: rows head u keeps.
+ *   k_out / v_out: device, sum_u new_budgets[u] rows; kept_idx: device int32, as many entries,
+ *      positions inside the head's own cache rows, ascending; cu_kept: device int32
+ *      [total heads + 1], the prefix sums of new_budgets.
+ * total heads <= AUDIOKV_MAX_REQ (else AUDIOKV_EUNSUPPORTED). The context's workspace must hold
+ * audiokv_reevict_workspace_bytes(p, cu_cache) bytes (0 on invalid arguments). */
+size_t audiokv_reevict_workspace_bytes(const audiokv_params* p, const int32_t* cu_cache);
+int audiokv_reevict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k_cache,
+                    const void* v_cache, const int32_t* cu_cache, const int32_t* new_budgets, void* k_out, void* v_out,
+                    int32_t* kept_idx, int32_t* cu_kept, audiokv_stream stream);
+
 /* Offline head score (Section 3.2, "Collecting Attention Hits to Audio Spans" and "Head Importance
  * Estimation"): the table S that audiokv_allocate consumes. For decode step t and head a, with
  * S = TopK(attention row, top_k) (ties: lower token index) and the inclusive audio-token span
@@ -231,7 +257,8 @@ int audiokv_hit_score(audiokv_ctx* ctx, const float* attn, int32_t n_steps, int3
  * no context: its scratch (the per-slab softmax statistics and the request table) is a fixed
  * 8 MiB array inside the library image, which every GPU that loads the library holds until
  * the process exits. It calls no cudaMalloc / cudaFree and no allocating library routine.
- *   - Limit: n_req * n_layers * n_kv_heads * ceil(max L / 512) * W * G * 8 bytes must fit in
+ *   - Limits: n_req <= 64 (more is AUDIOKV_EINVAL), and
+ *     n_req * n_layers * n_kv_heads * ceil(max L / 512) * W * G * 8 bytes must fit in
  *     8 MiB - 4 KiB (e.g. 28 layers x 4 KV heads at L = 8192, W = 32, G = 7 needs 3.1 MiB);
  *     larger problems return AUDIOKV_EWORKSPACE. fp32 FMA arithmetic for both element types.
  *   - The first call on a device looks up the array's device address; make that first call

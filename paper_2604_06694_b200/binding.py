@@ -42,6 +42,7 @@ class audiokv_params(ctypes.Structure):
         ("softmax_scale", ctypes.c_float), ("rho", ctypes.c_float), ("alpha", ctypes.c_float),
         ("transition_bins", ctypes.c_int32), ("base_per_head", ctypes.c_int32),
         ("smooth_mode", ctypes.c_int32), ("smooth_kappa", ctypes.c_float), ("pool_kernel", ctypes.c_int32),
+        ("q_req_offset", ctypes.POINTER(ctypes.c_int64)),
     ]
 
 
@@ -90,6 +91,10 @@ def lib() -> ctypes.CDLL:
         L.audiokv_allocate.argtypes = [vp, pp, vp, ctypes.POINTER(i64), vp, vp, vp]
         L.audiokv_select_gather.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.audiokv_evict.argtypes = [vp, pp, vp, vp, vp, vp, ctypes.POINTER(i64), vp, vp, vp, vp, vp, vp]
+        L.audiokv_reevict_workspace_bytes.restype = sz
+        L.audiokv_reevict_workspace_bytes.argtypes = [pp, ctypes.POINTER(i32)]
+        L.audiokv_reevict.argtypes = [vp, pp, vp, vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), vp, vp, vp, vp, vp]
+        L.audiokv_reevict.restype = ctypes.c_int
         L.audiokv_hit_score.argtypes = [vp, vp, i32, i32, i64, vp, vp, i32, vp, vp, vp]
         L.audiokv_hit_score.restype = ctypes.c_int
         L.audiokv_evict_host.argtypes = [vp, pp, vp, i64, vp, vp, i64, vp, ctypes.POINTER(i64), vp, vp, vp, vp, vp, vp]
@@ -108,8 +113,9 @@ class Problem:
                  seq_lens: Sequence[int], window: int, q_strides: Sequence[int], kv_strides: Sequence[int],
                  kv_req_offset: Optional[Sequence[int]] = None, softmax_scale: float = 0.0, rho: float = 0.5,
                  alpha: float = 0.5, transition_bins: int = 4, base_per_head: int = 0, smooth_mode: int = 0,
-                 smooth_kappa: float = 0.0, pool_kernel: int = 1):
+                 smooth_kappa: float = 0.0, pool_kernel: int = 1, q_req_offset: Optional[Sequence[int]] = None):
         n = len(seq_lens)
+        self._qoff = (ctypes.c_int64 * n)(*[int(x) for x in q_req_offset]) if q_req_offset is not None else None
         self._seq = (ctypes.c_int32 * n)(*[int(x) for x in seq_lens])
         self._off = (ctypes.c_int64 * n)(*[int(x) for x in kv_req_offset]) if kv_req_offset is not None else None
         p = audiokv_params()
@@ -122,6 +128,7 @@ class Problem:
         p.softmax_scale, p.rho, p.alpha = softmax_scale, rho, alpha
         p.transition_bins, p.base_per_head = transition_bins, base_per_head
         p.smooth_mode, p.smooth_kappa, p.pool_kernel = smooth_mode, smooth_kappa, pool_kernel
+        p.q_req_offset = ctypes.cast(self._qoff, ctypes.POINTER(ctypes.c_int64)) if self._qoff is not None else None
         self.p = p
         self.seq_lens = [int(x) for x in seq_lens]
 
@@ -272,6 +279,23 @@ def audiokv_evict(ctx: Context, prob: Problem, q_win, k, v, head_scores, total_b
                                    _dev(head_scores, "head_scores"), _budget_array(total_budget), _dev(k_out, "k_out"),
                                    _dev(v_out, "v_out"), _dev(kept_idx, "kept_idx"), _dev(budgets, "budgets"),
                                    _dev(cu_kept, "cu_kept"), _stream()), "audiokv_evict")
+
+
+def _i32_array(a: Sequence[int]):
+    return (ctypes.c_int32 * len(a))(*[int(x) for x in a])
+
+
+def audiokv_reevict_workspace_bytes(prob: Problem, cu_cache: Sequence[int]) -> int:
+    return int(lib().audiokv_reevict_workspace_bytes(prob.ref, _i32_array(cu_cache)))
+
+
+def audiokv_reevict(ctx: Context, prob: Problem, q_win, k_cache, v_cache, cu_cache: Sequence[int],
+                    new_budgets: Sequence[int], k_out, v_out, kept_idx, cu_kept) -> None:
+    """cu_cache and new_budgets are host sequences; everything else is a CUDA tensor."""
+    ctx._check(lib().audiokv_reevict(ctx.h, prob.ref, _dev(q_win, "q_win"), _dev(k_cache, "k_cache"),
+                                     _dev(v_cache, "v_cache"), _i32_array(cu_cache), _i32_array(new_budgets),
+                                     _dev(k_out, "k_out"), _dev(v_out, "v_out"), _dev(kept_idx, "kept_idx"),
+                                     _dev(cu_kept, "cu_kept"), _stream()), "audiokv_reevict")
 
 
 def audiokv_hit_score(ctx: Context, attn: torch.Tensor, row_len: torch.Tensor, span: torch.Tensor, top_k: int,

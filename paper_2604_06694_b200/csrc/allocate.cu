@@ -12,9 +12,12 @@ namespace {
 
 constexpr int kAllocThreads = 256;
 
+constexpr int kAllocChunk = 64;  // requests per launch: their totals travel as kernel arguments
+
 struct BudgetArgs {
-  int64_t total[AUDIOKV_MAX_REQ];    // B_r
-  int64_t cu_base[AUDIOKV_MAX_REQ];  // rows kept by the requests before r: sum of their B (budgets add up exactly)
+  int32_t r0;                    // first request of this launch
+  int64_t total[kAllocChunk];    // B_r of requests r0, r0 + 1, ...
+  int64_t cu_base[kAllocChunk];  // rows kept by the requests before r: sum of their B (budgets add up exactly)
 };
 
 __device__ __forceinline__ long long block_sum_ll(long long v, long long* red) {
@@ -40,12 +43,12 @@ allocate_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restr
   int* give = active + N;                         // [N] 1 when the head receives a left-over row this turn
   __shared__ long long red[kAllocThreads / 32];
 
-  const int r = blockIdx.x;
+  const int r = args.r0 + blockIdx.x;
   const ReqDesc rq = reqs[r];
   const float* S = head_scores + static_cast<int64_t>(r) * N;
   const long long f = static_cast<long long>(sh.window) + sh.base_per_head;
   const long long cap = rq.L - f;
-  long long R = args.total[r] - static_cast<long long>(N) * f;
+  long long R = args.total[blockIdx.x] - static_cast<long long>(N) * f;
 
   for (int h = threadIdx.x; h < N; h += kAllocThreads) {
     const double v = static_cast<double>(S[h]);
@@ -149,14 +152,14 @@ allocate_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restr
   __syncthreads();
   if (lane == 31) red[warp] = inc;
   __syncthreads();
-  long long run = args.cu_base[r] + inc - local;
+  long long run = args.cu_base[blockIdx.x] + inc - local;
   for (int w = 0; w < warp; ++w) run += red[w];
   for (int h = a; h < b; ++h) {
     cu_kept[rq.head_base + h] = static_cast<int32_t>(run);
     run += f + tk[h];
   }
   if (r == sh.n_req - 1 && threadIdx.x == 0)
-    cu_kept[sh.total_heads] = static_cast<int32_t>(args.cu_base[r] + args.total[r]);
+    cu_kept[sh.total_heads] = static_cast<int32_t>(args.cu_base[blockIdx.x] + args.total[blockIdx.x]);
 }
 
 }  // namespace
@@ -164,21 +167,27 @@ allocate_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restr
 cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float* head_scores,
                             const int64_t* h_total_budget, int32_t* budgets, int32_t* cu_kept, int* status,
                             Launch ln) {
-  BudgetArgs args;
-  int64_t rows = 0;
-  for (int r = 0; r < sh.n_req; ++r) {
-    args.total[r] = h_total_budget[r];
-    args.cu_base[r] = rows;
-    rows += h_total_budget[r];
-  }
-  if (rows > 0x7fffffffLL) return cudaErrorInvalidValue;  // cu_kept is int32
+  int64_t all = 0;
+  for (int r = 0; r < sh.n_req; ++r) all += h_total_budget[r];
+  if (all > 0x7fffffffLL) return cudaErrorInvalidValue;  // cu_kept is int32
   const size_t smem = static_cast<size_t>(sh.heads_per_req) * (3 * sizeof(long long) + 2 * sizeof(int));
   cudaError_t e = cudaFuncSetAttribute(allocate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  allocate_kernel<<<sh.n_req, kAllocThreads, smem, ln.stream>>>(sh, d_reqs, head_scores, args, budgets, cu_kept,
-                                                                 status);
-  ln.done("allocate");
-  return cudaGetLastError();
+  int64_t rows = 0;
+  for (int r0 = 0; r0 < sh.n_req; r0 += kAllocChunk) {
+    const int n = sh.n_req - r0 < kAllocChunk ? sh.n_req - r0 : kAllocChunk;
+    BudgetArgs args{};
+    args.r0 = r0;
+    for (int i = 0; i < n; ++i) {
+      args.total[i] = h_total_budget[r0 + i];
+      args.cu_base[i] = rows;
+      rows += h_total_budget[r0 + i];
+    }
+    allocate_kernel<<<n, kAllocThreads, smem, ln.stream>>>(sh, d_reqs, head_scores, args, budgets, cu_kept, status);
+    ln.done("allocate");
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace akv

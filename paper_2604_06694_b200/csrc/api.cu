@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <string>
+#include <unordered_map>
 #include <vector>
 
 #include "common.cuh"
@@ -22,19 +23,20 @@ constexpr int kMaxHeadsPerReq = 2048;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {  // byte offsets inside the workspace
-  size_t status, reqs, plans, tables, units, order, stats, fft_scratch, scores, kstar, end;
+  size_t status, reqs, plans, tables, units, order, stats, fft_scratch, scores, kstar, aux, end;
 };
 
 struct Plan {
   bool valid = false;
   audiokv_params p{};
   std::vector<int32_t> seq_len;
-  std::vector<int64_t> kv_off;
+  std::vector<int64_t> kv_off, q_off;
   Shape sh{};
   std::vector<ReqDesc> reqs;
   std::vector<FftPlan> fft;
   std::vector<ScoreUnit> units;   // sweep 1 (all keys, ascending) then sweep 2 (prefix keys, descending)
   int n_units1 = 0, n_units2 = 0;
+  std::vector<int> unit_pre1, unit_pre2;  // [n_req + 1]: units of the requests before r, per sweep
   std::vector<int32_t> sss_order;  // heads in the order the smoothing blocks take them (see build_plan); -1 = none
   int64_t table_len = 0;        // float2 elements
   int64_t scores_len = 0;
@@ -60,6 +62,9 @@ struct audiokv_ctx {
   int64_t launches = 0;
   Profiler prof;
   std::string cuda_error;
+  // audiokv_reevict: the per-head problem it hands to the eviction pass
+  std::vector<int32_t> re_len;
+  std::vector<int64_t> re_kv_off, re_q_off, re_budget;
 };
 
 namespace {
@@ -81,6 +86,7 @@ int check_params(const audiokv_params* p) {
   for (int r = 0; r < p->n_req; ++r) {
     if (p->seq_len[r] <= p->window || p->seq_len[r] > AUDIOKV_MAX_SEQ_LEN) return AUDIOKV_EINVAL;
     if (p->kv_req_offset && p->kv_req_offset[r] < 0) return AUDIOKV_EINVAL;
+    if (p->q_req_offset && p->q_req_offset[r] < 0) return AUDIOKV_EINVAL;
   }
   if (p->head_dim != 64 && p->head_dim != 128 && p->head_dim != 256) return AUDIOKV_EUNSUPPORTED;
   const int64_t rows = static_cast<int64_t>(p->window) * (p->n_q_heads / p->n_kv_heads);
@@ -93,9 +99,10 @@ int check_params(const audiokv_params* p) {
     if (s < 0) return AUDIOKV_EINVAL;
     if (s % per16) return AUDIOKV_EALIGN;
   }
-  if (p->kv_req_offset)
-    for (int r = 0; r < p->n_req; ++r)
-      if (p->kv_req_offset[r] % per16) return AUDIOKV_EALIGN;
+  for (int r = 0; r < p->n_req; ++r) {
+    if (p->kv_req_offset && p->kv_req_offset[r] % per16) return AUDIOKV_EALIGN;
+    if (p->q_req_offset && p->q_req_offset[r] % per16) return AUDIOKV_EALIGN;
+  }
   return AUDIOKV_OK;
 }
 
@@ -106,7 +113,7 @@ bool same_plan(const Plan& pl, const audiokv_params* p) {
   const audiokv_params& a = pl.p;
   if (a.dtype != p->dtype || a.n_layers != p->n_layers || a.n_q_heads != p->n_q_heads ||
       a.n_kv_heads != p->n_kv_heads || a.head_dim != p->head_dim || a.n_req != p->n_req || a.window != p->window ||
-      a.q_stride_req != p->q_stride_req || a.q_stride_layer != p->q_stride_layer ||
+      a.q_stride_layer != p->q_stride_layer ||
       a.q_stride_tok != p->q_stride_tok || a.q_stride_head != p->q_stride_head ||
       a.kv_stride_layer != p->kv_stride_layer || a.kv_stride_tok != p->kv_stride_tok ||
       a.kv_stride_head != p->kv_stride_head || a.softmax_scale != p->softmax_scale || a.rho != p->rho ||
@@ -116,6 +123,7 @@ bool same_plan(const Plan& pl, const audiokv_params* p) {
   for (int r = 0; r < p->n_req; ++r) {
     if (pl.seq_len[r] != p->seq_len[r]) return false;
     if (pl.kv_off[r] != (p->kv_req_offset ? p->kv_req_offset[r] : 0)) return false;
+    if (pl.q_off[r] != (p->q_req_offset ? p->q_req_offset[r] : r * p->q_stride_req)) return false;
   }
   return true;
 }
@@ -215,8 +223,11 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   pl->seq_len.assign(p->seq_len, p->seq_len + p->n_req);
   pl->kv_off.assign(p->n_req, 0);
   if (p->kv_req_offset) pl->kv_off.assign(p->kv_req_offset, p->kv_req_offset + p->n_req);
+  pl->q_off.resize(p->n_req);
+  for (int r = 0; r < p->n_req; ++r) pl->q_off[r] = p->q_req_offset ? p->q_req_offset[r] : r * p->q_stride_req;
   pl->p.seq_len = nullptr;
   pl->p.kv_req_offset = nullptr;
+  pl->p.q_req_offset = nullptr;
 
   Shape& sh = pl->sh;
   sh.dtype = p->dtype;
@@ -250,27 +261,26 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   pl->table_len = 0;
   pl->scores_len = 0;
   pl->max_L = pl->max_P = 0;
+  std::unordered_map<int, int> plan_of;  // prefix length -> index into pl->fft
   for (int r = 0; r < p->n_req; ++r) {
     ReqDesc& d = pl->reqs[r];
     d.L = p->seq_len[r];
     d.P = d.L - p->window;
     d.head_base = r * sh.heads_per_req;
     d.kv_offset = pl->kv_off[r];
-    d.q_offset = r * p->q_stride_req;
+    d.q_offset = pl->q_off[r];
     d.score_offset = pl->scores_len;
     pl->scores_len += static_cast<int64_t>(sh.heads_per_req) * d.P;
     pl->max_L = d.L > pl->max_L ? d.L : pl->max_L;
     pl->max_P = d.P > pl->max_P ? d.P : pl->max_P;
-    int found = -1;
-    for (size_t i = 0; i < pl->fft.size(); ++i)
-      if (pl->fft[i].n == d.P) found = static_cast<int>(i);
-    if (found < 0) {
+    auto it = plan_of.find(d.P);
+    if (it == plan_of.end()) {
       FftPlan fp;
       build_fft_plan(d.P, &fp, &pl->table_len);
       pl->fft.push_back(fp);
-      found = static_cast<int>(pl->fft.size()) - 1;
+      it = plan_of.emplace(d.P, static_cast<int>(pl->fft.size()) - 1).first;
     }
-    d.fft_plan = found;
+    d.fft_plan = it->second;
   }
   pl->n_slab = (pl->max_L + kSlabKeys - 1) / kSlabKeys;
   // Schedule of the tensor-core scoring: sweep 1 walks the heads in order; sweep 2 walks them backwards, since the
@@ -278,8 +288,11 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   pl->units.clear();
   for (int sweep = 1; sweep <= 2; ++sweep) {
     const size_t first = pl->units.size();
+    std::vector<int>& pre = sweep == 1 ? pl->unit_pre1 : pl->unit_pre2;
+    pre.assign(p->n_req + 1, 0);
     for (int r = 0; r < p->n_req; ++r) {
       const ReqDesc& d = pl->reqs[r];
+      pre[r] = static_cast<int>(pl->units.size() - first);
       const int range = sweep == 1 ? d.L : d.P;
       const int slabs = (range + kSlabKeys - 1) / kSlabKeys;
       for (int hr = 0; hr < sh.heads_per_req; ++hr)
@@ -299,6 +312,7 @@ int build_plan(const audiokv_params* p, Plan* pl) {
           pl->units.push_back(un);
         }
     }
+    pre[p->n_req] = static_cast<int>(pl->units.size() - first);
     if (sweep == 1) pl->n_units1 = static_cast<int>(pl->units.size());
     else {
       pl->n_units2 = static_cast<int>(pl->units.size() - first);
@@ -349,8 +363,8 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   Layout& L = pl->lay;
   size_t off = 0;
   L.status = off;      off = align_up(off + 64);
-  L.reqs = off;        off = align_up(off + sizeof(ReqDesc) * AUDIOKV_MAX_REQ);
-  L.plans = off;       off = align_up(off + sizeof(FftPlan) * kMaxPlans);
+  L.reqs = off;        off = align_up(off + sizeof(ReqDesc) * pl->reqs.size());
+  L.plans = off;       off = align_up(off + sizeof(FftPlan) * pl->fft.size());
   L.tables = off;      off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->table_len));
   L.units = off;       off = align_up(off + sizeof(ScoreUnit) * pl->units.size());
   L.order = off;       off = align_up(off + sizeof(int32_t) * pl->sss_order.size());
@@ -358,6 +372,7 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   L.fft_scratch = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->scratch_per_block) * pl->sss_grid);
   L.scores = off;      off = align_up(off + sizeof(float) * static_cast<size_t>(pl->scores_len));
   L.kstar = off;       off = align_up(off + sizeof(int32_t) * static_cast<size_t>(sh.total_heads));
+  L.aux = off;         off = align_up(off + 2 * sizeof(int32_t) * static_cast<size_t>(sh.total_heads));  // audiokv_reevict
   L.end = off;
   pl->valid = true;
   return AUDIOKV_OK;
@@ -429,8 +444,8 @@ int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cuda
   if (score_umma_takes(pl.sh))
   {
     const ScoreUnit* units = reinterpret_cast<const ScoreUnit*>(ctx->ws + pl.lay.units);
-    e = launch_score_umma(pl.sh, pl.reqs.data(), units, pl.n_units1, units + pl.n_units1, pl.n_units2, q, k, scores,
-                          stats, pl.n_slab, kSlabKeys, d_status(ctx), ln);
+    e = launch_score_umma(pl.sh, pl.reqs.data(), units, pl.unit_pre1.data(), units + pl.n_units1, pl.unit_pre2.data(),
+                          q, k, scores, stats, pl.n_slab, kSlabKeys, d_status(ctx), ln);
   }
   if (e == cudaErrorNotSupported)  // fp32 inputs, W * G above 256, or strides the copy engine cannot take
     e = launch_score_simt(pl.sh, d_reqs(ctx), q, k, scores, stats, pl.n_slab, kSlabKeys, ln);
@@ -708,6 +723,86 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
   float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
   if ((rc = do_smooth(ctx, ws_scores, ws_smoothed, ws_kstar, budgets, cu_kept, kept_idx, s))) return rc;
   return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, s);
+}
+
+namespace {
+
+// The per-head problem of a re-eviction: every head of the compacted cache becomes a request of one layer and one
+// KV head, with its own length, its own place in the packed cache and its own slice of the window queries.
+int reevict_problem(audiokv_ctx* ctx, const audiokv_params* p, const int32_t* cu_cache, const int32_t* new_budgets,
+                    audiokv_params* dp) {
+  if (!ctx || !p || !cu_cache) return AUDIOKV_EINVAL;
+  if (p->n_layers < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads || p->n_req < 1 ||
+      p->head_dim < 1)
+    return AUDIOKV_EINVAL;
+  const int64_t TH = static_cast<int64_t>(p->n_req) * p->n_layers * p->n_kv_heads;
+  if (TH > AUDIOKV_MAX_REQ) return AUDIOKV_EUNSUPPORTED;
+  const int G = p->n_q_heads / p->n_kv_heads;
+  ctx->re_len.resize(TH);
+  ctx->re_kv_off.resize(TH);
+  ctx->re_q_off.resize(TH);
+  ctx->re_budget.resize(TH);
+  if (cu_cache[0] != 0) return AUDIOKV_EINVAL;
+  int64_t u = 0;
+  for (int r = 0; r < p->n_req; ++r) {
+    const int64_t q_r = p->q_req_offset ? p->q_req_offset[r] : r * p->q_stride_req;
+    for (int l = 0; l < p->n_layers; ++l)
+      for (int h = 0; h < p->n_kv_heads; ++h, ++u) {
+        const int64_t n = static_cast<int64_t>(cu_cache[u + 1]) - cu_cache[u];
+        if (n <= p->window || n > AUDIOKV_MAX_SEQ_LEN) return AUDIOKV_EINVAL;
+        ctx->re_len[u] = static_cast<int32_t>(n);
+        ctx->re_kv_off[u] = static_cast<int64_t>(cu_cache[u]) * p->head_dim;
+        ctx->re_q_off[u] = q_r + l * p->q_stride_layer + static_cast<int64_t>(h) * G * p->q_stride_head;
+        if (new_budgets) {
+          if (new_budgets[u] < p->window || new_budgets[u] > n) return AUDIOKV_EINVAL;
+          ctx->re_budget[u] = new_budgets[u];
+        }
+      }
+  }
+  *dp = *p;
+  dp->n_req = static_cast<int32_t>(TH);
+  dp->n_layers = 1;
+  dp->n_kv_heads = 1;
+  dp->n_q_heads = G;
+  dp->seq_len = ctx->re_len.data();
+  dp->q_stride_req = 0;
+  dp->q_stride_layer = 0;
+  dp->kv_stride_layer = 0;
+  dp->kv_stride_head = 0;
+  dp->kv_stride_tok = p->head_dim;
+  dp->kv_req_offset = ctx->re_kv_off.data();
+  dp->q_req_offset = ctx->re_q_off.data();
+  dp->base_per_head = 0;
+  return AUDIOKV_OK;
+}
+
+}  // namespace
+
+size_t audiokv_reevict_workspace_bytes(const audiokv_params* p, const int32_t* cu_cache) {
+  audiokv_ctx tmp;
+  audiokv_params dp;
+  if (reevict_problem(&tmp, p, cu_cache, nullptr, &dp)) return 0;
+  return audiokv_workspace_bytes(&dp);
+}
+
+int audiokv_reevict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k_cache,
+                    const void* v_cache, const int32_t* cu_cache, const int32_t* new_budgets, void* k_out, void* v_out,
+                    int32_t* kept_idx, int32_t* cu_kept, audiokv_stream stream) {
+  if (!new_budgets) return AUDIOKV_EINVAL;
+  audiokv_params dp;
+  int rc = reevict_problem(ctx, p, cu_cache, new_budgets, &dp);
+  if (rc) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if ((rc = prepare(ctx, &dp, s))) return rc;
+  // One head per request: the allocation hands each its whole total, whatever the weight. The weights and the
+  // per-head budgets it writes live in the workspace.
+  const size_t TH = ctx->re_len.size();
+  float* weights = reinterpret_cast<float*>(ctx->ws + ctx->plan.lay.aux);
+  int32_t* budgets = reinterpret_cast<int32_t*>(weights + TH);
+  cudaError_t e = cudaMemsetAsync(weights, 0x3f, sizeof(float) * TH, s);  // 0x3f3f3f3f = 0.747
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return audiokv_evict(ctx, &dp, q_win, k_cache, v_cache, weights, ctx->re_budget.data(), k_out, v_out, kept_idx,
+                       budgets, cu_kept, s);
 }
 
 int audiokv_hit_score(audiokv_ctx* ctx, const float* attn, int32_t n_steps, int32_t n_heads, int64_t row_stride,

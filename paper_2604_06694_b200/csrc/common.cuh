@@ -69,7 +69,6 @@ struct FftPlan {
   int64_t pos_offset;     // float2 index of an int32 table: slot of bin k after the forward passes (direct)
 };
 
-constexpr int kMaxPlans = AUDIOKV_MAX_REQ;
 
 // float2 slots of a shared-memory work buffer of `len` elements: element i sits at i + (i >> 4) (see SkewBuf in sss.cu)
 __host__ __device__ inline int sss_padded(int len) { return len + (len >> 4) + 1; }
@@ -141,9 +140,10 @@ struct ScoreUnit {
 // h_reqs: host copy of the request table (the tensor maps are encoded on the host).
 bool score_umma_takes(const Shape& sh);
 // units1 / units2: device tables of the two sweeps (build_score_units gives their host form).
-cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, int n_units1,
-                              const ScoreUnit* units2, int n_units2, const void* q, const void* k, float* scores,
-                              float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln);
+// unit_pre1 / unit_pre2: host arrays [n_req + 1], units of the requests before r in either sweep.
+cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
+                              const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
+                              float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln);
 
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);

@@ -286,7 +286,8 @@ extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const 
   if (device < 0 || device >= kNoAllocMaxDevices) return AUDIOKV_EINVAL;
   if (p->dtype != AUDIOKV_F32 && p->dtype != AUDIOKV_BF16) return AUDIOKV_EINVAL;
   if (p->n_layers < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads) return AUDIOKV_EINVAL;
-  if (p->n_req < 1 || p->n_req > AUDIOKV_MAX_REQ || p->window < 1) return AUDIOKV_EINVAL;
+  constexpr int kNoAllocMaxReq = 64;  // the request table has a fixed slot in the static scratch
+  if (p->n_req < 1 || p->n_req > kNoAllocMaxReq || p->window < 1) return AUDIOKV_EINVAL;
   if (p->head_dim != 64 && p->head_dim != 128 && p->head_dim != 256) return AUDIOKV_EUNSUPPORTED;
   const int G = p->n_q_heads / p->n_kv_heads;
   const int64_t R = static_cast<int64_t>(p->window) * G;
@@ -299,7 +300,7 @@ extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const 
     if (s % per16) return AUDIOKV_EALIGN;
   }
   if ((reinterpret_cast<uintptr_t>(q_win) | reinterpret_cast<uintptr_t>(k)) & 15u) return AUDIOKV_EALIGN;
-  static_assert(sizeof(ReqDesc) * AUDIOKV_MAX_REQ <= kNoAllocTableBytes, "request table must fit its slot");
+  static_assert(sizeof(ReqDesc) * kNoAllocMaxReq <= kNoAllocTableBytes, "request table must fit its slot");
 
   Shape sh{};
   sh.dtype = p->dtype;
@@ -321,7 +322,7 @@ extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const 
   sh.softmax_scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(static_cast<float>(p->head_dim));
   sh.scale_log2e = static_cast<float>(static_cast<double>(sh.softmax_scale) * 1.4426950408889634);
 
-  ReqDesc reqs[AUDIOKV_MAX_REQ];
+  ReqDesc reqs[kNoAllocMaxReq];
   int max_L = 0;
   int64_t score_off = 0;
   for (int r = 0; r < p->n_req; ++r) {
@@ -330,7 +331,10 @@ extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const 
     const int64_t off = p->kv_req_offset ? p->kv_req_offset[r] : 0;
     if (off < 0) return AUDIOKV_EINVAL;
     if (off % per16) return AUDIOKV_EALIGN;
-    reqs[r] = ReqDesc{L, L - p->window, r * sh.heads_per_req, 0, off, r * p->q_stride_req, score_off};
+    const int64_t q_off = p->q_req_offset ? p->q_req_offset[r] : r * p->q_stride_req;
+    if (q_off < 0) return AUDIOKV_EINVAL;
+    if (q_off % per16) return AUDIOKV_EALIGN;
+    reqs[r] = ReqDesc{L, L - p->window, r * sh.heads_per_req, 0, off, q_off, score_off};
     score_off += static_cast<int64_t>(sh.heads_per_req) * (L - p->window);
     max_L = L > max_L ? L : max_L;
   }

@@ -36,9 +36,11 @@ constexpr int kMaxStages = 8;
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
 constexpr int kSmemLimit = 232448;               // 227 KB
 
+constexpr int kMapChunk = 64;  // requests per launch: their tensor maps travel as kernel arguments
+
 struct TmapPack {
-  CUtensorMap q;                   // 5-D: (d, query head, window row, layer, request)
-  CUtensorMap k[AUDIOKV_MAX_REQ];  // 4-D per request: (d, token, KV head, layer)
+  CUtensorMap q[kMapChunk];  // 4-D per request: (d, query head, window row, layer)
+  CUtensorMap k[kMapChunk];  // 4-D per request: (d, token, KV head, layer)
 };
 
 struct UmmaArgs {
@@ -53,6 +55,7 @@ struct UmmaArgs {
   int q_rows;     // rows of the Q tile in shared memory: 128 or 256
   int r_pad;      // W * G rounded up to 16
   int n_stages;   // K ring depth
+  int r0;         // first request of this launch: request r uses maps q[r - r0], k[r - r0]
 };
 
 struct Small {
@@ -125,15 +128,6 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3, int c4) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], "
-      "[%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-      : "memory");
-}
-
 // Shared-memory matrix descriptor of a K-major bf16 tile with the 128-byte swizzle: rows of
 // 128 bytes, groups of 8 rows 1024 bytes apart. `saddr` may point 32 * k bytes into the
 // first row to select the k-th slice of 16 elements along K.
@@ -429,7 +423,7 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
           const uint32_t bar = smem_u32(&sm->q_full);
           mbar_expect_tx(bar, static_cast<uint32_t>(R) * D * 2);
           for (int kb = 0; kb < KB; ++kb)
-            tma_load_5d(smem_u32(q_s + kb * q_blk), &tm.q, bar, kb * 64, U.h * G, 0, U.l, U.r);
+            tma_load_4d(smem_u32(q_s + kb * q_blk), &tm.q[U.r - a.r0], bar, kb * 64, U.h * G, 0, U.l);
           prev_u = U.u;
           ++heads;
         }
@@ -439,7 +433,7 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
           const uint32_t bar = smem_u32(&sm->k_full[s]);
           mbar_expect_tx(bar, kKStage);
           for (int kb = 0; kb < KB; ++kb)
-            tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r], bar, kb * 64, U.kt0 + t * kTileKeys, U.h,
+            tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r - a.r0], bar, kb * 64, U.kt0 + t * kTileKeys, U.h,
                         U.l);
           if (++s == S) {
             s = 0;
@@ -711,45 +705,13 @@ bool score_umma_takes(const Shape& sh) {
   return room >= 2 * stage;
 }
 
-cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, int n_units1,
-                              const ScoreUnit* units2, int n_units2, const void* q, const void* k, float* scores,
-                              float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln) {
+cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
+                              const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
+                              float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln) {
   if (!score_umma_takes(sh) || slab_keys % kTileKeys) return cudaErrorNotSupported;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
   const int R = sh.window * sh.group, d = sh.head_dim;
-
-  TmapPack tm;
-  memset(&tm, 0, sizeof(tm));
-  {
-    const cuuint64_t dims[5] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(sh.n_q_heads),
-                                static_cast<cuuint64_t>(sh.window), static_cast<cuuint64_t>(sh.n_layers),
-                                static_cast<cuuint64_t>(sh.n_req)};
-    const int64_t es[4] = {sh.q_stride_head, sh.q_stride_tok, sh.q_stride_layer,
-                           sh.n_req > 1 ? h_reqs[1].q_offset - h_reqs[0].q_offset : 0};
-    cuuint64_t strides[4];
-    if (!fill_strides(5, dims, es, strides)) return cudaErrorNotSupported;
-    const cuuint32_t box[5] = {64u, static_cast<cuuint32_t>(sh.group), static_cast<cuuint32_t>(sh.window), 1u, 1u};
-    const cuuint32_t ones[5] = {1u, 1u, 1u, 1u, 1u};
-    if (enc(&tm.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q), dims, strides, box, ones,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaErrorNotSupported;
-  }
-  for (int r = 0; r < sh.n_req; ++r) {
-    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(h_reqs[r].L),
-                                static_cast<cuuint64_t>(sh.n_kv_heads), static_cast<cuuint64_t>(sh.n_layers)};
-    const int64_t es[3] = {sh.kv_stride_tok, sh.kv_stride_head, sh.kv_stride_layer};
-    cuuint64_t strides[3];
-    if (!fill_strides(4, dims, es, strides)) return cudaErrorNotSupported;
-    const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(kTileKeys), 1u, 1u};
-    const cuuint32_t ones[4] = {1u, 1u, 1u, 1u};
-    void* base = const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(k) + h_reqs[r].kv_offset);
-    if (enc(&tm.k[r], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, ones,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaErrorNotSupported;
-  }
 
   UmmaArgs args{};
   args.sh = sh;
@@ -770,23 +732,66 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
 
-#define AKV_SWEEP(SW, DD, UNITS)                                                           \
-  args.n_units = (UNITS);                                                                  \
-  args.units = SW == 1 ? units1 : units2;                                                  \
-  e = launch_sweep<SW, DD>(tm, args, (UNITS) < n_sm ? (UNITS) : n_sm, smem, ln.stream);     \
-  if (e != cudaSuccess) return e;                                                          \
+  // Tensor maps are kernel arguments, kMapChunk requests' worth per launch: a longer batch takes both sweeps chunk
+  // by chunk. Sweep 1 lists the units by ascending request, sweep 2 by descending request, so a chunk of requests
+  // is one contiguous run of either list.
+  const int n_units2 = unit_pre2[sh.n_req];
+  for (int r0 = 0; r0 < sh.n_req; r0 += kMapChunk) {
+    const int r1 = r0 + kMapChunk < sh.n_req ? r0 + kMapChunk : sh.n_req;
+    TmapPack tm;
+    memset(&tm, 0, sizeof(tm));
+    for (int r = r0; r < r1; ++r) {
+      {
+        const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(sh.n_q_heads),
+                                    static_cast<cuuint64_t>(sh.window), static_cast<cuuint64_t>(sh.n_layers)};
+        const int64_t es[3] = {sh.q_stride_head, sh.q_stride_tok, sh.q_stride_layer};
+        cuuint64_t strides[3];
+        if (!fill_strides(4, dims, es, strides)) return cudaErrorNotSupported;
+        const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(sh.group), static_cast<cuuint32_t>(sh.window), 1u};
+        const cuuint32_t ones[4] = {1u, 1u, 1u, 1u};
+        void* base = const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(q) + h_reqs[r].q_offset);
+        if (enc(&tm.q[r - r0], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, ones,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+          return cudaErrorNotSupported;
+      }
+      const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(h_reqs[r].L),
+                                  static_cast<cuuint64_t>(sh.n_kv_heads), static_cast<cuuint64_t>(sh.n_layers)};
+      const int64_t es[3] = {sh.kv_stride_tok, sh.kv_stride_head, sh.kv_stride_layer};
+      cuuint64_t strides[3];
+      if (!fill_strides(4, dims, es, strides)) return cudaErrorNotSupported;
+      const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(kTileKeys), 1u, 1u};
+      const cuuint32_t ones[4] = {1u, 1u, 1u, 1u};
+      void* base = const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(k) + h_reqs[r].kv_offset);
+      if (enc(&tm.k[r - r0], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, ones,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorNotSupported;
+    }
+    args.r0 = r0;
+    const ScoreUnit* u1 = units1 + unit_pre1[r0];
+    const int n1 = unit_pre1[r1] - unit_pre1[r0];
+    const ScoreUnit* u2 = units2 + (n_units2 - unit_pre2[r1]);
+    const int n2 = unit_pre2[r1] - unit_pre2[r0];
+
+#define AKV_SWEEP(SW, DD, UNITS, N)                                                  \
+  args.n_units = (N);                                                                \
+  args.units = (UNITS);                                                              \
+  e = launch_sweep<SW, DD>(tm, args, (N) < n_sm ? (N) : n_sm, smem, ln.stream);      \
+  if (e != cudaSuccess) return e;                                                    \
   ln.done(SW == 1 ? "score_umma_stats" : "score_umma_colsum")
-  if (d == 64) {
-    AKV_SWEEP(1, 64, n_units1);
-    AKV_SWEEP(2, 64, n_units2);
-  } else if (d == 128) {
-    AKV_SWEEP(1, 128, n_units1);
-    AKV_SWEEP(2, 128, n_units2);
-  } else {
-    AKV_SWEEP(1, 256, n_units1);
-    AKV_SWEEP(2, 256, n_units2);
-  }
+    if (d == 64) {
+      AKV_SWEEP(1, 64, u1, n1);
+      AKV_SWEEP(2, 64, u2, n2);
+    } else if (d == 128) {
+      AKV_SWEEP(1, 128, u1, n1);
+      AKV_SWEEP(2, 128, u2, n2);
+    } else {
+      AKV_SWEEP(1, 256, u1, n1);
+      AKV_SWEEP(2, 256, u2, n2);
+    }
 #undef AKV_SWEEP
+  }
   return cudaSuccess;
 }
 

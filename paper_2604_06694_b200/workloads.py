@@ -201,3 +201,72 @@ def attention_rows(n_steps: int, n_heads: int, n_audio: int, n_text0: int = 16, 
         p = np.exp(z)
         attn[t, :, :L] = (p / p.sum(axis=1, keepdims=True)).astype(np.float32)
     return attn, row_len, span, g
+
+
+@dataclasses.dataclass
+class CompactedCache:
+    """A cache that has been evicted once and has decoded `n_new` tokens since: per-head ragged rows."""
+    spec: WorkloadSpec
+    q: np.ndarray            # raw storage [n_req][n_layers][W][n_q_heads][d]: queries of the last W decoded tokens
+    k: np.ndarray            # raw storage [rows][d], head u = (r * n_layers + l) * n_kv_heads + h at rows cu[u]..cu[u+1]
+    v: np.ndarray
+    cu: np.ndarray           # int32 [total heads + 1]
+    new_budgets: np.ndarray  # int32 [total heads]: rows each head keeps after the re-eviction (window included)
+
+    def q_strides(self):
+        s = self.spec
+        per_tok = s.n_q_heads * s.head_dim
+        return (s.n_layers * s.window * per_tok, s.window * per_tok, per_tok, s.head_dim)
+
+    def torch_dtype(self):
+        return torch.float32 if self.spec.dtype == "f32" else torch.bfloat16
+
+    def as_torch(self, a: np.ndarray) -> torch.Tensor:
+        t = torch.from_numpy(a)
+        return t if self.spec.dtype == "f32" or a.dtype != np.uint16 else t.view(torch.bfloat16)
+
+
+def compacted_cache(spec: WorkloadSpec, n_new: int, seed: int = 0, layers: Optional[int] = None,
+                    spread: float = 0.5) -> CompactedCache:
+    """Each head of each request kept b_u rows at prefill, b_u drawn uniformly within +-spread of the request's
+    mean budget (never below W + 1 nor above L), and has appended `n_new` decoded rows; the re-eviction brings it
+    back to b_u. Kept rows are AR(1) like the audio keys of `generate`, decoded rows are white."""
+    if layers is not None:
+        spec = dataclasses.replace(spec, n_layers=int(layers))
+    NL, Hq, Hkv, d, W = spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.window
+    G = Hq // Hkv
+    lens = list(spec.seq_lens)
+    st = np.uint16 if spec.dtype == "bf16" else np.float32
+    TH = len(lens) * NL * Hkv
+    rng_b = np.random.Generator(np.random.Philox(key=[seed, 77]))
+    cu = np.zeros(TH + 1, dtype=np.int64)
+    budgets = np.zeros(TH, dtype=np.int32)
+    u = 0
+    for L in lens:
+        mean = kept_total(spec, L) / (NL * Hkv)
+        for _ in range(NL * Hkv):
+            b = int(round(mean * (1.0 + spread * (2.0 * rng_b.random() - 1.0))))
+            budgets[u] = min(max(b, W + 1), L)
+            cu[u + 1] = cu[u] + budgets[u] + n_new
+            u += 1
+    rows = int(cu[-1])
+    k = np.zeros((rows, d), dtype=st)
+    v = np.zeros((rows, d), dtype=st)
+    q = np.zeros((len(lens), NL, W, Hq, d), dtype=st)
+    u = 0
+    for r in range(len(lens)):
+        for l in range(NL):
+            rng = np.random.Generator(np.random.Philox(key=[seed, (r << 20) + l + 1 + (1 << 40)]))
+            for h in range(Hkv):
+                n_old = int(budgets[u])
+                rho = spec.ar_rho if spec.ar_rho_range is None else float(rng.uniform(*spec.ar_rho_range))
+                for dst, is_k in ((k, True), (v, False)):
+                    x = rng.standard_normal(size=(n_old + n_new, d), dtype=np.float32)
+                    _ar1_inplace(x[:n_old], rho)
+                    if is_k and spec.n_sink:
+                        x[: spec.n_sink] *= 8.0
+                    dst[cu[u]:cu[u + 1]] = _store(x, spec.dtype)
+                xq = rng.standard_normal(size=(W, G * d), dtype=np.float32)
+                q[r, l, :, h * G:(h + 1) * G, :] = _store(xq, spec.dtype).reshape(W, G, d)
+                u += 1
+    return CompactedCache(spec, q, k, v, cu.astype(np.int32), budgets)

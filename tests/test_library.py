@@ -59,6 +59,32 @@ def test_sizes_and_param_checks(B):
     assert B.audiokv_strerror(B.AUDIOKV_EWORKSPACE) == "workspace too small"
 
 
+def test_many_requests_and_query_offsets(B):
+    """Batches beyond the 64 requests one launch carries are planned (no GPU work here), and a misaligned or
+    negative per-request query offset is refused."""
+    n = 300
+    lens = [200 + 7 * i for i in range(n)]
+    cu = [0]
+    for L in lens:
+        cu.append(cu[-1] + L)
+    p = _prob(B, seq_lens=lens, kv_strides=(2 * cu[-1] * 128, 128, cu[-1] * 128),
+              kv_req_offset=[c * 128 for c in cu[:-1]])
+    assert B.audiokv_scores_len(p) == 4 * sum(L - 32 for L in lens)
+    assert B.audiokv_workspace_bytes(p) > 0
+    ok = _prob(B, q_req_offset=[64, 0])
+    assert B.audiokv_workspace_bytes(ok) > 0
+    assert B.audiokv_scores_len(_prob(B, q_req_offset=[4, 0])) == B.AUDIOKV_EALIGN
+    assert B.audiokv_scores_len(_prob(B, q_req_offset=[0, -8])) == B.AUDIOKV_EINVAL
+
+
+def test_reevict_workspace_and_checks(B):
+    p = _prob(B)                               # 2 requests x 2 layers x 2 KV heads = 8 heads
+    cu = [0, 300, 700, 1000, 1500, 1900, 2000, 2600, 3000]
+    assert B.audiokv_reevict_workspace_bytes(p, cu) > 0
+    assert B.audiokv_reevict_workspace_bytes(p, [1] + cu[1:]) == 0          # must start at 0
+    assert B.audiokv_reevict_workspace_bytes(p, cu[:5] + [1510] + cu[6:]) == 0   # a head no longer than the window
+
+
 def test_binding_refuses_cpu_tensors(B):
     import torch
     with pytest.raises(ValueError):
