@@ -164,3 +164,22 @@ def test_q_req_offset_matches_stride(B):
     torch.cuda.synchronize()
     assert ctx.last_device_status() == 0
     assert torch.equal(ref, got)
+
+
+def test_reevict_full_size_sampled_heads(B):
+    """The 7B shape at L = 8192 after one eviction and 128 decoded tokens: 112 heads of 1.8k to 5k rows (two launches
+    of either scoring sweep, one transform plan per distinct length); sampled heads against the oracle, and for
+    every head the properties that hold at any size."""
+    c = wl.compacted_cache(wl.config(1), n_new=128, seed=1)
+    assert len(c.new_budgets) == 112
+    g = run_reevict(B, c)
+    assert check_heads(c, g, heads=[0, 17, 44, 63, 64, 111]) <= 6
+    W = c.spec.window
+    for u in range(112):
+        a, b = g["cu"][u], g["cu"][u + 1]
+        n = int(c.cu[u + 1] - c.cu[u])
+        idx = g["kept"][a:b]
+        assert b - a == c.new_budgets[u]
+        assert (np.diff(idx) > 0).all() and idx[0] >= 0 and np.array_equal(idx[-W:], np.arange(n - W, n))
+        assert np.array_equal(g["k_out"][a:b], c.k[c.cu[u]:c.cu[u + 1]][idx])
+        assert np.array_equal(g["v_out"][a:b], c.v[c.cu[u]:c.cu[u + 1]][idx])
