@@ -44,6 +44,8 @@ def _load():
         lib.akvo_smooth_variant.restype = ctypes.c_int
         lib.akvo_hit_score.argtypes = [vp, i32, i32, ctypes.c_int64, vp, vp, i32, vp, vp]
         lib.akvo_hit_score.restype = ctypes.c_int
+        lib.akvo_selection_spread.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
+        lib.akvo_selection_spread.restype = ctypes.c_int
         lib.akvo_allocate.argtypes = [vp, i32, i64, i32, i32, i32, vp]
         lib.akvo_select.argtypes = [vp, i32, i32, vp]
         lib.akvo_gather.argtypes = [vp, i32, i32, i64, vp, i32, vp]
@@ -153,6 +155,21 @@ def hit_score(attn: np.ndarray, row_len: np.ndarray, span: np.ndarray, K: int = 
     if rc != 0:
         raise ValueError("akvo_hit_score rejected its arguments")
     return s, counts
+
+
+def selection_spread(kept: np.ndarray, cu_kept: np.ndarray, P: int, n_bins: int):
+    """Histogram of one request's kept prefix tokens over n_bins stretches of the prefix, and its two summaries.
+    kept: int32, the heads' indices back to back; cu_kept: int32 [N + 1], relative to kept[0].
+    Returns (hist int64 [n_bins], balance, peak)."""
+    kept = np.ascontiguousarray(kept, dtype=np.int32)
+    cu_kept = np.ascontiguousarray(cu_kept, dtype=np.int32)
+    hist = np.zeros(n_bins, dtype=np.int64)
+    bal, pk = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = _load().akvo_selection_spread(_ptr(kept), _ptr(cu_kept), len(cu_kept) - 1, int(P), int(n_bins), _ptr(hist),
+                                       ctypes.byref(bal), ctypes.byref(pk))
+    if rc != 0:
+        raise ValueError("akvo_selection_spread rejected its arguments")
+    return hist, bal.value, pk.value
 
 
 def allocate(S: np.ndarray, B: int, w: int, r: int, L: int) -> np.ndarray:

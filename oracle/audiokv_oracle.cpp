@@ -387,6 +387,46 @@ int akvo_hit_score(const double* attn, int n_steps, int n_heads, int64_t row_str
 }
 
 // ---------------------------------------------------------------------------
+// Selection spread (Section 1, "Motivation 2" and the figure on the distribution of Top-K selections before and
+// after smoothing): where along the prefix the kept tokens of a request's heads fall. The prefix 0..P-1 is cut into
+// n_bins stretches, token j belonging to bin floor(j * n_bins / P); hist[b] counts, over all N heads, the kept prefix
+// tokens in bin b (window tokens, index >= P, are not counted). Two summaries of the histogram:
+//     balance = -sum_b p_b ln p_b / ln n_bins,  p_b = hist[b] / sum hist   (1 = flat, 0 = one bin; 0 when n_bins = 1)
+//     peak    = max_b hist[b] * n_bins / sum hist                          (busiest bin against the mean bin)
+// Both are 0 when nothing is kept. kept: the heads' kept indices back to back, head u at [cu_kept[u], cu_kept[u+1]).
+int akvo_selection_spread(const int32_t* kept, const int32_t* cu_kept, int N, int P, int n_bins, int64_t* hist,
+                          double* balance, double* peak) {
+  if (N < 1 || P < 1 || n_bins < 1) return -1;
+  for (int b = 0; b < n_bins; ++b) hist[b] = 0;
+  for (int u = 0; u < N; ++u)
+    for (int i = cu_kept[u]; i < cu_kept[u + 1]; ++i) {
+      const int j = kept[i];
+      if (j < 0) return -1;
+      if (j >= P) continue;
+      hist[static_cast<int64_t>(j) * n_bins / P] += 1;
+    }
+  int64_t total = 0, top = 0;
+  for (int b = 0; b < n_bins; ++b) {
+    total += hist[b];
+    top = std::max(top, hist[b]);
+  }
+  *balance = 0.0;
+  *peak = 0.0;
+  if (total == 0) return 0;
+  *peak = static_cast<double>(top) * n_bins / static_cast<double>(total);
+  if (n_bins > 1) {
+    double H = 0.0;
+    for (int b = 0; b < n_bins; ++b)
+      if (hist[b] > 0) {
+        const double p = static_cast<double>(hist[b]) / static_cast<double>(total);
+        H -= p * std::log(p);
+      }
+    *balance = H / std::log(static_cast<double>(n_bins));
+  }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
 // Step 3: head-wise budgets (Section 3.1, the allocation equation
 //   b = w + r + B_score * S / sum S,
 // of which Section 3.2's floor(B * S_hit / sum S_hit) is the case w = r = 0).
