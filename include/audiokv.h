@@ -235,6 +235,20 @@ int audiokv_reevict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win
                     const void* v_cache, const int32_t* cu_cache, const int32_t* new_budgets, void* k_out, void* v_out,
                     int32_t* kept_idx, int32_t* cu_kept, audiokv_stream stream);
 
+/* Selection spread (Section 1, the figure on the distribution of Top-K selections before
+ * and after smoothing): where along the prefix the kept tokens of a request's heads fall.
+ * Token j of request r's prefix belongs to stretch floor(j * n_bins / P_r); hist[r][b]
+ * counts, over the request's n_layers * n_kv_heads heads, the kept prefix tokens in
+ * stretch b (window tokens are not counted). stats[r] = {balance, peak}:
+ *   balance = -sum_b p_b ln p_b / ln n_bins, p_b = hist[r][b] / sum_b hist[r][b]
+ *             (1 = flat, 0 = one stretch; 0 when n_bins = 1),
+ *   peak    = max_b hist[r][b] * n_bins / sum_b hist[r][b];  both 0 when nothing is kept.
+ * kept_idx, cu_kept: device, as audiokv_evict / audiokv_select_gather wrote them.
+ * n_bins: 1..4096. hist: device int32 [n_req][n_bins]; stats: device fp32 [n_req][2]. */
+int audiokv_selection_spread(audiokv_ctx* ctx, const audiokv_params* p, const int32_t* kept_idx,
+                             const int32_t* cu_kept, int32_t n_bins, int32_t* hist, float* stats,
+                             audiokv_stream stream);
+
 /* Offline head score (Section 3.2, "Collecting Attention Hits to Audio Spans" and "Head Importance
  * Estimation"): the table S that audiokv_allocate consumes. For decode step t and head a, with
  * S = TopK(attention row, top_k) (ties: lower token index) and the inclusive audio-token span

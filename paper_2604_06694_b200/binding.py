@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.audiokv_reevict_workspace_bytes.argtypes = [pp, ctypes.POINTER(i32)]
         L.audiokv_reevict.argtypes = [vp, pp, vp, vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), vp, vp, vp, vp, vp]
         L.audiokv_reevict.restype = ctypes.c_int
+        L.audiokv_selection_spread.argtypes = [vp, pp, vp, vp, i32, vp, vp, vp]
+        L.audiokv_selection_spread.restype = ctypes.c_int
         L.audiokv_hit_score.argtypes = [vp, vp, i32, i32, i64, vp, vp, i32, vp, vp, vp]
         L.audiokv_hit_score.restype = ctypes.c_int
         L.audiokv_evict_host.argtypes = [vp, pp, vp, i64, vp, vp, i64, vp, ctypes.POINTER(i64), vp, vp, vp, vp, vp, vp]
@@ -296,6 +298,13 @@ def audiokv_reevict(ctx: Context, prob: Problem, q_win, k_cache, v_cache, cu_cac
                                      _dev(v_cache, "v_cache"), _i32_array(cu_cache), _i32_array(new_budgets),
                                      _dev(k_out, "k_out"), _dev(v_out, "v_out"), _dev(kept_idx, "kept_idx"),
                                      _dev(cu_kept, "cu_kept"), _stream()), "audiokv_reevict")
+
+
+def audiokv_selection_spread(ctx: Context, prob: Problem, kept_idx, cu_kept, n_bins: int, hist, stats) -> None:
+    """hist: CUDA int32 [n_req][n_bins]; stats: CUDA fp32 [n_req][2] (balance, peak)."""
+    ctx._check(lib().audiokv_selection_spread(ctx.h, prob.ref, _dev(kept_idx, "kept_idx"), _dev(cu_kept, "cu_kept"),
+                                              n_bins, _dev(hist, "hist"), _dev(stats, "stats"), _stream()),
+               "audiokv_selection_spread")
 
 
 def audiokv_hit_score(ctx: Context, attn: torch.Tensor, row_len: torch.Tensor, span: torch.Tensor, top_k: int,

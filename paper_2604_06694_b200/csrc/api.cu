@@ -821,6 +821,20 @@ int audiokv_hit_score(audiokv_ctx* ctx, const float* attn, int32_t n_steps, int3
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 
+int audiokv_selection_spread(audiokv_ctx* ctx, const audiokv_params* p, const int32_t* kept_idx,
+                             const int32_t* cu_kept, int32_t n_bins, int32_t* hist, float* stats,
+                             audiokv_stream stream) {
+  if (!kept_idx || !cu_kept || !hist || !stats) return AUDIOKV_EINVAL;
+  if (n_bins < 1 || n_bins > 4096) return AUDIOKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(ctx, p, s);
+  if (rc) return rc;
+  Launch ln{s, &ctx->launches, &ctx->prof};
+  cudaError_t e = launch_selection_spread(ctx->plan.sh, d_reqs(ctx), kept_idx, cu_kept, n_bins, hist, stats,
+                                          d_status(ctx), ln);
+  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
+}
+
 int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, int64_t q_elems, const void* k,
                        const void* v, int64_t kv_elems, const float* head_scores, const int64_t* total_budget,
                        void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* cu_kept,

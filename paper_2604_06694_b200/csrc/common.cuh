@@ -169,4 +169,10 @@ cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t*
 cudaError_t launch_hit_score(const float* attn, int n_steps, int n_heads, int64_t row_stride, const int32_t* row_len,
                              const int32_t* span, int top_k, int32_t* counts, float* s_hit, int* status, Launch ln);
 
+// spread.cu: histogram of the kept prefix tokens over n_bins stretches of each request's prefix (hist int32
+// [n_req][n_bins], cleared here) and its summaries (stats fp32 [n_req][2]: balance, peak).
+cudaError_t launch_selection_spread(const Shape& sh, const ReqDesc* d_reqs, const int32_t* kept_idx,
+                                    const int32_t* cu_kept, int n_bins, int32_t* hist, float* stats, int* status,
+                                    Launch ln);
+
 }  // namespace akv
