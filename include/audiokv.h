@@ -93,6 +93,15 @@ typedef struct {
   int32_t pool_kernel;           /* AUDIOKV_SMOOTH_*_POOL: odd window, 1 .. 1023 tokens          */
   const int64_t* q_req_offset;   /* host [n_req], or NULL: element offset of request r's window queries,
                                     replacing r*q_stride_req (which is then ignored)              */
+  /* Paged K/V (page_size = 0: off). K and V are then pools of n_pages pages of page_size tokens, and
+   * K/V(r,l,h,j,t) = l*kv_stride_layer + h*kv_stride_head + (page_table[r][j / page_size]*page_size
+   * + j % page_size)*kv_stride_tok + t; kv_req_offset is ignored. Tokens of a page beyond L_r may hold
+   * anything. A page id outside [0, n_pages) is not followed: AUDIOKV_EDEVICE in the status word.   */
+  int32_t page_size;             /* 0, 16, 32, 64 or 128 tokens                                  */
+  int32_t n_pages;               /* pages in the pool                                            */
+  const int32_t* page_table;     /* DEVICE int32 [n_req][page_table_stride], read when the kernels run;
+                                    request r uses its first ceil(L_r / page_size) entries        */
+  int64_t page_table_stride;     /* >= ceil(max L / page_size)                                   */
 } audiokv_params;
 
 #define AUDIOKV_MAX_REQ 8192

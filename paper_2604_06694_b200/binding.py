@@ -43,6 +43,8 @@ class audiokv_params(ctypes.Structure):
         ("transition_bins", ctypes.c_int32), ("base_per_head", ctypes.c_int32),
         ("smooth_mode", ctypes.c_int32), ("smooth_kappa", ctypes.c_float), ("pool_kernel", ctypes.c_int32),
         ("q_req_offset", ctypes.POINTER(ctypes.c_int64)),
+        ("page_size", ctypes.c_int32), ("n_pages", ctypes.c_int32), ("page_table", ctypes.c_void_p),
+        ("page_table_stride", ctypes.c_int64),
     ]
 
 
@@ -115,7 +117,8 @@ class Problem:
                  seq_lens: Sequence[int], window: int, q_strides: Sequence[int], kv_strides: Sequence[int],
                  kv_req_offset: Optional[Sequence[int]] = None, softmax_scale: float = 0.0, rho: float = 0.5,
                  alpha: float = 0.5, transition_bins: int = 4, base_per_head: int = 0, smooth_mode: int = 0,
-                 smooth_kappa: float = 0.0, pool_kernel: int = 1, q_req_offset: Optional[Sequence[int]] = None):
+                 smooth_kappa: float = 0.0, pool_kernel: int = 1, q_req_offset: Optional[Sequence[int]] = None,
+                 page_size: int = 0, n_pages: int = 0, page_table: Optional[torch.Tensor] = None):
         n = len(seq_lens)
         self._qoff = (ctypes.c_int64 * n)(*[int(x) for x in q_req_offset]) if q_req_offset is not None else None
         self._seq = (ctypes.c_int32 * n)(*[int(x) for x in seq_lens])
@@ -131,6 +134,14 @@ class Problem:
         p.transition_bins, p.base_per_head = transition_bins, base_per_head
         p.smooth_mode, p.smooth_kappa, p.pool_kernel = smooth_mode, smooth_kappa, pool_kernel
         p.q_req_offset = ctypes.cast(self._qoff, ctypes.POINTER(ctypes.c_int64)) if self._qoff is not None else None
+        if page_size:
+            # page_table: CUDA int32 [n_req][stride], kept alive here; the kv strides then describe the pool
+            if page_table is None or not page_table.is_cuda or page_table.dtype != torch.int32 or page_table.dim() != 2 \
+                    or not page_table.is_contiguous():
+                raise ValueError("page_table must be a contiguous CUDA int32 tensor [n_req][stride]")
+            self._page_table = page_table
+            p.page_size, p.n_pages = page_size, n_pages
+            p.page_table, p.page_table_stride = page_table.data_ptr(), page_table.shape[1]
         self.p = p
         self.seq_lens = [int(x) for x in seq_lens]
 

@@ -99,6 +99,13 @@ int check_params(const audiokv_params* p) {
     if (s < 0) return AUDIOKV_EINVAL;
     if (s % per16) return AUDIOKV_EALIGN;
   }
+  if (p->page_size != 0) {
+    if (p->page_size != 16 && p->page_size != 32 && p->page_size != 64 && p->page_size != 128) return AUDIOKV_EUNSUPPORTED;
+    if (p->n_pages < 1 || !p->page_table || p->kv_stride_tok < 1) return AUDIOKV_EINVAL;
+    if (static_cast<int64_t>(p->n_pages) * p->page_size > 0x7fffffffLL) return AUDIOKV_EUNSUPPORTED;
+    for (int r = 0; r < p->n_req; ++r)
+      if ((p->seq_len[r] + p->page_size - 1) / p->page_size > p->page_table_stride) return AUDIOKV_EINVAL;
+  }
   for (int r = 0; r < p->n_req; ++r) {
     if (p->kv_req_offset && p->kv_req_offset[r] % per16) return AUDIOKV_EALIGN;
     if (p->q_req_offset && p->q_req_offset[r] % per16) return AUDIOKV_EALIGN;
@@ -118,7 +125,8 @@ bool same_plan(const Plan& pl, const audiokv_params* p) {
       a.kv_stride_layer != p->kv_stride_layer || a.kv_stride_tok != p->kv_stride_tok ||
       a.kv_stride_head != p->kv_stride_head || a.softmax_scale != p->softmax_scale || a.rho != p->rho ||
       a.alpha != p->alpha || a.transition_bins != p->transition_bins || a.base_per_head != p->base_per_head ||
-      a.smooth_mode != p->smooth_mode || a.smooth_kappa != p->smooth_kappa || a.pool_kernel != p->pool_kernel)
+      a.smooth_mode != p->smooth_mode || a.smooth_kappa != p->smooth_kappa || a.pool_kernel != p->pool_kernel ||
+      a.page_size != p->page_size || a.n_pages != p->n_pages || a.page_table_stride != p->page_table_stride)
     return false;
   for (int r = 0; r < p->n_req; ++r) {
     if (pl.seq_len[r] != p->seq_len[r]) return false;
@@ -228,6 +236,7 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   pl->p.seq_len = nullptr;
   pl->p.kv_req_offset = nullptr;
   pl->p.q_req_offset = nullptr;
+  pl->p.page_table = nullptr;
 
   Shape& sh = pl->sh;
   sh.dtype = p->dtype;
@@ -255,6 +264,13 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   sh.smooth_mode = p->smooth_mode;
   sh.smooth_kappa = p->smooth_kappa;
   sh.pool_kernel = p->pool_kernel;
+  sh.page_size = p->page_size;
+  sh.page_shift = 0;
+  while (p->page_size && (1 << sh.page_shift) < p->page_size) ++sh.page_shift;
+  sh.n_pages = p->n_pages;
+  sh.page_table_stride = p->page_table_stride;
+  sh.page_table = nullptr;  // set per call, with the status word
+  sh.page_status = nullptr;
 
   pl->reqs.assign(p->n_req, ReqDesc{});
   pl->fft.clear();
@@ -395,6 +411,8 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
   }
   Plan& pl = ctx->plan;
   if (pl.lay.end > ctx->ws_bytes) return AUDIOKV_EWORKSPACE;
+  pl.sh.page_table = p->page_size ? p->page_table : nullptr;  // device data of this call, not part of the plan
+  pl.sh.page_status = reinterpret_cast<int*>(ctx->ws + pl.lay.status);
   if (!ctx->plan_uploaded) {
     // earlier calls on other streams may still read the old tables
     if ((e = cudaStreamWaitEvent(stream, ctx->plan_ready, 0)) != cudaSuccess) return cuda_fail(ctx, e);
@@ -773,6 +791,10 @@ int reevict_problem(audiokv_ctx* ctx, const audiokv_params* p, const int32_t* cu
   dp->kv_req_offset = ctx->re_kv_off.data();
   dp->q_req_offset = ctx->re_q_off.data();
   dp->base_per_head = 0;
+  dp->page_size = 0;  // the compacted cache is packed, not paged
+  dp->n_pages = 0;
+  dp->page_table = nullptr;
+  dp->page_table_stride = 0;
   return AUDIOKV_OK;
 }
 
@@ -841,6 +863,7 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
                        audiokv_stream stream) {
   if (!q_win || !k || !v || !head_scores || !total_budget || !k_out || !v_out || !kept_idx || !budgets || !cu_kept)
     return AUDIOKV_EINVAL;
+  if (p && p->page_size != 0) return AUDIOKV_EUNSUPPORTED;  // a page table is device data: use audiokv_evict
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int rc = prepare(ctx, p, s);
   if (rc) return rc;

@@ -33,7 +33,24 @@ struct Shape {
   int32_t transition_bins, base_per_head;
   int32_t smooth_mode, pool_kernel;  // AUDIOKV_SMOOTH_*; window of the pooling modes
   float smooth_kappa;                // cut-off fraction of AUDIOKV_SMOOTH_FIXED_FRACTION
+  // paged K / V: page_size 0 = contiguous; page_shift = log2(page_size)
+  int32_t page_size, page_shift, n_pages;
+  int64_t page_table_stride;
+  const int32_t* page_table;  // device [n_req][page_table_stride]
+  int* page_status;           // status word that a page id outside the pool is reported to (may be null)
 };
+
+// Element offset of token j of request r inside K / V, without the layer and head terms. A page id outside the pool
+// is reported through the status word and read as page 0, so that no address leaves the pool.
+__device__ __forceinline__ int64_t kv_token_offset(const Shape& sh, const ReqDesc& rq, int r, int j) {
+  if (sh.page_size == 0) return rq.kv_offset + static_cast<int64_t>(j) * sh.kv_stride_tok;
+  int page = __ldg(sh.page_table + r * sh.page_table_stride + (j >> sh.page_shift));
+  if (page < 0 || page >= sh.n_pages) {
+    if (sh.page_status) atomicExch(sh.page_status, AUDIOKV_EDEVICE);
+    page = 0;
+  }
+  return ((static_cast<int64_t>(page) << sh.page_shift) + (j & (sh.page_size - 1))) * sh.kv_stride_tok;
+}
 
 // Maps a flat head index to (request, layer, kv head). n_req is small: linear search.
 __device__ __forceinline__ int find_req(const ReqDesc* __restrict__ reqs, int n_req, int heads_per_req, int u) {

@@ -102,7 +102,7 @@ __global__ void __launch_bounds__(kThreads) score_simt_kernel(Shape sh, const Re
   const int j1 = min(j_end, j0 + slab_keys);
   float2* my_stats = stats + (static_cast<int64_t>(u) * n_slab + slab) * R;
 
-  const T* kbase = k + rq.kv_offset + hc.l * sh.kv_stride_layer + hc.h * sh.kv_stride_head;
+  const T* kbase = k + hc.l * sh.kv_stride_layer + hc.h * sh.kv_stride_head;  // the token term: kv_token_offset
   const T* qbase = q + rq.q_offset + hc.l * sh.q_stride_layer + static_cast<int64_t>(hc.h) * G * sh.q_stride_head;
 
   if (SWEEP == 1) {
@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(kThreads) score_simt_kernel(Shape sh, const Re
 
   for (int kt = j0; kt < j1; kt += kTile) {
     const int nk = min(kTile, j1 - kt);
-    stage_rows<T, D>(Ks, nk, [&](int row) { return kbase + static_cast<int64_t>(kt + row) * sh.kv_stride_tok; });
+    stage_rows<T, D>(Ks, nk, [&](int row) { return kbase + kv_token_offset(sh, rq, hc.r, kt + row); });
     float colsum = 0.f;  // sweep 2, threads 0..63
     for (int rc = 0; rc < R; rc += kTile) {
       const int nr = min(kTile, R - rc);
@@ -289,6 +289,7 @@ extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const 
   constexpr int kNoAllocMaxReq = 64;  // the request table has a fixed slot in the static scratch
   if (p->n_req < 1 || p->n_req > kNoAllocMaxReq || p->window < 1) return AUDIOKV_EINVAL;
   if (p->head_dim != 64 && p->head_dim != 128 && p->head_dim != 256) return AUDIOKV_EUNSUPPORTED;
+  if (p->page_size != 0) return AUDIOKV_EUNSUPPORTED;  // contiguous K only
   const int G = p->n_q_heads / p->n_kv_heads;
   const int64_t R = static_cast<int64_t>(p->window) * G;
   if (R > 1024) return AUDIOKV_EUNSUPPORTED;

@@ -432,9 +432,35 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
           if (!ok) break;
           const uint32_t bar = smem_u32(&sm->k_full[s]);
           mbar_expect_tx(bar, kKStage);
-          for (int kb = 0; kb < KB; ++kb)
-            tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r - a.r0], bar, kb * 64, U.kt0 + t * kTileKeys, U.h,
-                        U.l);
+          if (a.sh.page_size == 0) {
+            for (int kb = 0; kb < KB; ++kb)
+              tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r - a.r0], bar, kb * 64,
+                          U.kt0 + t * kTileKeys, U.h, U.l);
+          } else {
+            // Paged pool: k[0] maps the whole pool as (d, page * page_size + token in page, KV head, layer) with a box
+            // of one page; the tile is filled page by page (page_size >= 16 rows of 128 bytes: whole swizzle groups).
+            // Pages past the request's last token start outside the map and arrive as zeros; so does a page id
+            // outside the pool, which is also reported.
+            const int ps = a.sh.page_size, n_sub = kTileKeys >> a.sh.page_shift, L = U.P + a.sh.window;
+            const int32_t* tab = a.sh.page_table + U.r * a.sh.page_table_stride;
+            const int tok0 = U.kt0 + t * kTileKeys;
+            int y[kTileKeys / 16];
+#pragma unroll
+            for (int i = 0; i < kTileKeys / 16; ++i) {
+              y[i] = a.sh.n_pages << a.sh.page_shift;
+              if (i < n_sub && tok0 + i * ps < L) {
+                const int pg = __ldg(tab + ((tok0 + i * ps) >> a.sh.page_shift));
+                if (pg >= 0 && pg < a.sh.n_pages) y[i] = pg << a.sh.page_shift;
+                else atomicExch(a.status, AUDIOKV_EDEVICE);
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < kTileKeys / 16; ++i)
+              if (i < n_sub)
+                for (int kb = 0; kb < KB; ++kb)
+                  tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk + i * ps * 128), &tm.k[0], bar, kb * 64, y[i],
+                              U.h, U.l);
+          }
           if (++s == S) {
             s = 0;
             ph ^= 1;
@@ -755,14 +781,18 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
           return cudaErrorNotSupported;
       }
-      const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(h_reqs[r].L),
+      if (sh.page_size != 0 && r > r0) continue;  // one map of the whole pool serves every request
+      const bool paged = sh.page_size != 0;
+      const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d),
+                                  paged ? static_cast<cuuint64_t>(sh.n_pages) * sh.page_size
+                                        : static_cast<cuuint64_t>(h_reqs[r].L),
                                   static_cast<cuuint64_t>(sh.n_kv_heads), static_cast<cuuint64_t>(sh.n_layers)};
       const int64_t es[3] = {sh.kv_stride_tok, sh.kv_stride_head, sh.kv_stride_layer};
       cuuint64_t strides[3];
       if (!fill_strides(4, dims, es, strides)) return cudaErrorNotSupported;
-      const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(kTileKeys), 1u, 1u};
+      const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(paged ? sh.page_size : kTileKeys), 1u, 1u};
       const cuuint32_t ones[4] = {1u, 1u, 1u, 1u};
-      void* base = const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(k) + h_reqs[r].kv_offset);
+      void* base = const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(k) + (paged ? 0 : h_reqs[r].kv_offset));
       if (enc(&tm.k[r - r0], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, ones,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)

@@ -68,7 +68,8 @@ gather_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const int32_t* __restr
       const int lh = u - rq.head_base;
       const int l = lh / sh.n_kv_heads, h = lh - l * sh.n_kv_heads;
       const int tok = __ldg(kept_idx + row);
-      my_src = (rq.kv_offset + l * sh.kv_stride_layer + h * sh.kv_stride_head + tok * sh.kv_stride_tok) / elems_per_chunk;
+      my_src = (l * sh.kv_stride_layer + h * sh.kv_stride_head + kv_token_offset(sh, rq, u / sh.heads_per_req, tok)) /
+               elems_per_chunk;
     }
     const int n_rows = static_cast<int>(min(static_cast<int64_t>(kGatherRows), total_rows - row0));
     int64_t so[kGatherRows];  // every lane gets the eight source rows (all lanes take part in the shuffles)

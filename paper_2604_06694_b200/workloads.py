@@ -270,3 +270,38 @@ def compacted_cache(spec: WorkloadSpec, n_new: int, seed: int = 0, layers: Optio
                 q[r, l, :, h * G:(h + 1) * G, :] = _store(xq, spec.dtype).reshape(W, G, d)
                 u += 1
     return CompactedCache(spec, q, k, v, cu.astype(np.int32), budgets)
+
+
+def paged_pool(w: Workload, page_size: int, seed: int = 0, spare: int = 3):
+    """The K and V of `w` scattered into pools of pages, the way a serving stack's block allocator holds them.
+
+    Returns (k_pool, v_pool, page_table, n_pages, kv_strides): pools are raw storage [n_layers][n_pages * page_size]
+    [n_kv_heads][d] (token-major inside a page), page_table is int32 [n_req][max pages of a request] with -1 in unused
+    slots, pages are handed out in a random order, `spare` pages belong to nobody, and every pool slot that holds no
+    token (page tails, spare pages) is filled with NaN, which a correct reader never lets through.
+    kv_strides = (layer, token, head) strides of the pools in elements."""
+    s = w.spec
+    NL, Hkv, d = s.n_layers, s.n_kv_heads, s.head_dim
+    lens = list(s.seq_lens)
+    per_req = [(L + page_size - 1) // page_size for L in lens]
+    n_pages = sum(per_req) + spare
+    rng = np.random.Generator(np.random.Philox(key=[seed, 4242]))
+    order = rng.permutation(n_pages)
+    table = np.full((len(lens), max(per_req)), -1, dtype=np.int32)
+    nan = np.uint16(0x7FC0) if w.k.dtype == np.uint16 else np.float32(np.nan)
+    k_pool = np.full((NL, n_pages * page_size, Hkv, d), nan, dtype=w.k.dtype)
+    v_pool = np.full((NL, n_pages * page_size, Hkv, d), nan, dtype=w.v.dtype)
+    nxt = 0
+    for r, L in enumerate(lens):
+        base = int(w.cu_seqlen[r])
+        for i in range(per_req[r]):
+            pg = int(order[nxt])
+            nxt += 1
+            table[r, i] = pg
+            n = min(page_size, L - i * page_size)
+            src = slice(base + i * page_size, base + i * page_size + n)
+            dst = slice(pg * page_size, pg * page_size + n)
+            k_pool[:, dst] = np.transpose(w.k[:, :, src], (0, 2, 1, 3))
+            v_pool[:, dst] = np.transpose(w.v[:, :, src], (0, 2, 1, 3))
+    strides = (n_pages * page_size * Hkv * d, Hkv * d, d)
+    return k_pool, v_pool, table, n_pages, strides
