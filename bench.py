@@ -181,13 +181,20 @@ def run_cuda(args):
     w = wl.generate(spec, seed=rank_seed(rank), layers=args.layers)   # every rank evicts its own request: no exchange step
     spec = w.spec
     L = spec.seq_lens[0]
-    prob = B.Problem.from_workload(w, smooth_mode=args.smooth_mode, smooth_kappa=args.kappa,
-                                   pool_kernel=args.pool_kernel)
+    over = dict(smooth_mode=args.smooth_mode, smooth_kappa=args.kappa, pool_kernel=args.pool_kernel)
+    k_host, v_host = w.k, w.v
+    if args.page_size:
+        # the same rows held in a pool of pages handed out in random order (the host-buffer leg has no paged form)
+        k_host, v_host, table, n_pages, strides = wl.paged_pool(w, args.page_size, seed=rank_seed(rank))
+        over.update(kv_strides=strides, kv_req_offset=None, page_size=args.page_size, n_pages=n_pages,
+                    page_table=torch.from_numpy(table).cuda())
+        args.skip_e2e = True
+    prob = B.Problem.from_workload(w, **over)
     tb = [int(x) for x in w.total_budget]
     rows, TH = sum(tb), prob.total_heads
     es = w.torch_dtype()
 
-    q, k, v = (w.as_torch(a).cuda() for a in (w.q, w.k, w.v))
+    q, k, v = (w.as_torch(a).cuda() for a in (w.q, k_host, v_host))
     S = torch.from_numpy(w.head_scores).cuda()
     k_out = torch.empty((rows, spec.head_dim), dtype=es, device="cuda")
     v_out = torch.empty_like(k_out)
@@ -309,7 +316,7 @@ def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_m
                    "head_dim": spec.head_dim, "L": L, "window": spec.window, "keep": spec.keep,
                    "requests_per_gpu": 1, "l2": "inputs larger than L2 (K+V of a step = %d MB)" % (2 * w.k.nbytes // 2**20),
                    "parallelism": f"replicas x{world}, no collective",
-                   "smooth_mode": args.smooth_mode},
+                   "smooth_mode": args.smooth_mode, "page_size": args.page_size},
         "tokens_heads_per_s": round(L * spec.n_kv_heads * NL * world / (ms_step * 1e-3), 1),
         "hbm_gbs": round(hbm_gbs, 1),
         "hbm_frac_of_nominal_8tbs": round(hbm_gbs / NOMINAL_HBM_GBS, 4),
@@ -398,6 +405,8 @@ def main():
                          "the mean, 3 average pooling, 4 max pooling (variants for ablation-style runs, not bench lines)")
     ap.add_argument("--kappa", type=float, default=0.5, help="cut-off fraction of --smooth-mode 1")
     ap.add_argument("--pool-kernel", type=int, default=7, help="window of --smooth-mode 3 and 4 (odd)")
+    ap.add_argument("--page-size", type=int, default=0, choices=[0, 16, 32, 64, 128],
+                    help="hold K and V in a pool of pages of this many tokens (0 = contiguous, the bench line)")
     ap.add_argument("--layers", type=int, default=None,
                     help="truncate the stack to its first LAYERS layers (small cases for profiler captures; not a bench line)")
     args = ap.parse_args()
