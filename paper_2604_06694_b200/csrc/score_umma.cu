@@ -408,8 +408,14 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
   auto share_units = [&](int g) { return g == 0 ? u_split : n16 - u_split; };  // sweep 2: units of 16 rows
 
   if (warp == kProducerWarp) {
-    if (lane == 0) {
-      // ---- TMA producer ----
+    // ---- TMA producer ----
+    // Lane 0 runs the ring. With a paged pool the 128 / page_size pages of a tile are fetched by as many lanes,
+    // one page each (a copy costs its issuing thread about a hundred cycles, and a tile of 16-token pages is 8 to 32
+    // copies): those lanes walk the same schedule, lane 0 alone waits and arms the barriers, and its verdict reaches
+    // the others through the shuffle that also orders their copies after the arming.
+    const int n_sub = a.sh.page_size ? kTileKeys >> a.sh.page_shift : 1;
+    const uint32_t lanes = (1u << n_sub) - 1u;
+    if (lane < n_sub) {
       int it = 0, heads = 0, prev_u = -1, s = 0;  // s, ph: slot of the K ring and its phase
       uint32_t ph = 0;
       bool ok = true;
@@ -417,49 +423,48 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
       for (int n = unit_begin; n < unit_end && ok; ++n) {
         const ScoreUnit U = Unext;
         if (n + 1 < unit_end) Unext = a.units[n + 1];  // the next descriptor arrives under this unit's work
-        if (U.u != prev_u) {
-          if (heads > 0) ok = mbar_wait(smem_u32(&sm->q_empty), (heads - 1) & 1, abort);  // MMAs on the old Q are done
-          if (!ok) break;
-          const uint32_t bar = smem_u32(&sm->q_full);
-          mbar_expect_tx(bar, static_cast<uint32_t>(R) * D * 2);
-          for (int kb = 0; kb < KB; ++kb)
-            tma_load_4d(smem_u32(q_s + kb * q_blk), &tm.q[U.r - a.r0], bar, kb * 64, U.h * G, 0, U.l);
-          prev_u = U.u;
-          ++heads;
-        }
         for (int t = 0; t < U.n_tiles; ++t, ++it) {
-          ok = mbar_wait(smem_u32(&sm->k_empty[s]), ph ^ 1, abort);
-          if (!ok) break;
           const uint32_t bar = smem_u32(&sm->k_full[s]);
-          mbar_expect_tx(bar, kKStage);
+          int page_y = 0;
+          if (a.sh.page_size) {
+            // this lane's page of the tile; past the request's last token, or with an id outside the pool (which is
+            // reported), the copy starts outside the map and delivers zeros
+            const int tok = U.kt0 + t * kTileKeys + lane * a.sh.page_size;
+            page_y = a.sh.n_pages << a.sh.page_shift;
+            if (tok < U.P + a.sh.window) {
+              const int pg = __ldg(a.sh.page_table + U.r * a.sh.page_table_stride + (tok >> a.sh.page_shift));
+              if (pg >= 0 && pg < a.sh.n_pages) page_y = pg << a.sh.page_shift;
+              else atomicExch(a.status, AUDIOKV_EDEVICE);
+            }
+          }
+          bool mine = true;
+          if (lane == 0) {
+            if (t == 0 && U.u != prev_u) {
+              if (heads > 0) mine = mbar_wait(smem_u32(&sm->q_empty), (heads - 1) & 1, abort);  // MMAs on the old Q are done
+              if (mine) {
+                const uint32_t qbar = smem_u32(&sm->q_full);
+                mbar_expect_tx(qbar, static_cast<uint32_t>(R) * D * 2);
+                for (int kb = 0; kb < KB; ++kb)
+                  tma_load_4d(smem_u32(q_s + kb * q_blk), &tm.q[U.r - a.r0], qbar, kb * 64, U.h * G, 0, U.l);
+                prev_u = U.u;
+                ++heads;
+              }
+            }
+            if (mine) mine = mbar_wait(smem_u32(&sm->k_empty[s]), ph ^ 1, abort);
+            if (mine) mbar_expect_tx(bar, kKStage);
+          }
+          ok = __shfl_sync(lanes, mine, 0);
+          if (!ok) break;
           if (a.sh.page_size == 0) {
             for (int kb = 0; kb < KB; ++kb)
               tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r - a.r0], bar, kb * 64,
                           U.kt0 + t * kTileKeys, U.h, U.l);
           } else {
-            // Paged pool: k[0] maps the whole pool as (d, page * page_size + token in page, KV head, layer) with a box
-            // of one page; the tile is filled page by page (page_size >= 16 rows of 128 bytes: whole swizzle groups).
-            // Pages past the request's last token start outside the map and arrive as zeros; so does a page id
-            // outside the pool, which is also reported.
-            const int ps = a.sh.page_size, n_sub = kTileKeys >> a.sh.page_shift, L = U.P + a.sh.window;
-            const int32_t* tab = a.sh.page_table + U.r * a.sh.page_table_stride;
-            const int tok0 = U.kt0 + t * kTileKeys;
-            int y[kTileKeys / 16];
-#pragma unroll
-            for (int i = 0; i < kTileKeys / 16; ++i) {
-              y[i] = a.sh.n_pages << a.sh.page_shift;
-              if (i < n_sub && tok0 + i * ps < L) {
-                const int pg = __ldg(tab + ((tok0 + i * ps) >> a.sh.page_shift));
-                if (pg >= 0 && pg < a.sh.n_pages) y[i] = pg << a.sh.page_shift;
-                else atomicExch(a.status, AUDIOKV_EDEVICE);
-              }
-            }
-#pragma unroll
-            for (int i = 0; i < kTileKeys / 16; ++i)
-              if (i < n_sub)
-                for (int kb = 0; kb < KB; ++kb)
-                  tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk + i * ps * 128), &tm.k[0], bar, kb * 64, y[i],
-                              U.h, U.l);
+            // k[0] maps the whole pool as (d, page * page_size + token in page, KV head, layer) with a box of one
+            // page: at least 16 rows of 128 bytes, whole swizzle groups, so the tile comes out as in the contiguous case
+            for (int kb = 0; kb < KB; ++kb)
+              tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk + lane * a.sh.page_size * 128), &tm.k[0], bar,
+                          kb * 64, page_y, U.h, U.l);
           }
           if (++s == S) {
             s = 0;
@@ -467,7 +472,7 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
           }
         }
       }
-      if (*abort) {  // let the copies still in flight land before the CTA goes away
+      if (lane == 0 && *abort) {  // let the copies still in flight land before the CTA goes away
         const long long short_limit = 200000000LL;
         for (int j = it > S ? it - S : 0; j < it; ++j)
           mbar_wait(smem_u32(&sm->k_full[j % S]), (j / S) & 1, abort, short_limit);
