@@ -7,6 +7,7 @@ Prints ONE JSON line (rank 0). `--impl reference` times the CPU oracle instead.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -178,7 +179,14 @@ def run_cuda(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     spec = wl.config(args.config)
-    w = wl.generate(spec, seed=rank_seed(rank), layers=args.layers)   # every rank evicts its own request: no exchange step
+    sharded = args.shard == "layers"
+    if sharded:
+        # one request for the whole job, its layers dealt out over the ranks; no exchange step either: the budgets need
+        # every head's score, which is a table of a few hundred floats that every rank holds
+        n_full = args.layers or spec.n_layers
+        w = wl.generate(spec, seed=0, layers=args.layers, layer_range=wl.layer_shard(n_full, world, rank))
+    else:
+        w = wl.generate(spec, seed=rank_seed(rank), layers=args.layers)   # every rank evicts its own request
     spec = w.spec
     L = spec.seq_lens[0]
     over = dict(smooth_mode=args.smooth_mode, smooth_kappa=args.kappa, pool_kernel=args.pool_kernel)
@@ -207,6 +215,29 @@ def run_cuda(args):
     def step():
         B.audiokv_evict(ctx, prob, q, k, v, S, tb, k_out, v_out, kept, budgets, cu)
 
+    if sharded:
+        # every step: the allocation over the whole stack (a second context planned for all layers; it touches no
+        # K, V or Q), then steps 1, 2, 4 on this rank's layers with its slice of the budgets. With one request the
+        # slice is a contiguous run of the table: a view, no copy.
+        assert len(spec.seq_lens) == 1
+        w_all = dataclasses.replace(w, spec=dataclasses.replace(spec, n_layers=w.full_layers))
+        prob_all = B.Problem.from_workload(w_all, **over)
+        ctx_all = B.Context(prob_all, device=local)
+        TH_all = prob_all.total_heads
+        budgets_all = torch.empty(TH_all, dtype=torch.int32, device="cuda")
+        cu_all = torch.empty(TH_all + 1, dtype=torch.int32, device="cuda")
+        mine = budgets_all[w.layer_begin * spec.n_kv_heads:(w.layer_begin + spec.n_layers) * spec.n_kv_heads]
+        B.audiokv_allocate(ctx_all, prob_all, S, tb, budgets_all, cu_all)
+        rows = int(mine.sum().item())
+        k_out = torch.empty((rows, spec.head_dim), dtype=es, device="cuda")
+        v_out = torch.empty_like(k_out)
+        kept = torch.empty(rows, dtype=torch.int32, device="cuda")
+        args.skip_e2e = True
+
+        def step():
+            B.audiokv_allocate(ctx_all, prob_all, S, tb, budgets_all, cu_all)
+            B.audiokv_evict_budgeted(ctx, prob, q, k, v, mine, k_out, v_out, kept, cu)
+
     def barrier():
         if world > 1:
             torch.distributed.barrier()
@@ -226,7 +257,7 @@ def run_cuda(args):
         step()
     e1.record(stream)
     barrier()
-    launches = ctx.launch_count() - n0
+    launches = ctx.launch_count() - n0 + (args.steps if sharded else 0)   # + the allocation of the other context
     ms_total = e0.elapsed_time(e1)
     ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
     clocks = None
@@ -264,7 +295,8 @@ def run_cuda(args):
         if world > 1:
             torch.distributed.destroy_process_group()
         return
-    report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_ms, h2d, d2h)
+    job_layers = w.full_layers if sharded else spec.n_layers * world
+    report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_ms, h2d, d2h, job_layers, sharded)
     if world > 1:
         torch.distributed.destroy_process_group()
 
@@ -295,29 +327,30 @@ def run_e2e(B, ctx, prob, w, spec, tb, rows, TH, es, barrier, world, args):
     return e2e_ms, h2d, d2h
 
 
-def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_ms, h2d, d2h):
+def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_ms, h2d, d2h, job_layers, sharded):
     NL = spec.n_layers
     peaks, peak_kind = measured_peaks()
-    us_layer = whole_job_us_per_layer(ms_step, NL, world)
+    us_layer = ms_step * 1e3 / job_layers     # replicas: whole_job_us_per_layer(ms_step, NL, world)
     cbytes = contract_bytes_per_layer(spec, L)
-    hbm_gbs = cbytes * NL * world / (ms_step * 1e-3) / 1e9
+    hbm_gbs = cbytes * job_layers / (ms_step * 1e-3) / 1e9
     kern = {n: statistics.mean(v) for n, v in per_kernel.items()}
     tot = sum(kern.values()) or 1.0
     dom = max(kern, key=kern.get)
     sm_max = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz")
-    per_kernel_roofline = [kernel_roofline(n, v, spec, w, peaks, sm_max) for n, v in kern.items() if n != "allocate"]
+    per_kernel_roofline = [kernel_roofline(n, v, spec, w, peaks, sm_max) for n, v in kern.items() if n not in ("allocate", "budget_prefix")]
     roof = dict(next(r for r in per_kernel_roofline if r["kernel"] == dom))
     roof["peak_source"] = peak_kind
     line = {
         "metric": METRIC, "value": round(us_layer, 4), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "higher_is_better": False,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": spec.name, "layers": NL, "q_heads": spec.n_q_heads, "kv_heads": spec.n_kv_heads,
+        "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "layers": job_layers if sharded else NL, "q_heads": spec.n_q_heads, "kv_heads": spec.n_kv_heads,
                    "head_dim": spec.head_dim, "L": L, "window": spec.window, "keep": spec.keep,
                    "requests_per_gpu": 1, "l2": "inputs larger than L2 (K+V of a step = %d MB)" % (2 * w.k.nbytes // 2**20),
-                   "parallelism": f"replicas x{world}, no collective",
+                   "parallelism": (f"one request, layers sharded over {world} ranks ({NL} on rank 0), no collective"
+                                   if sharded else f"replicas x{world}, no collective"),
                    "smooth_mode": args.smooth_mode, "page_size": args.page_size},
-        "tokens_heads_per_s": round(L * spec.n_kv_heads * NL * world / (ms_step * 1e-3), 1),
+        "tokens_heads_per_s": round(L * spec.n_kv_heads * job_layers / (ms_step * 1e-3), 1),
         "hbm_gbs": round(hbm_gbs, 1),
         "hbm_frac_of_nominal_8tbs": round(hbm_gbs / NOMINAL_HBM_GBS, 4),
         "hbm_frac_of_measured": round(hbm_gbs / peaks["hbm_gbs"], 4),
@@ -332,7 +365,7 @@ def report(args, spec, w, L, world, ms_step, launches, per_kernel, clocks, e2e_m
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
         "clocks": clocks,
     }
-    if not args.skip_cpu:
+    if not args.skip_cpu and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, spec, budget_s=15.0)
     print(json.dumps(line), flush=True)
 
@@ -405,6 +438,9 @@ def main():
                          "the mean, 3 average pooling, 4 max pooling (variants for ablation-style runs, not bench lines)")
     ap.add_argument("--kappa", type=float, default=0.5, help="cut-off fraction of --smooth-mode 1")
     ap.add_argument("--pool-kernel", type=int, default=7, help="window of --smooth-mode 3 and 4 (odd)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "layers"],
+                    help="N > 1: 'replicas' = one request per rank (weak scaling, the default); 'layers' = one request, "
+                         "its layers dealt out over the ranks, budgets from one allocation over the whole stack (strong)")
     ap.add_argument("--page-size", type=int, default=0, choices=[0, 16, 32, 64, 128],
                     help="hold K and V in a pool of pages of this many tokens (0 = contiguous, the bench line)")
     ap.add_argument("--layers", type=int, default=None,

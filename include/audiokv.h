@@ -220,6 +220,18 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
 size_t audiokv_workspace_bytes_host(const audiokv_params* p, int64_t q_elems, int64_t kv_elems,
                                     const int64_t* total_budget);
 
+/* The pass with budgets chosen by the caller: steps 1, 2 and 4 of audiokv_evict, step 3 left
+ * out. For a run that shards the heads over several GPUs (the allocation of Section 3.1
+ * normalises over ALL layers and heads of a request, so it is computed once for the whole
+ * stack with audiokv_allocate and each GPU evicts its layers with its slice of the result),
+ * and for budget rules other than the paper's.
+ * budgets: device int32 [total heads], W <= budgets[u] <= L_r; a value outside is clamped
+ * into that range and reported as AUDIOKV_EINVAL in the status word. cu_kept is an output
+ * (prefix sums of the budgets); k_out, v_out, kept_idx need sum_u budgets[u] rows. */
+int audiokv_evict_budgeted(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k, const void* v,
+                           const int32_t* budgets, void* k_out, void* v_out, int32_t* kept_idx, int32_t* cu_kept,
+                           audiokv_stream stream);
+
 /* Decode-time re-eviction of an already compacted cache (Section 3.3: the importance
  * sequence may also come from a sliding window of decoding steps; Fig. 3, decoding phase).
  * After an eviction every head has its own length, so the cache is ragged per head: head

@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.audiokv_allocate.argtypes = [vp, pp, vp, ctypes.POINTER(i64), vp, vp, vp]
         L.audiokv_select_gather.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.audiokv_evict.argtypes = [vp, pp, vp, vp, vp, vp, ctypes.POINTER(i64), vp, vp, vp, vp, vp, vp]
+        L.audiokv_evict_budgeted.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.audiokv_evict_budgeted.restype = ctypes.c_int
         L.audiokv_reevict_workspace_bytes.restype = sz
         L.audiokv_reevict_workspace_bytes.argtypes = [pp, ctypes.POINTER(i32)]
         L.audiokv_reevict.argtypes = [vp, pp, vp, vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), vp, vp, vp, vp, vp]
@@ -292,6 +294,14 @@ def audiokv_evict(ctx: Context, prob: Problem, q_win, k, v, head_scores, total_b
                                    _dev(head_scores, "head_scores"), _budget_array(total_budget), _dev(k_out, "k_out"),
                                    _dev(v_out, "v_out"), _dev(kept_idx, "kept_idx"), _dev(budgets, "budgets"),
                                    _dev(cu_kept, "cu_kept"), _stream()), "audiokv_evict")
+
+
+def audiokv_evict_budgeted(ctx: Context, prob: Problem, q_win, k, v, budgets, k_out, v_out, kept_idx, cu_kept) -> None:
+    """budgets: CUDA int32 [total heads], chosen by the caller (e.g. a slice of audiokv_allocate's output)."""
+    ctx._check(lib().audiokv_evict_budgeted(ctx.h, prob.ref, _dev(q_win, "q_win"), _dev(k, "k"), _dev(v, "v"),
+                                            _dev(budgets, "budgets"), _dev(k_out, "k_out"), _dev(v_out, "v_out"),
+                                            _dev(kept_idx, "kept_idx"), _dev(cu_kept, "cu_kept"), _stream()),
+               "audiokv_evict_budgeted")
 
 
 def _i32_array(a: Sequence[int]):

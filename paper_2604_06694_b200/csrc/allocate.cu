@@ -162,7 +162,55 @@ allocate_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restr
     cu_kept[sh.total_heads] = static_cast<int32_t>(args.cu_base[blockIdx.x] + args.total[blockIdx.x]);
 }
 
+// Budgets handed in by the caller: a checked copy (each clamped into [W, L] of its request, a clamp being reported
+// through the status word) and its exclusive prefix sums. One block; the heads are walked in chunks of the block size.
+__global__ void __launch_bounds__(1024)
+budget_prefix_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const int32_t* __restrict__ given,
+                     int32_t* __restrict__ budgets, int32_t* __restrict__ cu_kept, int* __restrict__ status) {
+  __shared__ long long warp_sum[32];
+  __shared__ long long carry;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int u0 = 0; u0 < sh.total_heads; u0 += 1024) {
+    const int u = u0 + threadIdx.x;
+    long long b = 0;
+    if (u < sh.total_heads) {
+      const int L = reqs[u / sh.heads_per_req].L;
+      int g = given[u];
+      if (g < sh.window || g > L) {
+        atomicExch(status, AUDIOKV_EINVAL);
+        g = g < sh.window ? sh.window : L;
+      }
+      budgets[u] = g;
+      b = g;
+    }
+    long long inc = b;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const long long t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    if (lane == 31) warp_sum[warp] = inc;
+    __syncthreads();
+    long long before = carry;
+    for (int w = 0; w < warp; ++w) before += warp_sum[w];
+    if (u < sh.total_heads) cu_kept[u] = static_cast<int32_t>(before + inc - b);
+    __syncthreads();
+    if (threadIdx.x == 1023) carry = before + inc;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) cu_kept[sh.total_heads] = static_cast<int32_t>(carry);
+}
+
 }  // namespace
+
+cudaError_t launch_budget_prefix(const Shape& sh, const ReqDesc* d_reqs, const int32_t* given, int32_t* budgets,
+                                 int32_t* cu_kept, int* status, Launch ln) {
+  budget_prefix_kernel<<<1, 1024, 0, ln.stream>>>(sh, d_reqs, given, budgets, cu_kept, status);
+  ln.done("budget_prefix");
+  return cudaGetLastError();
+}
 
 cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float* head_scores,
                             const int64_t* h_total_budget, int32_t* budgets, int32_t* cu_kept, int* status,

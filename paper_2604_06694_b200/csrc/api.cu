@@ -743,6 +743,29 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
   return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, s);
 }
 
+int audiokv_evict_budgeted(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k, const void* v,
+                           const int32_t* budgets, void* k_out, void* v_out, int32_t* kept_idx, int32_t* cu_kept,
+                           audiokv_stream stream) {
+  if (!q_win || !k || !v || !budgets || !k_out || !v_out || !kept_idx || !cu_kept) return AUDIOKV_EINVAL;
+  if (!aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+    return AUDIOKV_EALIGN;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = prepare(ctx, p, s);
+  if (rc) return rc;
+  Plan& pl = ctx->plan;
+  float* ws_scores = reinterpret_cast<float*>(ctx->ws + pl.lay.scores);
+  int32_t* ws_kstar = reinterpret_cast<int32_t*>(ctx->ws + pl.lay.kstar);
+  int32_t* ws_budgets = reinterpret_cast<int32_t*>(ctx->ws + pl.lay.aux);  // the checked copy the selection reads
+  profile_begin(ctx, s);
+  Launch ln{s, &ctx->launches, &ctx->prof};
+  cudaError_t e = launch_budget_prefix(pl.sh, d_reqs(ctx), budgets, ws_budgets, cu_kept, d_status(ctx), ln);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  if ((rc = do_score(ctx, q_win, k, ws_scores, s))) return rc;
+  float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
+  if ((rc = do_smooth(ctx, ws_scores, ws_smoothed, ws_kstar, ws_budgets, cu_kept, kept_idx, s))) return rc;
+  return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, s);
+}
+
 namespace {
 
 // The per-head problem of a re-eviction: every head of the compacted cache becomes a request of one layer and one

@@ -176,6 +176,10 @@ cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float*
                             const int64_t* h_total_budget, int32_t* budgets, int32_t* cu_kept, int* status,
                             Launch ln);
 
+// given: device int32 [total heads], budgets chosen by the caller; budgets: their checked copy; cu_kept: prefix sums.
+cudaError_t launch_budget_prefix(const Shape& sh, const ReqDesc* d_reqs, const int32_t* given, int32_t* budgets,
+                                 int32_t* cu_kept, int* status, Launch ln);
+
 // select_gather.cu
 cudaError_t launch_select(const Shape& sh, const ReqDesc* d_reqs, const float* smoothed, const int32_t* budgets,
                           const int32_t* cu_kept, int32_t* kept_idx, int max_P, int* status, Launch ln);

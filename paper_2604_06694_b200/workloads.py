@@ -20,7 +20,7 @@ from __future__ import annotations
 
 import dataclasses
 import math
-from typing import List, Optional, Sequence
+from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
 import torch
@@ -88,6 +88,8 @@ class Workload:
     cu_seqlen: np.ndarray         # int64 [n_req + 1] token offsets of the requests
     total_budget: np.ndarray      # int64 [n_req]
     base: int                     # r (tokens per head)
+    layer_begin: int = 0          # a layer shard: spec.n_layers layers starting here; head_scores and
+    full_layers: Optional[int] = None  # total_budget still cover the full_layers layers of the whole stack
 
     @property
     def n_req(self) -> int:
@@ -134,21 +136,27 @@ def _ar1_inplace(x: np.ndarray, rho: float) -> None:
     x[...] = lfilter([1.0], [1.0, -rho], drive, axis=0)
 
 
-def generate(spec: WorkloadSpec, seed: int = 0, layers: Optional[int] = None) -> Workload:
+def generate(spec: WorkloadSpec, seed: int = 0, layers: Optional[int] = None,
+             layer_range: Optional[Tuple[int, int]] = None) -> Workload:
     """Draw one workload. `layers` truncates the stack (the first `layers` layers) for small parity cases;
-    budgets are then computed for the truncated stack."""
+    budgets are then computed for the truncated stack. `layer_range` = (l0, l1) draws only layers l0..l1-1 of
+    that stack, bit-identical to the same layers of the full draw (a layer shard of a multi-GPU run): q, k, v hold
+    l1 - l0 layers, while head_scores and total_budget stay those of the whole stack, which the allocation needs."""
     if layers is not None:
         spec = dataclasses.replace(spec, n_layers=int(layers))
     NL, Hq, Hkv, d, W = spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.window
+    l0, l1 = (0, NL) if layer_range is None else (int(layer_range[0]), int(layer_range[1]))
+    if not 0 <= l0 < l1 <= NL:
+        raise ValueError("layer_range outside the stack")
     lens = list(spec.seq_lens)
     cu = np.zeros(len(lens) + 1, dtype=np.int64)
     cu[1:] = np.cumsum(lens)
     sumL = int(cu[-1])
     G = Hq // Hkv
     st = np.uint16 if spec.dtype == "bf16" else np.float32
-    k = np.zeros((NL, Hkv, sumL, d), dtype=st)
-    v = np.zeros((NL, Hkv, sumL, d), dtype=st)
-    q = np.zeros((len(lens), NL, W, Hq, d), dtype=st)
+    k = np.zeros((l1 - l0, Hkv, sumL, d), dtype=st)
+    v = np.zeros((l1 - l0, Hkv, sumL, d), dtype=st)
+    q = np.zeros((len(lens), l1 - l0, W, Hq, d), dtype=st)
     S = np.zeros((len(lens), NL, Hkv), dtype=np.float32)
     for r, L in enumerate(lens):
         n_audio = int(round(spec.audio_frac[r] * L))
@@ -157,7 +165,7 @@ def generate(spec: WorkloadSpec, seed: int = 0, layers: Optional[int] = None) ->
             S[r] = rng_s.uniform(0.0, 1.0, size=(NL, Hkv)).astype(np.float32)
         else:
             S[r] = rng_s.beta(0.5, 2.0, size=(NL, Hkv)).astype(np.float32)
-        for l in range(NL):
+        for l in range(l0, l1):
             rng = np.random.Generator(np.random.Philox(key=[seed, (r << 20) + l + 1]))
             for h in range(Hkv):
                 rho = spec.ar_rho if spec.ar_rho_range is None else float(rng.uniform(*spec.ar_rho_range))
@@ -166,15 +174,32 @@ def generate(spec: WorkloadSpec, seed: int = 0, layers: Optional[int] = None) ->
                     _ar1_inplace(x[:n_audio], rho)
                     if is_k and spec.n_sink:
                         x[: spec.n_sink] *= 8.0
-                    dst[l, h, cu[r]:cu[r] + L] = _store(x, spec.dtype)
+                    dst[l - l0, h, cu[r]:cu[r] + L] = _store(x, spec.dtype)
                 # window queries of this KV head's group; window tokens inside the audio segment continue an AR(1) chain
                 xq = rng.standard_normal(size=(W, G * d), dtype=np.float32)
                 n_aw = max(0, min(W, n_audio - (L - W)))
                 _ar1_inplace(xq[:n_aw], rho)
-                q[r, l, :, h * G:(h + 1) * G, :] = _store(xq, spec.dtype).reshape(W, G, d)
+                q[r, l - l0, :, h * G:(h + 1) * G, :] = _store(xq, spec.dtype).reshape(W, G, d)
     B = np.array([kept_total(spec, L) for L in lens], dtype=np.int64)
     base = base_per_head(spec, min(lens))
-    return Workload(spec, q, k, v, S, cu, B, base)
+    if layer_range is None:
+        return Workload(spec, q, k, v, S, cu, B, base)
+    return Workload(dataclasses.replace(spec, n_layers=l1 - l0), q, k, v, S, cu, B, base, layer_begin=l0, full_layers=NL)
+
+
+def layer_shard(n_layers: int, world: int, rank: int) -> Tuple[int, int]:
+    """Layers [l0, l1) of rank `rank` when the stack is dealt out in contiguous runs, the first n_layers % world ranks
+    taking one more."""
+    q, rem = divmod(n_layers, world)
+    l0 = rank * q + min(rank, rem)
+    return l0, l0 + q + (1 if rank < rem else 0)
+
+
+def shard_heads(n_req: int, n_layers: int, n_kv_heads: int, l0: int, l1: int) -> np.ndarray:
+    """Flat indices u = (r * n_layers + l) * n_kv_heads + h of the heads of layers l0..l1-1, in the order the shard's
+    own flat index runs (request, layer, head)."""
+    r, l, h = np.meshgrid(np.arange(n_req), np.arange(l0, l1), np.arange(n_kv_heads), indexing="ij")
+    return ((r * n_layers + l) * n_kv_heads + h).reshape(-1)
 
 
 def attention_rows(n_steps: int, n_heads: int, n_audio: int, n_text0: int = 16, seed: int = 0, word_tokens: int = 12):

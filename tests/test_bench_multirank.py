@@ -1,5 +1,6 @@
 """The multi-GPU path of bench.py is N independent replicas (one request per rank, no exchange step): what the
-ranks share is the barrier, the max-over-ranks timing and the whole-job arithmetic. Two CPU processes over gloo."""
+ranks share is the barrier, the max-over-ranks timing and the whole-job arithmetic. Its other mode deals the layers of
+one request out over the ranks. Two CPU processes over gloo."""
 import os
 import subprocess
 import sys
@@ -29,6 +30,21 @@ CHILD = textwrap.dedent("""
     out = [None] * world
     dist.all_gather_object(out, digest)
     assert out[0] != out[1]
+    # the layer-sharded mode: one request, its layers dealt out over the ranks; the shards are disjoint, cover the
+    # stack, hold exactly the full draw's layers, and every rank holds the whole head-score table and total budget
+    import dataclasses, numpy as np
+    spec3 = dataclasses.replace(spec, n_layers=3)
+    full = wl.generate(spec3, seed=0)
+    l0, l1 = wl.layer_shard(3, world, rank)
+    mine = wl.generate(spec3, seed=0, layer_range=(l0, l1))
+    assert np.array_equal(mine.k, full.k[l0:l1]) and np.array_equal(mine.q, full.q[:, l0:l1])
+    assert np.array_equal(mine.head_scores, full.head_scores) and np.array_equal(mine.total_budget, full.total_budget)
+    assert mine.layer_begin == l0 and mine.full_layers == 3 and mine.spec.n_layers == l1 - l0
+    heads = wl.shard_heads(len(spec3.seq_lens), 3, spec3.n_kv_heads, l0, l1).tolist()
+    parts = [None] * world
+    dist.all_gather_object(parts, (l0, l1, heads))
+    assert [p[:2] for p in parts] == [(0, 2), (2, 3)]
+    assert sorted(h for p in parts for h in p[2]) == list(range(len(spec3.seq_lens) * 3 * spec3.n_kv_heads))
     dist.destroy_process_group()
     print("rank", rank, "ok")
 """) % ROOT
