@@ -88,7 +88,7 @@ class ClockSampler:
 
 
 def contract_bytes_per_layer(spec, L):
-    """K read once plus kept K and V written (the roofline the benchmark spec defines)."""
+    """K read once plus kept K and V written: the least traffic one layer of the pass can have."""
     e = 4 if spec.dtype == "f32" else 2
     row = spec.n_kv_heads * spec.head_dim * e
     return L * row + 2 * int(spec.keep * L) * row

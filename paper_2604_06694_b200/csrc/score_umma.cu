@@ -411,7 +411,7 @@ score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
     // ---- TMA producer ----
     // Lane 0 runs the ring. With a paged pool the 128 / page_size pages of a tile are fetched by as many lanes,
     // one page each (a copy costs its issuing thread about a hundred cycles, and a tile of 16-token pages is 8 to 32
-    // copies): those lanes walk the same schedule, lane 0 alone waits and arms the barriers, and its verdict reaches
+    // copies): those lanes walk the same schedule, lane 0 alone waits and arms the barriers, and its result reaches
     // the others through the shuffle that also orders their copies after the arming.
     const int n_sub = a.sh.page_size ? kTileKeys >> a.sh.page_shift : 1;
     const uint32_t lanes = (1u << n_sub) - 1u;

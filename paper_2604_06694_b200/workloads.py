@@ -49,7 +49,7 @@ class WorkloadSpec:
 
 
 def config(i: int, seed: int = 0) -> WorkloadSpec:
-    """The five benchmark configurations (index as in the benchmark's list)."""
+    """The five benchmark configurations, smallest first; index 1 is the one the benchmark line is quoted on."""
     if i == 0:
         return WorkloadSpec("c1_tiny_f32", "f32", 1, 8, 2, 64, [1024], [768 / 1024], 1, head_score_dist="uniform")
     if i == 1:
