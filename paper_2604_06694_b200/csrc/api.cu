@@ -730,13 +730,12 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
     if ((e = cudaStreamWaitEvent(ctx->side, ctx->fork, 0)) != cudaSuccess) return cuda_fail(ctx, e);
   }
   rc = do_allocate(ctx, head_scores, total_budget, budgets, cu_kept, beside ? ctx->side : s);
-  if (beside) {
-    // recorded even after a failed launch, so that the side stream always rejoins the caller's
-    if ((e = cudaEventRecord(ctx->join, ctx->side)) != cudaSuccess) return cuda_fail(ctx, e);
-    if ((e = cudaStreamWaitEvent(s, ctx->join, 0)) != cudaSuccess) return cuda_fail(ctx, e);
-  }
+  // recorded even after a failed launch, so that the side stream always rejoins the caller's
+  if (beside && (e = cudaEventRecord(ctx->join, ctx->side)) != cudaSuccess) return cuda_fail(ctx, e);
+  if (!rc) rc = do_score(ctx, q_win, k, ws_scores, s);
+  // the selection is the first reader of the budgets: the scoring sweeps do not wait for them
+  if (beside && (e = cudaStreamWaitEvent(s, ctx->join, 0)) != cudaSuccess) return cuda_fail(ctx, e);
   if (rc) return rc;
-  if ((rc = do_score(ctx, q_win, k, ws_scores, s))) return rc;
   // the pooling variants hand their result to the selection through the score buffer itself
   float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
   if ((rc = do_smooth(ctx, ws_scores, ws_smoothed, ws_kstar, budgets, cu_kept, kept_idx, s))) return rc;
