@@ -49,3 +49,16 @@ def test_config5_ragged_batch_of_eight_in_one_launch(B):
     g = run_evict(B, w)
     assert g["launches"] == 5 + 2
     check_against_oracle(w, g)
+
+
+def test_maximum_sequence_length(B):
+    """L = 131072, the longest request the library takes: 1024 key tiles per head, a transform of 65520 complex points
+    that runs block by block through global scratch, budgets up to 98 k rows per head."""
+    spec = dataclasses.replace(wl.config(1), seq_lens=(131072,), audio_frac=(0.9,), n_layers=1, n_q_heads=14,
+                               n_kv_heads=2)
+    w = wl.generate(spec, seed=3)
+    check_against_oracle(w, run_evict(B, w))
+    from paper_2604_06694_b200 import binding
+    too_long = binding.Problem.from_workload(w)
+    too_long._seq[0] = 131073
+    assert binding.audiokv_scores_len(too_long) == binding.AUDIOKV_EINVAL
