@@ -59,6 +59,10 @@ struct audiokv_ctx {
   cudaEvent_t plan_ready = nullptr;
   cudaStream_t side = nullptr;            // audiokv_evict runs the allocation here, beside the scoring
   cudaEvent_t fork = nullptr, join = nullptr;
+  // audiokv_evict_host: copies in on `side`, kernels on the caller's stream, copies out on `out`, chunk by chunk
+  static constexpr int kMaxChunks = 8;
+  cudaStream_t out = nullptr;
+  cudaEvent_t chunk_in[kMaxChunks] = {}, chunk_done[kMaxChunks] = {}, copies_out = nullptr;
   int64_t launches = 0;
   Profiler prof;
   std::string cuda_error;
@@ -454,7 +458,9 @@ void profile_begin(audiokv_ctx* ctx, cudaStream_t stream) {
 const ReqDesc* d_reqs(audiokv_ctx* c) { return reinterpret_cast<const ReqDesc*>(c->ws + c->plan.lay.reqs); }
 int* d_status(audiokv_ctx* c) { return reinterpret_cast<int*>(c->ws + c->plan.lay.status); }
 
-int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cudaStream_t stream) {
+// head_end >= 0 (one request, tensor-core path only): the heads [head_begin, head_end) alone.
+int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cudaStream_t stream, int head_begin = 0,
+             int head_end = -1) {
   Plan& pl = ctx->plan;
   Launch ln{stream, &ctx->launches, &ctx->prof};
   float2* stats = reinterpret_cast<float2*>(ctx->ws + pl.lay.stats);
@@ -463,31 +469,37 @@ int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cuda
   {
     const ScoreUnit* units = reinterpret_cast<const ScoreUnit*>(ctx->ws + pl.lay.units);
     e = launch_score_umma(pl.sh, pl.reqs.data(), units, pl.unit_pre1.data(), units + pl.n_units1, pl.unit_pre2.data(),
-                          q, k, scores, stats, pl.n_slab, kSlabKeys, d_status(ctx), ln);
+                          q, k, scores, stats, pl.n_slab, kSlabKeys, d_status(ctx), ln, head_begin, head_end);
   }
+  if (head_end >= 0 && e != cudaSuccess) return cuda_fail(ctx, e);  // no head ranges in the FMA kernel
   if (e == cudaErrorNotSupported)  // fp32 inputs, W * G above 256, or strides the copy engine cannot take
     e = launch_score_simt(pl.sh, d_reqs(ctx), q, k, scores, stats, pl.n_slab, kSlabKeys, ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 
 // Smoothing; with budgets, cu_kept and kept_idx it also selects each head's kept tokens (smoothed may then be null).
+// head_end < 0: all heads, in the plan's cost-sorted order; else the heads [head_begin, head_end) in index order.
 int do_smooth(audiokv_ctx* ctx, const float* scores, float* smoothed, int32_t* kstar, const int32_t* budgets,
-              const int32_t* cu_kept, int32_t* kept_idx, cudaStream_t stream) {
+              const int32_t* cu_kept, int32_t* kept_idx, cudaStream_t stream, int head_begin = 0, int head_end = -1) {
   Plan& pl = ctx->plan;
   Launch ln{stream, &ctx->launches, &ctx->prof};
+  const bool all = head_end < 0;
+  const int count = all ? static_cast<int>(pl.sss_order.size()) : head_end - head_begin;
   cudaError_t e = launch_sss(pl.sh, d_reqs(ctx), reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans),
                              reinterpret_cast<const float2*>(ctx->ws + pl.lay.tables), scores, smoothed, kstar,
                              reinterpret_cast<float2*>(ctx->ws + pl.lay.fft_scratch), pl.scratch_per_block,
-                             pl.sss_grid, pl.sss_smem, reinterpret_cast<const int32_t*>(ctx->ws + pl.lay.order),
-                             static_cast<int>(pl.sss_order.size()), budgets, cu_kept, kept_idx, d_status(ctx), ln);
+                             all ? pl.sss_grid : (count < pl.sss_grid ? count : pl.sss_grid), pl.sss_smem,
+                             all ? reinterpret_cast<const int32_t*>(ctx->ws + pl.lay.order) : nullptr, count,
+                             head_begin, budgets, cu_kept, kept_idx, d_status(ctx), ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 
 int do_gather(audiokv_ctx* ctx, const int32_t* cu_kept, const int32_t* kept_idx, const void* k, const void* v,
-              void* k_out, void* v_out, cudaStream_t stream) {
+              void* k_out, void* v_out, cudaStream_t stream, int head_begin = 0, int head_end = -1) {
   Plan& pl = ctx->plan;
   Launch ln{stream, &ctx->launches, &ctx->prof};
-  cudaError_t e = launch_gather(pl.sh, d_reqs(ctx), cu_kept, kept_idx, k, v, k_out, v_out, ln);
+  cudaError_t e = launch_gather(pl.sh, d_reqs(ctx), cu_kept, kept_idx, k, v, k_out, v_out, head_begin,
+                                head_end < 0 ? pl.sh.total_heads : head_end, ln);
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 
@@ -607,6 +619,15 @@ int audiokv_create(audiokv_ctx** out, int device, size_t workspace_bytes) {
     delete c;
     return AUDIOKV_ECUDA;
   }
+  bool ok = cudaStreamCreateWithFlags(&c->out, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&c->copies_out, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < audiokv_ctx::kMaxChunks && ok; ++i)
+    ok = cudaEventCreateWithFlags(&c->chunk_in[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&c->chunk_done[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    audiokv_destroy(c);
+    return AUDIOKV_ECUDA;
+  }
   *out = c;
   return AUDIOKV_OK;
 }
@@ -618,6 +639,12 @@ int audiokv_destroy(audiokv_ctx* ctx) {
   cudaEventDestroy(ctx->fork);
   cudaEventDestroy(ctx->join);
   cudaStreamDestroy(ctx->side);
+  if (ctx->out) cudaStreamDestroy(ctx->out);
+  if (ctx->copies_out) cudaEventDestroy(ctx->copies_out);
+  for (int i = 0; i < audiokv_ctx::kMaxChunks; ++i) {
+    if (ctx->chunk_in[i]) cudaEventDestroy(ctx->chunk_in[i]);
+    if (ctx->chunk_done[i]) cudaEventDestroy(ctx->chunk_done[i]);
+  }
   for (cudaEvent_t e : ctx->prof.ev)
     if (e) cudaEventDestroy(e);
   cudaFree(ctx->ws);
@@ -906,8 +933,64 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
   char* db = ctx->ws + off;   off = align_up(off + sizeof(int32_t) * TH);
   char* dcu = ctx->ws + off;
   cudaError_t e;
-#define AKV_CP(dst, src, n, kind) \
-  if ((e = cudaMemcpyAsync(dst, src, n, kind, s)) != cudaSuccess) return cuda_fail(ctx, e)
+#define AKV_CP_ON(st, dst, src, n, kind) \
+  if ((e = cudaMemcpyAsync(dst, src, n, kind, st)) != cudaSuccess) return cuda_fail(ctx, e)
+#define AKV_CP(dst, src, n, kind) AKV_CP_ON(s, dst, src, n, kind)
+  // One request whose K and V are laid out layer by layer, scored on the tensor cores: the pass runs in chunks of
+  // layers, so that the copy of the next chunk's K and V (in), this chunk's kernels, and the copy of the previous
+  // chunk's kept rows (out) overlap; in and out use the two directions of the link. Everything else: in, pass, out.
+  const int NL = pl.sh.n_layers, Hkv = pl.sh.n_kv_heads;
+  const bool layered = pl.sh.n_req == 1 && NL > 1 && score_umma_takes(pl.sh) && !ctx->prof.on &&
+                       p->kv_stride_layer > 0 && kv_elems == static_cast<int64_t>(NL) * p->kv_stride_layer &&
+                       p->kv_stride_layer >= p->kv_stride_tok * pl.reqs[0].L && p->kv_stride_layer >= p->kv_stride_head * Hkv;
+  if (layered) {
+    const int n_chunks = NL < audiokv_ctx::kMaxChunks ? NL : audiokv_ctx::kMaxChunks;
+    int32_t* d_budgets = reinterpret_cast<int32_t*>(db);
+    int32_t* d_cu = reinterpret_cast<int32_t*>(dcu);
+    AKV_CP(dq, q_win, q_elems * es, cudaMemcpyHostToDevice);
+    AKV_CP(dS, head_scores, sizeof(float) * TH, cudaMemcpyHostToDevice);
+    if ((rc = do_allocate(ctx, reinterpret_cast<float*>(dS), total_budget, d_budgets, d_cu, s))) return rc;
+    // the chunk boundaries of the output: the prefix sums come back first (a few hundred bytes)
+    AKV_CP(budgets, db, sizeof(int32_t) * TH, cudaMemcpyDeviceToHost);
+    AKV_CP(cu_kept, dcu, sizeof(int32_t) * (TH + 1), cudaMemcpyDeviceToHost);
+    if ((e = cudaEventRecord(ctx->fork, s)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(ctx, e);
+    // the copy streams start behind everything the caller's stream holds so far (the workspace may be in use)
+    if ((e = cudaStreamWaitEvent(ctx->side, ctx->fork, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaStreamWaitEvent(ctx->out, ctx->fork, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+    float* ws_scores = reinterpret_cast<float*>(ctx->ws + pl.lay.scores);
+    int32_t* ws_kstar = reinterpret_cast<int32_t*>(ctx->ws + pl.lay.kstar);
+    float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
+    const size_t layer_bytes = static_cast<size_t>(p->kv_stride_layer) * es, row_bytes = static_cast<size_t>(p->head_dim) * es;
+    for (int c = 0; c < n_chunks; ++c) {
+      const int l0 = static_cast<int>(static_cast<int64_t>(NL) * c / n_chunks);
+      const int l1 = static_cast<int>(static_cast<int64_t>(NL) * (c + 1) / n_chunks);
+      const size_t off = l0 * layer_bytes, len = (l1 - l0) * layer_bytes;
+      AKV_CP_ON(ctx->side, dk + off, static_cast<const char*>(k) + off, len, cudaMemcpyHostToDevice);
+      AKV_CP_ON(ctx->side, dv + off, static_cast<const char*>(v) + off, len, cudaMemcpyHostToDevice);
+      if ((e = cudaEventRecord(ctx->chunk_in[c], ctx->side)) != cudaSuccess) return cuda_fail(ctx, e);
+      if ((e = cudaStreamWaitEvent(s, ctx->chunk_in[c], 0)) != cudaSuccess) return cuda_fail(ctx, e);
+      const int u0 = l0 * Hkv, u1 = l1 * Hkv;
+      if ((rc = do_score(ctx, dq, dk, ws_scores, s, u0, u1))) return rc;
+      if ((rc = do_smooth(ctx, ws_scores, ws_smoothed, ws_kstar, d_budgets, d_cu, reinterpret_cast<int32_t*>(dki), s, u0, u1)))
+        return rc;
+      if ((rc = do_gather(ctx, d_cu, reinterpret_cast<int32_t*>(dki), dk, dv, dko, dvo, s, u0, u1))) return rc;
+      if ((e = cudaEventRecord(ctx->chunk_done[c], s)) != cudaSuccess) return cuda_fail(ctx, e);
+      if ((e = cudaStreamWaitEvent(ctx->out, ctx->chunk_done[c], 0)) != cudaSuccess) return cuda_fail(ctx, e);
+      const size_t r0 = static_cast<size_t>(cu_kept[u0]), r1 = static_cast<size_t>(cu_kept[u1]);  // host copy, read above
+      AKV_CP_ON(ctx->out, static_cast<char*>(k_out) + r0 * row_bytes, dko + r0 * row_bytes, (r1 - r0) * row_bytes,
+                cudaMemcpyDeviceToHost);
+      AKV_CP_ON(ctx->out, static_cast<char*>(v_out) + r0 * row_bytes, dvo + r0 * row_bytes, (r1 - r0) * row_bytes,
+                cudaMemcpyDeviceToHost);
+      AKV_CP_ON(ctx->out, reinterpret_cast<char*>(kept_idx) + r0 * sizeof(int32_t), dki + r0 * sizeof(int32_t),
+                (r1 - r0) * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    }
+    // the caller's stream ends behind the last copy out, then the host waits for it
+    if ((e = cudaEventRecord(ctx->copies_out, ctx->out)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaStreamWaitEvent(s, ctx->copies_out, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(ctx, e);
+    return AUDIOKV_OK;
+  }
   AKV_CP(dq, q_win, q_elems * es, cudaMemcpyHostToDevice);
   AKV_CP(dk, k, kv_elems * es, cudaMemcpyHostToDevice);
   AKV_CP(dv, v, kv_elems * es, cudaMemcpyHostToDevice);
@@ -921,6 +1004,7 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
   AKV_CP(budgets, db, sizeof(int32_t) * TH, cudaMemcpyDeviceToHost);
   AKV_CP(cu_kept, dcu, sizeof(int32_t) * (TH + 1), cudaMemcpyDeviceToHost);
 #undef AKV_CP
+#undef AKV_CP_ON
   if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(ctx, e);
   return AUDIOKV_OK;
 }

@@ -158,18 +158,22 @@ struct ScoreUnit {
 bool score_umma_takes(const Shape& sh);
 // units1 / units2: device tables of the two sweeps (build_score_units gives their host form).
 // unit_pre1 / unit_pre2: host arrays [n_req + 1], units of the requests before r in either sweep.
+// head_begin / head_end (single request only): score the heads [head_begin, head_end) alone; -1 = all heads.
 cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
                               const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
-                              float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln);
+                              float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
+                              int head_begin = 0, int head_end = -1);
 
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);
-// order: n_order head indices (or -1); block b takes entries b, b + grid, ... . smoothed may be null when budgets, cu_kept and kept_idx are given: the kernel then goes on to the
+// order: n_order head indices (or -1); block b takes entries b, b + grid, ... ; a null order stands for the n_order heads
+// first_head, first_head + 1, ... . smoothed may be null when budgets, cu_kept and kept_idx are given: the kernel then goes on to the
 // top-k selection of each head from the smoothed scores it holds on chip (step 4a of the pass).
 cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_plans, const float2* d_tables,
                        const float* scores, float* smoothed, int32_t* kstar, float2* scratch,
                        int64_t scratch_per_block, int grid, size_t smem_bytes, const int32_t* order, int n_order,
-                       const int32_t* budgets, const int32_t* cu_kept, int32_t* kept_idx, int* status, Launch ln);
+                       int first_head, const int32_t* budgets, const int32_t* cu_kept, int32_t* kept_idx, int* status,
+                       Launch ln);
 
 // allocate.cu (h_total_budget: host array [n_req])
 cudaError_t launch_allocate(const Shape& sh, const ReqDesc* d_reqs, const float* head_scores,
@@ -183,8 +187,10 @@ cudaError_t launch_budget_prefix(const Shape& sh, const ReqDesc* d_reqs, const i
 // select_gather.cu
 cudaError_t launch_select(const Shape& sh, const ReqDesc* d_reqs, const float* smoothed, const int32_t* budgets,
                           const int32_t* cu_kept, int32_t* kept_idx, int max_P, int* status, Launch ln);
+// head_begin / head_end: the rows of heads [head_begin, head_end) only (0, total heads = everything).
 cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t* cu_kept, const int32_t* kept_idx,
-                          const void* k, const void* v, void* k_out, void* v_out, Launch ln);
+                          const void* k, const void* v, void* k_out, void* v_out, int head_begin, int head_end,
+                          Launch ln);
 
 // hit_score.cu: offline head score. counts: int32 [n_heads] (cleared here, then the hit totals).
 cudaError_t launch_hit_score(const float* attn, int n_steps, int n_heads, int64_t row_stride, const int32_t* row_len,

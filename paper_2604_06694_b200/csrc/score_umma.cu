@@ -738,8 +738,10 @@ bool score_umma_takes(const Shape& sh) {
 
 cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
                               const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
-                              float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln) {
+                              float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
+                              int head_begin, int head_end) {
   if (!score_umma_takes(sh) || slab_keys % kTileKeys) return cudaErrorNotSupported;
+  if (head_end >= 0 && sh.n_req != 1) return cudaErrorInvalidValue;  // head ranges: one request only
   EncodeTiledFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
   const int R = sh.window * sh.group, d = sh.head_dim;
@@ -805,9 +807,17 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
     }
     args.r0 = r0;
     const ScoreUnit* u1 = units1 + unit_pre1[r0];
-    const int n1 = unit_pre1[r1] - unit_pre1[r0];
+    int n1 = unit_pre1[r1] - unit_pre1[r0];
     const ScoreUnit* u2 = units2 + (n_units2 - unit_pre2[r1]);
-    const int n2 = unit_pre2[r1] - unit_pre2[r0];
+    int n2 = unit_pre2[r1] - unit_pre2[r0];
+    if (head_end >= 0) {
+      // one request: every head has the same number of slabs in a sweep, and its units are consecutive
+      const int s1 = n1 / sh.heads_per_req, s2 = n2 / sh.heads_per_req;
+      u1 += head_begin * s1;
+      n1 = (head_end - head_begin) * s1;
+      u2 += (sh.heads_per_req - head_end) * s2;  // sweep 2 lists the heads backwards
+      n2 = (head_end - head_begin) * s2;
+    }
 
 #define AKV_SWEEP(SW, DD, UNITS, N)                                                  \
   args.n_units = (N);                                                                \

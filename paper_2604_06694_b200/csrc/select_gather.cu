@@ -41,24 +41,26 @@ select_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restric
 // eight independent loads in flight per lane before the stores. log2_chunks: log2 of the chunks per row.
 constexpr int kGatherRows = 8;
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)  // three blocks per SM: at most 80 registers per thread
 gather_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const int32_t* __restrict__ cu_kept,
               const int32_t* __restrict__ kept_idx, const uint4* __restrict__ k, const uint4* __restrict__ v,
-              uint4* __restrict__ k_out, uint4* __restrict__ v_out, int log2_chunks, int elems_per_chunk) {
+              uint4* __restrict__ k_out, uint4* __restrict__ v_out, int log2_chunks, int elems_per_chunk,
+              int head_begin, int head_end) {
   chain_release();
   chain_wait();  // kept_idx and cu_kept come from the kernels before
-  const int64_t total_rows = cu_kept[sh.total_heads];
-  const int64_t n_batches = (total_rows + kGatherRows - 1) / kGatherRows;
+  const int64_t first_row = cu_kept[head_begin];  // the rows of heads [head_begin, head_end)
+  const int64_t total_rows = cu_kept[head_end];
+  const int64_t n_batches = (total_rows - first_row + kGatherRows - 1) / kGatherRows;
   const int lane = threadIdx.x & 31;
   const int64_t warp0 = (blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x) >> 5;
   const int64_t n_warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
   const int chunks = 1 << log2_chunks;
   for (int64_t bt = warp0; bt < n_batches; bt += n_warps) {
-    const int64_t row0 = bt * kGatherRows;
+    const int64_t row0 = first_row + bt * kGatherRows;
     int64_t my_src = 0;  // lane i < 8: first 16-byte chunk of the source row of output row row0 + i
     if (lane < kGatherRows && row0 + lane < total_rows) {
       const int64_t row = row0 + lane;
-      int lo = 0, hi = sh.total_heads;  // largest u with cu_kept[u] <= row
+      int lo = head_begin, hi = head_end;  // largest u with cu_kept[u] <= row
       while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
         if (__ldg(cu_kept + mid) <= row) lo = mid; else hi = mid;
@@ -107,7 +109,8 @@ cudaError_t launch_select(const Shape& sh, const ReqDesc* d_reqs, const float* s
 }
 
 cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t* cu_kept, const int32_t* kept_idx,
-                          const void* k, const void* v, void* k_out, void* v_out, Launch ln) {
+                          const void* k, const void* v, void* k_out, void* v_out, int head_begin, int head_end,
+                          Launch ln) {
   const int esize = sh.dtype == AUDIOKV_F32 ? 4 : 2;
   const int elems_per_chunk = 16 / esize;
   const int chunks_per_row = sh.head_dim / elems_per_chunk;  // 8 .. 64: head_dim is 64, 128 or 256
@@ -115,7 +118,7 @@ cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t*
   while ((1 << log2_chunks) < chunks_per_row) ++log2_chunks;
   cudaError_t e = launch_chained(gather_kernel, dim3(148 * 8), dim3(256), 0, ln.stream, sh, d_reqs, cu_kept, kept_idx,
                                  (const uint4*)k, (const uint4*)v, (uint4*)k_out, (uint4*)v_out, log2_chunks,
-                                 elems_per_chunk);
+                                 elems_per_chunk, head_begin, head_end);
   ln.done("gather");
   return e;
 }

@@ -636,8 +636,8 @@ __global__ void __launch_bounds__(kSssThreads, 1)
 sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict__ plans,
            const float2* __restrict__ tables, const float* scores, float* smoothed /* may alias scores */,
            int32_t* __restrict__ kstar_out, float2* __restrict__ scratch, int64_t scratch_per_block,
-           const int32_t* __restrict__ order, int n_order, const int32_t* __restrict__ budgets, const int32_t* __restrict__ cu_kept, int32_t* __restrict__ kept_idx,
-           int* __restrict__ status) {
+           const int32_t* __restrict__ order, int n_order, int first_head, const int32_t* __restrict__ budgets,
+           const int32_t* __restrict__ cu_kept, int32_t* __restrict__ kept_idx, int* __restrict__ status) {
   extern __shared__ __align__(16) float2 sbuf[];
   __shared__ FftPlan pl;
   __shared__ float2 wp[128];
@@ -649,7 +649,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
 
   int loaded_plan = -1;  // plan whose tables sit in shared memory
   for (int slot = blockIdx.x; slot < n_order; slot += gridDim.x) {
-    const int u = order[slot];
+    const int u = order ? order[slot] : first_head + slot;  // no list: heads first_head, first_head + 1, ...
     if (u < 0) continue;
     const int r = u / sh.heads_per_req;
     const ReqDesc rq = reqs[r];
@@ -974,12 +974,13 @@ cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_pl
 cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_plans, const float2* d_tables,
                        const float* scores, float* smoothed, int32_t* kstar, float2* scratch,
                        int64_t scratch_per_block, int grid, size_t smem_bytes, const int32_t* order, int n_order,
-                       const int32_t* budgets, const int32_t* cu_kept, int32_t* kept_idx, int* status, Launch ln) {
+                       int first_head, const int32_t* budgets, const int32_t* cu_kept, int32_t* kept_idx, int* status,
+                       Launch ln) {
   cudaError_t e = cudaFuncSetAttribute(sss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   if (e != cudaSuccess) return e;
   sss_kernel<<<grid, kSssThreads, smem_bytes, ln.stream>>>(sh, d_reqs, d_plans, d_tables, scores, smoothed, kstar,
-                                                           scratch, scratch_per_block, order, n_order, budgets, cu_kept, kept_idx,
-                                                           status);
+                                                           scratch, scratch_per_block, order, n_order, first_head, budgets,
+                                                           cu_kept, kept_idx, status);
   ln.done(budgets ? "sss_select" : "sss");
   return cudaGetLastError();
 }

@@ -110,6 +110,32 @@ def test_evict_host_buffers_equal_device_buffers(B):
         assert np.array_equal(a[key], b[key]), key
 
 
+@pytest.mark.parametrize("layers", [2, 5, 11])
+def test_evict_host_buffers_in_chunks_of_layers(B, layers):
+    """One bf16 request with its cache laid out layer by layer: the host-buffer call copies in, evicts and copies out
+    chunk by chunk (at most 8 chunks: 11 layers make uneven ones); the result is the device-buffer call's."""
+    spec = dataclasses.replace(wl.config(1), seq_lens=[1301], audio_frac=[0.9])
+    w = wl.generate(spec, seed=8, layers=layers)
+    a = run_evict(B, w)
+    b = run_evict(B, w, host=True)
+    for key in ("k_out", "v_out", "kept", "budgets", "cu"):
+        assert np.array_equal(a[key], b[key]), key
+    assert b["launches"] == 2 + 1 + 4 * min(layers, 8)      # tables, allocation, then 4 kernels per chunk
+    if layers == 5:
+        check_against_oracle(w, b)
+
+
+def test_evict_host_buffers_ragged_batch(B):
+    """Several requests: no chunking, one copy in, one pass, one copy out."""
+    spec = dataclasses.replace(wl.config(1), seq_lens=[700, 1301], audio_frac=[0.8, 0.9])
+    w = wl.generate(spec, seed=8, layers=2)
+    a = run_evict(B, w)
+    b = run_evict(B, w, host=True)
+    for key in ("k_out", "v_out", "kept", "budgets", "cu"):
+        assert np.array_equal(a[key], b[key]), key
+    assert b["launches"] == 2 + 5
+
+
 def test_evict_is_deterministic(B):
     w = wl.generate(wl.config(1), layers=1)
     a, b = run_evict(B, w), run_evict(B, w)
