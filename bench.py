@@ -322,7 +322,8 @@ def run_e2e(B, ctx, prob, w, spec, tb, rows, TH, es, barrier, world, args):
         step_host()
     barrier()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / n_e2e, world, "cuda")
-    h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv, hS))
+    # V is pinned: the gather fetches its kept rows from the host buffer itself, the other rows never cross the link
+    h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hS)) + hvo.numel() * hvo.element_size()
     d2h = sum(x.numel() * x.element_size() for x in (hko, hvo, hkept, hb, hcu))
     return e2e_ms, h2d, d2h
 

@@ -962,19 +962,30 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
     int32_t* ws_kstar = reinterpret_cast<int32_t*>(ctx->ws + pl.lay.kstar);
     float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
     const size_t layer_bytes = static_cast<size_t>(p->kv_stride_layer) * es, row_bytes = static_cast<size_t>(p->head_dim) * es;
+    // V is only ever read by the gather, and only its kept rows: when the caller's V is pinned memory the device can
+    // address, the gather fetches those rows straight from it and the rest of V never crosses the link.
+    const void* v_src = dv;
+    {
+      cudaPointerAttributes at{};
+      if (cudaPointerGetAttributes(&at, v) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer &&
+          aligned16(at.devicePointer))
+        v_src = at.devicePointer;
+      else
+        cudaGetLastError();  // pageable memory is reported as an error by older drivers: not one of this call's
+    }
     for (int c = 0; c < n_chunks; ++c) {
       const int l0 = static_cast<int>(static_cast<int64_t>(NL) * c / n_chunks);
       const int l1 = static_cast<int>(static_cast<int64_t>(NL) * (c + 1) / n_chunks);
       const size_t off = l0 * layer_bytes, len = (l1 - l0) * layer_bytes;
       AKV_CP_ON(ctx->side, dk + off, static_cast<const char*>(k) + off, len, cudaMemcpyHostToDevice);
-      AKV_CP_ON(ctx->side, dv + off, static_cast<const char*>(v) + off, len, cudaMemcpyHostToDevice);
+      if (v_src == dv) AKV_CP_ON(ctx->side, dv + off, static_cast<const char*>(v) + off, len, cudaMemcpyHostToDevice);
       if ((e = cudaEventRecord(ctx->chunk_in[c], ctx->side)) != cudaSuccess) return cuda_fail(ctx, e);
       if ((e = cudaStreamWaitEvent(s, ctx->chunk_in[c], 0)) != cudaSuccess) return cuda_fail(ctx, e);
       const int u0 = l0 * Hkv, u1 = l1 * Hkv;
       if ((rc = do_score(ctx, dq, dk, ws_scores, s, u0, u1))) return rc;
       if ((rc = do_smooth(ctx, ws_scores, ws_smoothed, ws_kstar, d_budgets, d_cu, reinterpret_cast<int32_t*>(dki), s, u0, u1)))
         return rc;
-      if ((rc = do_gather(ctx, d_cu, reinterpret_cast<int32_t*>(dki), dk, dv, dko, dvo, s, u0, u1))) return rc;
+      if ((rc = do_gather(ctx, d_cu, reinterpret_cast<int32_t*>(dki), dk, v_src, dko, dvo, s, u0, u1))) return rc;
       if ((e = cudaEventRecord(ctx->chunk_done[c], s)) != cudaSuccess) return cuda_fail(ctx, e);
       if ((e = cudaStreamWaitEvent(ctx->out, ctx->chunk_done[c], 0)) != cudaSuccess) return cuda_fail(ctx, e);
       const size_t r0 = static_cast<size_t>(cu_kept[u0]), r1 = static_cast<size_t>(cu_kept[u1]);  // host copy, read above

@@ -20,7 +20,7 @@ def B():
     return binding
 
 
-def run_evict(B, w, host=False, **over):
+def run_evict(B, w, host=False, pin=False, **over):
     prob = B.Problem.from_workload(w, **over)
     s = w.spec
     TH = prob.total_heads
@@ -37,8 +37,10 @@ def run_evict(B, w, host=False, **over):
     if host:
         ws = B.audiokv_workspace_bytes_host(prob, w.q.size, w.k.size, tb)
         ctx = B.Context(prob, workspace_bytes=ws)
-        B.audiokv_evict_host(ctx, prob, w.as_torch(w.q), w.as_torch(w.k), w.as_torch(w.v), S, tb, k_out, v_out, kept,
-                             budgets, cu)
+        hq, hk, hv = w.as_torch(w.q), w.as_torch(w.k), w.as_torch(w.v)
+        if pin:
+            hq, hk, hv = hq.pin_memory(), hk.pin_memory(), hv.pin_memory()
+        B.audiokv_evict_host(ctx, prob, hq, hk, hv, S, tb, k_out, v_out, kept, budgets, cu)
     else:
         ctx = B.Context(prob)
         B.audiokv_evict(ctx, prob, to_dev(w, w.q), to_dev(w, w.k), to_dev(w, w.v), S.cuda(), tb, k_out, v_out, kept,
@@ -123,6 +125,10 @@ def test_evict_host_buffers_in_chunks_of_layers(B, layers):
     assert b["launches"] == 2 + 1 + 4 * min(layers, 8)      # tables, allocation, then 4 kernels per chunk
     if layers == 5:
         check_against_oracle(w, b)
+    # pinned inputs: the gather reads the kept V rows from the caller's buffer itself, V is not copied in
+    c = run_evict(B, w, host=True, pin=True)
+    for key in ("k_out", "v_out", "kept", "budgets", "cu"):
+        assert np.array_equal(a[key], c[key]), key
 
 
 def test_evict_host_buffers_ragged_batch(B):
