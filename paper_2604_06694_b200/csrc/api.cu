@@ -56,6 +56,8 @@ struct audiokv_ctx {
   size_t ws_bytes = 0;
   Plan plan;
   bool plan_uploaded = false;
+  uint64_t plan_id = 0;      // counts plan rebuilds
+  ScoreMapCache score_maps;
   cudaEvent_t plan_ready = nullptr;
   cudaStream_t side = nullptr;            // audiokv_evict runs the allocation here, beside the scoring
   cudaEvent_t fork = nullptr, join = nullptr;
@@ -410,6 +412,7 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   if (!same_plan(ctx->plan, p)) {
     int rc = build_plan(p, &ctx->plan);
+    ctx->plan_id += 1;
     if (rc) return rc;
     ctx->plan_uploaded = false;
   }
@@ -469,7 +472,8 @@ int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cuda
   {
     const ScoreUnit* units = reinterpret_cast<const ScoreUnit*>(ctx->ws + pl.lay.units);
     e = launch_score_umma(pl.sh, pl.reqs.data(), units, pl.unit_pre1.data(), units + pl.n_units1, pl.unit_pre2.data(),
-                          q, k, scores, stats, pl.n_slab, kSlabKeys, d_status(ctx), ln, head_begin, head_end);
+                          q, k, scores, stats, pl.n_slab, kSlabKeys, d_status(ctx), ln, head_begin, head_end,
+                          &ctx->score_maps, ctx->plan_id);
   }
   if (head_end >= 0 && e != cudaSuccess) return cuda_fail(ctx, e);  // no head ranges in the FMA kernel
   if (e == cudaErrorNotSupported)  // fp32 inputs, W * G above 256, or strides the copy engine cannot take

@@ -3,6 +3,8 @@
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+
+#include <vector>
 #include <stdint.h>
 
 #include "../../include/audiokv.h"
@@ -156,13 +158,23 @@ struct ScoreUnit {
 // cannot be described to the copy engine, and the caller then scores with launch_score_simt.
 // h_reqs: host copy of the request table (the tensor maps are encoded on the host).
 bool score_umma_takes(const Shape& sh);
+// The encoded tensor maps of the last call, kept by the context: encoding a few hundred maps costs more host time than
+// the kernels take on a short cache, and a serving loop calls with the same buffers and the same plan again and again.
+struct ScoreMapCache {
+  const void* q = nullptr;
+  const void* k = nullptr;
+  uint64_t plan_id = 0;   // changes whenever the plan is rebuilt
+  int page_size = -1;
+  std::vector<unsigned char> packs;  // one argument pack per launch chunk
+};
 // units1 / units2: device tables of the two sweeps (build_score_units gives their host form).
 // unit_pre1 / unit_pre2: host arrays [n_req + 1], units of the requests before r in either sweep.
 // head_begin / head_end (single request only): score the heads [head_begin, head_end) alone; -1 = all heads.
 cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
                               const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
                               float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
-                              int head_begin = 0, int head_end = -1);
+                              int head_begin = 0, int head_end = -1, ScoreMapCache* cache = nullptr,
+                              uint64_t plan_id = 0);
 
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);

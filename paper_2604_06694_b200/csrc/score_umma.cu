@@ -36,7 +36,7 @@ constexpr int kMaxStages = 8;
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
 constexpr int kSmemLimit = 232448;               // 227 KB
 
-constexpr int kMapChunk = 64;  // requests per launch: their tensor maps travel as kernel arguments
+constexpr int kMapChunk = 120;  // requests per launch: their tensor maps travel as kernel arguments (32 KB at most)
 
 struct TmapPack {
   CUtensorMap q[kMapChunk];  // 4-D per request: (d, query head, window row, layer)
@@ -72,6 +72,7 @@ struct Small {
   uint32_t tmem_base;
   int abort;
 };
+static_assert(sizeof(TmapPack) + sizeof(UmmaArgs) <= 32764, "kernel arguments are limited to 32764 bytes");
 static_assert(offsetof(Small, negc) % 16 == 0 && offsetof(Small, k_full) % 8 == 0, "alignment of the small shared area");
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -739,7 +740,7 @@ bool score_umma_takes(const Shape& sh) {
 cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
                               const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
                               float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
-                              int head_begin, int head_end) {
+                              int head_begin, int head_end, ScoreMapCache* cache, uint64_t plan_id) {
   if (!score_umma_takes(sh) || slab_keys % kTileKeys) return cudaErrorNotSupported;
   if (head_end >= 0 && sh.n_req != 1) return cudaErrorInvalidValue;  // head ranges: one request only
   EncodeTiledFn enc = encode_fn();
@@ -769,11 +770,22 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
   // by chunk. Sweep 1 lists the units by ascending request, sweep 2 by descending request, so a chunk of requests
   // is one contiguous run of either list.
   const int n_units2 = unit_pre2[sh.n_req];
+  const int n_chunks = (sh.n_req + kMapChunk - 1) / kMapChunk;
+  // the maps depend on the buffers, the request table and the strides: the same buffers under the same plan reuse them
+  std::vector<unsigned char> local;
+  std::vector<unsigned char>& packs = cache ? cache->packs : local;
+  const size_t pack_bytes = sizeof(TmapPack) * static_cast<size_t>(n_chunks) + 64;  // + room to align to 64 bytes
+  const bool reuse = cache && cache->q == q && cache->k == k && cache->plan_id == plan_id &&
+                     cache->page_size == sh.page_size && packs.size() == pack_bytes;
+  if (!reuse) {
+    if (cache) cache->q = nullptr;  // stays invalid if the encoding below fails half way
+    packs.assign(pack_bytes, 0);
+  }
+  unsigned char* pack0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(packs.data()) + 63) & ~uintptr_t(63));
   for (int r0 = 0; r0 < sh.n_req; r0 += kMapChunk) {
     const int r1 = r0 + kMapChunk < sh.n_req ? r0 + kMapChunk : sh.n_req;
-    TmapPack tm;
-    memset(&tm, 0, sizeof(tm));
-    for (int r = r0; r < r1; ++r) {
+    TmapPack& tm = *reinterpret_cast<TmapPack*>(pack0 + sizeof(TmapPack) * static_cast<size_t>(r0 / kMapChunk));
+    for (int r = r0; r < r1 && !reuse; ++r) {
       {
         const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(sh.n_q_heads),
                                     static_cast<cuuint64_t>(sh.window), static_cast<cuuint64_t>(sh.n_layers)};
@@ -836,6 +848,12 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
       AKV_SWEEP(2, 256, u2, n2);
     }
 #undef AKV_SWEEP
+  }
+  if (cache && !reuse) {
+    cache->q = q;
+    cache->k = k;
+    cache->plan_id = plan_id;
+    cache->page_size = sh.page_size;
   }
   return cudaSuccess;
 }
