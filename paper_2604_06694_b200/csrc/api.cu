@@ -421,6 +421,14 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
   pl.sh.page_table = p->page_size ? p->page_table : nullptr;  // device data of this call, not part of the plan
   pl.sh.page_status = reinterpret_cast<int*>(ctx->ws + pl.lay.status);
   if (!ctx->plan_uploaded) {
+    // A new plan goes up with copies from pageable memory, which a stream capture cannot hold: the first call with
+    // a given shape has to run outside capture (later ones add nothing but kernels and may be captured).
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if ((e = cudaStreamIsCapturing(stream, &cap)) != cudaSuccess) return cuda_fail(ctx, e);
+    if (cap != cudaStreamCaptureStatusNone) {
+      ctx->cuda_error = "the plan of these params is not on the device yet: make one call outside stream capture first";
+      return AUDIOKV_ECUDA;
+    }
     // earlier calls on other streams may still read the old tables
     if ((e = cudaStreamWaitEvent(stream, ctx->plan_ready, 0)) != cudaSuccess) return cuda_fail(ctx, e);
     if ((e = cudaMemsetAsync(ctx->ws + pl.lay.status, 0, 64, stream)) != cudaSuccess) return cuda_fail(ctx, e);
@@ -440,10 +448,11 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
     e = launch_fft_tables(static_cast<int>(pl.fft.size()), reinterpret_cast<float2*>(ctx->ws + pl.lay.tables),
                           reinterpret_cast<const FftPlan*>(ctx->ws + pl.lay.plans), ln);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
+    // The host waits until the plan is resident (once per shape): calls that follow, on any stream or inside a
+    // capture, then need no ordering against the upload.
     if ((e = cudaEventRecord(ctx->plan_ready, stream)) != cudaSuccess) return cuda_fail(ctx, e);
+    if ((e = cudaEventSynchronize(ctx->plan_ready)) != cudaSuccess) return cuda_fail(ctx, e);
     ctx->plan_uploaded = true;
-  } else {
-    if ((e = cudaStreamWaitEvent(stream, ctx->plan_ready, 0)) != cudaSuccess) return cuda_fail(ctx, e);
   }
   return AUDIOKV_OK;
 }
