@@ -186,3 +186,36 @@ def test_rejections(B):
     with pytest.raises(B.AudioKVError) as e:
         B.audiokv_score(ctx, prob, to_dev(w, w.q), kd.reshape(-1)[1:], scores)      # misaligned K
     assert e.value.status == B.AUDIOKV_EALIGN
+
+
+def test_one_context_alternating_shapes_and_buffers(B):
+    """One context serving two shapes in turn, and one shape with two sets of buffers: every switch rebuilds the plan
+    (tables, schedule, and the tensor maps the context keeps from the last call), and every result must equal what a
+    fresh context gives."""
+    spec_a = dataclasses.replace(wl.config(1), seq_lens=[900], audio_frac=[0.9])
+    spec_b = dataclasses.replace(wl.config(1), seq_lens=[1301, 640], audio_frac=[0.9, 0.8])
+    wa1, wa2 = wl.generate(spec_a, seed=1, layers=2), wl.generate(spec_a, seed=2, layers=2)
+    wb = wl.generate(spec_b, seed=3, layers=2)
+    fresh = {id(w): run_evict(B, w) for w in (wa1, wa2, wb)}
+    pa, pb = B.Problem.from_workload(wa1), B.Problem.from_workload(wb)
+    ctx = B.Context(pb, workspace_bytes=max(B.audiokv_workspace_bytes(pa), B.audiokv_workspace_bytes(pb)))
+
+    def call(w, prob):
+        s = w.spec
+        rows, TH = int(w.total_budget.sum()), prob.total_heads
+        k_out = torch.zeros((rows, s.head_dim), dtype=torch.bfloat16, device="cuda")
+        v_out = torch.zeros_like(k_out)
+        kept = torch.zeros(rows, dtype=torch.int32, device="cuda")
+        budgets = torch.zeros(TH, dtype=torch.int32, device="cuda")
+        cu = torch.zeros(TH + 1, dtype=torch.int32, device="cuda")
+        B.audiokv_evict(ctx, prob, to_dev(w, w.q), to_dev(w, w.k), to_dev(w, w.v), torch.from_numpy(w.head_scores).cuda(),
+                        [int(x) for x in w.total_budget], k_out, v_out, kept, budgets, cu)
+        torch.cuda.synchronize()
+        assert ctx.last_device_status() == 0
+        want = fresh[id(w)]
+        assert np.array_equal(kept.cpu().numpy(), want["kept"]) and np.array_equal(cu.cpu().numpy(), want["cu"])
+        assert np.array_equal(k_out.cpu().view(torch.uint16).numpy(), want["k_out"])
+        assert np.array_equal(v_out.cpu().view(torch.uint16).numpy(), want["v_out"])
+
+    for w, prob in ((wa1, pa), (wb, pb), (wa2, pa), (wa1, pa), (wb, pb), (wb, pb), (wa2, pa)):
+        call(w, prob)
