@@ -132,7 +132,12 @@ size_t audiokv_workspace_bytes(const audiokv_params* p);
  * allocation the library makes). *ctx is set on success. */
 int audiokv_create(audiokv_ctx** ctx, int device, size_t workspace_bytes);
 
-/* Stream capture: every device-buffer entry point may be recorded into a CUDA graph, once the
+/* Threads and streams: a context holds one plan, one workspace and the tensor maps of its last
+ * call, so calls on ONE context must not run concurrently, neither from two host threads nor on
+ * two streams whose work may overlap on the GPU (their kernels would share the score buffers).
+ * Use one context per stream; contexts are independent of one another.
+ *
+ * Stream capture: every device-buffer entry point may be recorded into a CUDA graph, once the
  * context has seen its params in a call OUTSIDE capture (the first call with a new shape copies
  * the plan up from pageable memory and waits for it; inside a capture it returns AUDIOKV_ECUDA
  * and says so in audiokv_last_cuda_error). audiokv_evict forks to a stream of the context for the

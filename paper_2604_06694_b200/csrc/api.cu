@@ -48,6 +48,12 @@ struct Plan {
   Layout lay{};
 };
 
+// Host arrays of the per-head problem that audiokv_reevict derives from its arguments.
+struct ReevictArrays {
+  std::vector<int32_t> len;
+  std::vector<int64_t> kv_off, q_off, budget;
+};
+
 }  // namespace
 
 struct audiokv_ctx {
@@ -68,9 +74,7 @@ struct audiokv_ctx {
   int64_t launches = 0;
   Profiler prof;
   std::string cuda_error;
-  // audiokv_reevict: the per-head problem it hands to the eviction pass
-  std::vector<int32_t> re_len;
-  std::vector<int64_t> re_kv_off, re_q_off, re_budget;
+  ReevictArrays re;  // audiokv_reevict: the per-head problem it hands to the eviction pass
 };
 
 namespace {
@@ -809,19 +813,19 @@ namespace {
 
 // The per-head problem of a re-eviction: every head of the compacted cache becomes a request of one layer and one
 // KV head, with its own length, its own place in the packed cache and its own slice of the window queries.
-int reevict_problem(audiokv_ctx* ctx, const audiokv_params* p, const int32_t* cu_cache, const int32_t* new_budgets,
+int reevict_problem(ReevictArrays* a, const audiokv_params* p, const int32_t* cu_cache, const int32_t* new_budgets,
                     audiokv_params* dp) {
-  if (!ctx || !p || !cu_cache) return AUDIOKV_EINVAL;
+  if (!a || !p || !cu_cache) return AUDIOKV_EINVAL;
   if (p->n_layers < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads || p->n_req < 1 ||
       p->head_dim < 1)
     return AUDIOKV_EINVAL;
   const int64_t TH = static_cast<int64_t>(p->n_req) * p->n_layers * p->n_kv_heads;
   if (TH > AUDIOKV_MAX_REQ) return AUDIOKV_EUNSUPPORTED;
   const int G = p->n_q_heads / p->n_kv_heads;
-  ctx->re_len.resize(TH);
-  ctx->re_kv_off.resize(TH);
-  ctx->re_q_off.resize(TH);
-  ctx->re_budget.resize(TH);
+  a->len.resize(TH);
+  a->kv_off.resize(TH);
+  a->q_off.resize(TH);
+  a->budget.resize(TH);
   if (cu_cache[0] != 0) return AUDIOKV_EINVAL;
   int64_t u = 0;
   for (int r = 0; r < p->n_req; ++r) {
@@ -830,12 +834,12 @@ int reevict_problem(audiokv_ctx* ctx, const audiokv_params* p, const int32_t* cu
       for (int h = 0; h < p->n_kv_heads; ++h, ++u) {
         const int64_t n = static_cast<int64_t>(cu_cache[u + 1]) - cu_cache[u];
         if (n <= p->window || n > AUDIOKV_MAX_SEQ_LEN) return AUDIOKV_EINVAL;
-        ctx->re_len[u] = static_cast<int32_t>(n);
-        ctx->re_kv_off[u] = static_cast<int64_t>(cu_cache[u]) * p->head_dim;
-        ctx->re_q_off[u] = q_r + l * p->q_stride_layer + static_cast<int64_t>(h) * G * p->q_stride_head;
+        a->len[u] = static_cast<int32_t>(n);
+        a->kv_off[u] = static_cast<int64_t>(cu_cache[u]) * p->head_dim;
+        a->q_off[u] = q_r + l * p->q_stride_layer + static_cast<int64_t>(h) * G * p->q_stride_head;
         if (new_budgets) {
           if (new_budgets[u] < p->window || new_budgets[u] > n) return AUDIOKV_EINVAL;
-          ctx->re_budget[u] = new_budgets[u];
+          a->budget[u] = new_budgets[u];
         }
       }
   }
@@ -844,14 +848,14 @@ int reevict_problem(audiokv_ctx* ctx, const audiokv_params* p, const int32_t* cu
   dp->n_layers = 1;
   dp->n_kv_heads = 1;
   dp->n_q_heads = G;
-  dp->seq_len = ctx->re_len.data();
+  dp->seq_len = a->len.data();
   dp->q_stride_req = 0;
   dp->q_stride_layer = 0;
   dp->kv_stride_layer = 0;
   dp->kv_stride_head = 0;
   dp->kv_stride_tok = p->head_dim;
-  dp->kv_req_offset = ctx->re_kv_off.data();
-  dp->q_req_offset = ctx->re_q_off.data();
+  dp->kv_req_offset = a->kv_off.data();
+  dp->q_req_offset = a->q_off.data();
   dp->base_per_head = 0;
   dp->page_size = 0;  // the compacted cache is packed, not paged
   dp->n_pages = 0;
@@ -863,7 +867,7 @@ int reevict_problem(audiokv_ctx* ctx, const audiokv_params* p, const int32_t* cu
 }  // namespace
 
 size_t audiokv_reevict_workspace_bytes(const audiokv_params* p, const int32_t* cu_cache) {
-  audiokv_ctx tmp;
+  ReevictArrays tmp;
   audiokv_params dp;
   if (reevict_problem(&tmp, p, cu_cache, nullptr, &dp)) return 0;
   return audiokv_workspace_bytes(&dp);
@@ -872,20 +876,20 @@ size_t audiokv_reevict_workspace_bytes(const audiokv_params* p, const int32_t* c
 int audiokv_reevict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k_cache,
                     const void* v_cache, const int32_t* cu_cache, const int32_t* new_budgets, void* k_out, void* v_out,
                     int32_t* kept_idx, int32_t* cu_kept, audiokv_stream stream) {
-  if (!new_budgets) return AUDIOKV_EINVAL;
+  if (!ctx || !new_budgets) return AUDIOKV_EINVAL;
   audiokv_params dp;
-  int rc = reevict_problem(ctx, p, cu_cache, new_budgets, &dp);
+  int rc = reevict_problem(&ctx->re, p, cu_cache, new_budgets, &dp);
   if (rc) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if ((rc = prepare(ctx, &dp, s))) return rc;
   // One head per request: the allocation hands each its whole total, whatever the weight. The weights and the
   // per-head budgets it writes live in the workspace.
-  const size_t TH = ctx->re_len.size();
+  const size_t TH = ctx->re.len.size();
   float* weights = reinterpret_cast<float*>(ctx->ws + ctx->plan.lay.aux);
   int32_t* budgets = reinterpret_cast<int32_t*>(weights + TH);
   cudaError_t e = cudaMemsetAsync(weights, 0x3f, sizeof(float) * TH, s);  // 0x3f3f3f3f = 0.747
   if (e != cudaSuccess) return cuda_fail(ctx, e);
-  return audiokv_evict(ctx, &dp, q_win, k_cache, v_cache, weights, ctx->re_budget.data(), k_out, v_out, kept_idx,
+  return audiokv_evict(ctx, &dp, q_win, k_cache, v_cache, weights, ctx->re.budget.data(), k_out, v_out, kept_idx,
                        budgets, cu_kept, s);
 }
 
