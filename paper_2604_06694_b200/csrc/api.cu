@@ -191,14 +191,19 @@ void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
     fp->M = 0;
   } else {
     fp->bluestein = 1;
-    // convolution length: the smallest 2^a 3^b 5^c 7^d (a >= 2) that holds 2N - 1 points; close to 2N - 1
+    // An odd real length is transformed at full complex length N = n, but only bins 0 .. (n-1)/2 are wanted (the rest
+    // mirror them) and only those go back into the inverse: differences between input and output indices then span
+    // N + (N-1)/2 values instead of 2N - 1, and the convolution may be that much shorter.
+    fp->half = fp->packed ? 0 : 1;
+    const int64_t need = fp->half ? static_cast<int64_t>(N) + (N - 1) / 2 : 2LL * N - 1;
+    // convolution length: the smallest 2^a 3^b 5^c 7^d (a >= 2) that holds `need` points; close to it
     // instead of up to twice that for a power of two, which also keeps more transforms in shared memory
     int M = 0;
     for (int64_t p7 = 1; p7 < 4LL * N; p7 *= 7)
       for (int64_t p5 = p7; p5 < 4LL * N; p5 *= 5)
         for (int64_t p3 = p5; p3 < 4LL * N; p3 *= 3)
           for (int64_t p2 = p3 * 4; p2 < 8LL * N; p2 *= 2)
-            if (p2 >= 2LL * N - 1) {
+            if (p2 >= need) {
               if (M == 0 || p2 < M) M = static_cast<int>(p2);
               break;
             }
@@ -230,6 +235,10 @@ void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
     *table_len += N;
     fp->filter_offset = *table_len;
     *table_len += fp->M;
+    if (fp->half) {
+      fp->filter2_offset = *table_len;
+      *table_len += fp->M;
+    }
   }
 }
 

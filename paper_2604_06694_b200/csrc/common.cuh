@@ -76,7 +76,8 @@ struct FftPlan {
   int32_t n;         // real length
   int32_t packed;    // 1: n even, transform z_m = x_2m + i x_2m+1 of length n/2; 0: length n with zero imaginary part
   int32_t N;         // complex transform length (n/2 or n)
-  int32_t bluestein; // 1: N goes through a chirp-z convolution of length M (a power of two)
+  int32_t bluestein; // 1: N goes through a chirp-z convolution of length M (a product of 2, 3, 5, 7)
+  int32_t half;      // bluestein, not packed (odd n): only bins 0 .. (n-1)/2 are computed and fed back, M >= N + (N-1)/2
   int32_t M;         // convolution length (bluestein only)
   int32_t in_smem;   // 1: the work buffer fits in shared memory
   int32_t tabs_smem; // 1: twiddles, post-twiddles and bin positions are staged in shared memory after the buffer
@@ -84,6 +85,7 @@ struct FftPlan {
   FftSeq seq;        // passes for length N (direct) or M (bluestein)
   int64_t chirp_offset;   // float2 index of c_j = exp(-i pi j^2 / N), j in [0, N)      (bluestein)
   int64_t filter_offset;  // float2 index of FFT_M of the wrapped conjugate chirp / M    (bluestein)
+  int64_t filter2_offset; // half: the same for the inverse direction's wrap (few inputs, all outputs)
   int64_t post_offset;    // float2 index of exp(-2 pi i k / n), k in [0, N/2]           (packed)
   int64_t pos_offset;     // float2 index of an int32 table: slot of bin k after the forward passes (direct)
 };

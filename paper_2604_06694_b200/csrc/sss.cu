@@ -565,17 +565,18 @@ __device__ __forceinline__ int seq_pos(const FftSeq& sq, int k) {
   return p;
 }
 
-// Chirp-z: buf[0..N) holds y (natural order) on entry and DFT_N(y) (natural order) on exit.
-// CONJ: conjugate on the way in and out, which turns the forward transform into the
-// unnormalised inverse.
+// Chirp-z: buf[0..n_in) holds y (natural order; entries from n_in on count as zero) on entry and bins 0..n_out-1
+// of DFT_N(y) (natural order) on exit. `filt` is the transformed wrapped chirp that fits this pair of ranges: the
+// plan's filter for n_in = n_out = N, and for a half plan the filter (N in, (N+1)/2 out) or filter2 ((N+1)/2 in,
+// N out). CONJ: conjugate on the way in and out, which turns the forward transform into the unnormalised inverse.
 template <bool CONJ>
-__device__ __forceinline__ void bluestein(SkewBuf buf, const FftPlan& pl, const float2* tables, float2* wp, float2* sbuf) {
+__device__ __forceinline__ void bluestein(SkewBuf buf, const FftPlan& pl, const float2* tables, float2* wp, float2* sbuf,
+                                          int n_in, int n_out, const float2* filt) {
   const float2* chirp = tables + pl.chirp_offset;
-  const float2* filt = tables + pl.filter_offset;
-  const int N = pl.N, M = pl.M;
+  const int M = pl.M;
   for (int j = threadIdx.x; j < M; j += kSssThreads) {
     float2 v = make_float2(0.f, 0.f);
-    if (j < N) {
+    if (j < n_in) {
       v = buf[j];
       if (CONJ) v = cconj(v);
       v = cmul(v, __ldg(chirp + j));
@@ -589,7 +590,7 @@ __device__ __forceinline__ void bluestein(SkewBuf buf, const FftPlan& pl, const 
   __syncthreads();
   if (pl.in_smem) fft_dit_inv(buf, pl.seq, tables + pl.seq.tw_offset, wp);
   else fft_dit_inv_big(buf, pl.seq, pl.g_pass, tables + pl.seq.tw_offset, wp, sbuf);
-  for (int j = threadIdx.x; j < N; j += kSssThreads) {
+  for (int j = threadIdx.x; j < n_out; j += kSssThreads) {
     float2 v = cmul(buf[j], __ldg(chirp + j));
     buf[j] = CONJ ? cconj(v) : v;
   }
@@ -733,7 +734,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
 
     // 2. forward complex transform; bin k then sits at POS(k)
     if (pl.bluestein)
-      bluestein<false>(buf, pl, tables, wp, sbuf);
+      bluestein<false>(buf, pl, tables, wp, sbuf, N, pl.half ? Kb + 1 : N, tables + pl.filter_offset);
     else if (pl.in_smem)
       fft_dif(buf, pl.seq, tw, wp);
     else
@@ -847,6 +848,9 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
           buf[pq] = cconj(csub(E, iO));
         }
       }
+    } else if (pl.half) {
+      // bins 0 .. Kb alone go back: x_j = (2 / N) Re sum_{k <= Kb} h_k e^{+2 pi i j k / N}, h_0 = F_0 / 2, h_k = F_k
+      for (int k = threadIdx.x; k <= Kb; k += kSssThreads) buf[k] = cscale(buf[k], k == 0 ? 0.5f * weight(0) : weight(k));
     } else {
       for (int k = threadIdx.x; k < N; k += kSssThreads) {
         const int kk = k <= Kb ? k : N - k;
@@ -858,7 +862,8 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
 
     // 6. inverse complex transform (unnormalised), natural order out
     if (pl.bluestein)
-      bluestein<true>(buf, pl, tables, wp, sbuf);
+      bluestein<true>(buf, pl, tables, wp, sbuf, pl.half ? Kb + 1 : N, N,
+                      tables + (pl.half ? pl.filter2_offset : pl.filter_offset));
     else if (pl.in_smem)
       fft_dit_inv(buf, pl.seq, tw, wp);
     else
@@ -867,7 +872,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
 
     // 7. residual mix. `smoothed` (optional) gets the result; when budgets are given the result
     //    also stays in the work buffer, as order-preserving keys, for the selection below.
-    const float inv = 1.f / static_cast<float>(N), al = sh.alpha, om = 1.f - sh.alpha;
+    const float inv = (pl.half ? 2.f : 1.f) / static_cast<float>(N), al = sh.alpha, om = 1.f - sh.alpha;
     const bool sel = budgets != nullptr;
     // packed: the keys of tokens 2m and 2m+1 replace element m; otherwise the key of token m goes to the real part of element m
     if (pl.packed) {
@@ -929,20 +934,32 @@ __global__ void fft_table_kernel(const FftPlan* __restrict__ plans, int n_plans,
   }
   if (pl.bluestein) {
     const int N = pl.N, M = pl.M;
+    // Wrapped conjugate chirp b[d] = exp(+i pi d^2 / N) at position d for index differences d = out - in >= 0 and at
+    // M - |d| for d < 0, zero elsewhere. Full plan: |d| < N both ways. Half plan: the forward filter serves d in
+    // [-(N-1), Kb] (N inputs, Kb + 1 outputs), the inverse one d in [-Kb, N-1].
+    const int Kb = (pl.n - 1) / 2;
+    const int pos_f = pl.half ? Kb + 1 : N, neg_f = N;       // forward filter: d in (-neg_f, pos_f)
+    const int pos_i = N, neg_i = pl.half ? Kb + 1 : N;       // inverse filter (half plans only)
+    auto chirp_at = [&](int d) -> float2 {  // exp(+i pi d^2 / N), the exponent reduced exactly
+      const long long q = (static_cast<long long>(d) * d) % (2LL * N);
+      double s, c;
+      sincospi(static_cast<double>(q) / N, &s, &c);
+      return make_float2(static_cast<float>(c), static_cast<float>(s));
+    };
     for (int j = gid; j < M; j += gsz) {
-      // wrapped conjugate chirp b[j] = exp(+i pi j^2 / N) at j and M - j, j < N; zero elsewhere
-      int jj = -1;
-      if (j < N) jj = j;
-      else if (M - j < N) jj = M - j;
-      float2 b = make_float2(0.f, 0.f);
-      if (jj >= 0) {
-        const long long q = (static_cast<long long>(jj) * jj) % (2LL * N);
-        double s, c;
-        sincospi(static_cast<double>(q) / N, &s, &c);
-        b = make_float2(static_cast<float>(c), static_cast<float>(s));
-        if (j < N) tables[pl.chirp_offset + j] = make_float2(b.x, -b.y);
+      if (j < N) {
+        const float2 b = chirp_at(j);
+        tables[pl.chirp_offset + j] = make_float2(b.x, -b.y);
       }
-      tables[pl.filter_offset + j] = b;
+      // position j holds difference +j inside the positive support, difference -(M - j) inside the negative one
+      // (they never collide: M is at least their total length), zero in between
+      auto wrapped = [&](int pos, int neg) -> float2 {
+        if (j < pos) return chirp_at(j);
+        if (M - j < neg) return chirp_at(M - j);
+        return make_float2(0.f, 0.f);
+      };
+      tables[pl.filter_offset + j] = wrapped(pos_f, neg_f);
+      if (pl.half) tables[pl.filter2_offset + j] = wrapped(pos_i, neg_i);
     }
   }
 }
@@ -955,10 +972,13 @@ fft_filter_kernel(const FftPlan* __restrict__ plans, float2* __restrict__ tables
   if (threadIdx.x == 0) pl = plans[blockIdx.x];
   __syncthreads();
   if (!pl.bluestein) return;
-  float2* f = tables + pl.filter_offset;
-  fft_dif(SkewBuf{f, 31, 0}, pl.seq, tables + pl.seq.tw_offset, wp);
-  const float inv = 1.f / static_cast<float>(pl.M);
-  for (int j = threadIdx.x; j < pl.M; j += kSssThreads) f[j] = cscale(f[j], inv);
+  for (int which = 0; which < (pl.half ? 2 : 1); ++which) {
+    float2* f = tables + (which ? pl.filter2_offset : pl.filter_offset);
+    __syncthreads();
+    fft_dif(SkewBuf{f, 31, 0}, pl.seq, tables + pl.seq.tw_offset, wp);
+    const float inv = 1.f / static_cast<float>(pl.M);
+    for (int j = threadIdx.x; j < pl.M; j += kSssThreads) f[j] = cscale(f[j], inv);
+  }
 }
 
 }  // namespace
