@@ -36,11 +36,15 @@ constexpr int kMaxStages = 8;
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
 constexpr int kSmemLimit = 232448;               // 227 KB
 
-constexpr int kMapChunk = 120;  // requests per launch: their tensor maps travel as kernel arguments (32 KB at most)
+// Tensor maps travel as kernel arguments, CAP requests' worth per launch. Two sizes: 8 for the usual small batch (the
+// arguments are copied at every launch, and 31 KB of them cost each sweep about 1.5 us), 120 for long batches such
+// as one request per head (32 KB of arguments at most).
+constexpr int kMapChunkSmall = 8, kMapChunkLarge = 120;
 
+template <int CAP>
 struct TmapPack {
-  CUtensorMap q[kMapChunk];  // 4-D per request: (d, query head, window row, layer)
-  CUtensorMap k[kMapChunk];  // 4-D per request: (d, token, KV head, layer)
+  CUtensorMap q[CAP];  // 4-D per request: (d, query head, window row, layer)
+  CUtensorMap k[CAP];  // 4-D per request: (d, token, KV head, layer)
 };
 
 struct UmmaArgs {
@@ -72,7 +76,7 @@ struct Small {
   uint32_t tmem_base;
   int abort;
 };
-static_assert(sizeof(TmapPack) + sizeof(UmmaArgs) <= 32764, "kernel arguments are limited to 32764 bytes");
+static_assert(sizeof(TmapPack<kMapChunkLarge>) + sizeof(UmmaArgs) <= 32764, "kernel arguments are limited to 32764 bytes");
 static_assert(offsetof(Small, negc) % 16 == 0 && offsetof(Small, k_full) % 8 == 0, "alignment of the small shared area");
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -332,9 +336,9 @@ __device__ __forceinline__ float colsum_tile(uint32_t taddr, int n_u, const floa
   return hsum(a0, a1, a2, a3);
 }
 
-template <int SWEEP, int D>
+template <int SWEEP, int D, int CAP>
 __global__ void __launch_bounds__(kThreads, 1)
-score_umma_kernel(const __grid_constant__ TmapPack tm, const UmmaArgs a) {
+score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   constexpr int KB = D / 64;                 // 64-element (128-byte) blocks along the head dimension
@@ -717,13 +721,19 @@ bool fill_strides(int rank, const cuuint64_t* dims, const int64_t* elem_strides,
   return true;
 }
 
-template <int SWEEP, int D>
-cudaError_t launch_sweep(const TmapPack& tm, const UmmaArgs& args, int grid, size_t smem, cudaStream_t stream) {
-  auto kern = score_umma_kernel<SWEEP, D>;
+template <int SWEEP, int D, int CAP>
+cudaError_t launch_sweep(const TmapPack<CAP>& tm, const UmmaArgs& args, int grid, size_t smem, cudaStream_t stream) {
+  auto kern = score_umma_kernel<SWEEP, D, CAP>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
   return launch_chained(kern, dim3(grid), dim3(kThreads), smem, stream, tm, args);
 }
+
+template <int CAP>
+cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
+                                  const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
+                                  float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
+                                  int head_begin, int head_end, ScoreMapCache* cache, uint64_t plan_id);
 
 }  // namespace
 
@@ -741,6 +751,22 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
                               const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
                               float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
                               int head_begin, int head_end, ScoreMapCache* cache, uint64_t plan_id) {
+  if (sh.n_req <= kMapChunkSmall)
+    return launch_score_umma_cap<kMapChunkSmall>(sh, h_reqs, units1, unit_pre1, units2, unit_pre2, q, k, scores, stats_ws,
+                                                 n_slab, slab_keys, status, ln, head_begin, head_end, cache, plan_id);
+  return launch_score_umma_cap<kMapChunkLarge>(sh, h_reqs, units1, unit_pre1, units2, unit_pre2, q, k, scores, stats_ws,
+                                               n_slab, slab_keys, status, ln, head_begin, head_end, cache, plan_id);
+}
+
+namespace {
+
+template <int CAP>
+cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
+                                  const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
+                                  float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
+                                  int head_begin, int head_end, ScoreMapCache* cache, uint64_t plan_id) {
+  constexpr int kMapChunk = CAP;
+  using Pack = TmapPack<CAP>;
   if (!score_umma_takes(sh) || slab_keys % kTileKeys) return cudaErrorNotSupported;
   if (head_end >= 0 && sh.n_req != 1) return cudaErrorInvalidValue;  // head ranges: one request only
   EncodeTiledFn enc = encode_fn();
@@ -766,7 +792,7 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
 
-  // Tensor maps are kernel arguments, kMapChunk requests' worth per launch: a longer batch takes both sweeps chunk
+  // Tensor maps are kernel arguments, CAP requests' worth per launch: a longer batch takes both sweeps chunk
   // by chunk. Sweep 1 lists the units by ascending request, sweep 2 by descending request, so a chunk of requests
   // is one contiguous run of either list.
   const int n_units2 = unit_pre2[sh.n_req];
@@ -774,7 +800,7 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
   // the maps depend on the buffers, the request table and the strides: the same buffers under the same plan reuse them
   std::vector<unsigned char> local;
   std::vector<unsigned char>& packs = cache ? cache->packs : local;
-  const size_t pack_bytes = sizeof(TmapPack) * static_cast<size_t>(n_chunks) + 64;  // + room to align to 64 bytes
+  const size_t pack_bytes = sizeof(Pack) * static_cast<size_t>(n_chunks) + 64;  // + room to align to 64 bytes
   const bool reuse = cache && cache->q == q && cache->k == k && cache->plan_id == plan_id &&
                      cache->page_size == sh.page_size && packs.size() == pack_bytes;
   if (!reuse) {
@@ -784,7 +810,7 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
   unsigned char* pack0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(packs.data()) + 63) & ~uintptr_t(63));
   for (int r0 = 0; r0 < sh.n_req; r0 += kMapChunk) {
     const int r1 = r0 + kMapChunk < sh.n_req ? r0 + kMapChunk : sh.n_req;
-    TmapPack& tm = *reinterpret_cast<TmapPack*>(pack0 + sizeof(TmapPack) * static_cast<size_t>(r0 / kMapChunk));
+    Pack& tm = *reinterpret_cast<Pack*>(pack0 + sizeof(Pack) * static_cast<size_t>(r0 / kMapChunk));
     for (int r = r0; r < r1 && !reuse; ++r) {
       {
         const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(sh.n_q_heads),
@@ -857,5 +883,7 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
   }
   return cudaSuccess;
 }
+
+}  // namespace
 
 }  // namespace akv
