@@ -13,7 +13,9 @@
 // invariants and brute force. Parity unpinned by the paper: the width T of the
 // cosine transition band and the default values of rho and alpha (the paper gives
 // the shape "cosine" and the ranges only); the conventions are documented at
-// akvo_sss below.
+// akvo_sss below. Also unpinned by the paper: the selection-spread statistic
+// (akvo_selection_spread), for which the paper has a figure and no formula; its
+// arithmetic is pinned against numpy's histogram and closed forms all the same.
 
 #include <algorithm>
 #include <cmath>
