@@ -45,3 +45,27 @@ def test_random_shape(B, case):
     ties = check_against_oracle(w, g)
     heads = spec.n_layers * spec.n_kv_heads * len(spec.seq_lens)
     assert ties <= 4 * heads, (spec, ties)
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_random_shape_paged(B, case):
+    """The same draws with K and V in a pool of pages of a random size (bf16 and fp32): identical to the contiguous run."""
+    from test_gpu_paged import run_paged
+    spec = draw(100 + case)
+    w = wl.generate(spec, seed=case)
+    ref = run_evict(B, w)
+    g = run_paged(B, w, int(np.random.default_rng(case).choice([16, 32, 64, 128])))
+    assert g["status"] == 0
+    for key in ("budgets", "cu", "kept", "k_out", "v_out"):
+        assert np.array_equal(g[key], ref[key]), key
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_random_shape_reevict(B, case):
+    """Random compacted caches (per-head lengths, decoded tokens, element type) against the oracle head by head."""
+    from test_gpu_reevict import check_heads, run_reevict
+    spec = draw(200 + case)
+    rng = np.random.default_rng(case)
+    c = wl.compacted_cache(spec, n_new=int(rng.integers(spec.window, 200)), seed=case, spread=float(rng.uniform(0.0, 0.8)))
+    g = run_reevict(B, c)
+    assert check_heads(c, g) <= 4 * len(c.new_budgets)
