@@ -40,8 +40,8 @@ def measured_peaks():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on the benchmark workload, from
 # the ncu capture summarised in profiles/score_umma_c2.md and profiles/sss_select_gather_c2.md (ncu flushes the
 # caches before each kernel, so the column-sum sweep's K re-read counts in full). Only valid for config 1, all layers.
-NCU_TRAFFIC_BYTES = {"score_umma_stats": 254286080, "score_umma_colsum": 262274816, "sss_select": 3874304,
-                     "gather": 334588416}
+NCU_TRAFFIC_BYTES = {"score_umma_stats": 254511360, "score_umma_colsum": 251568896, "sss_select": 3869696,
+                     "gather": 331371264}
 
 
 class ClockSampler:
