@@ -109,6 +109,10 @@ typedef struct {
 
 /* ---- host-side helpers (no GPU work) ------------------------------------------------ */
 
+/* sizeof(audiokv_params) as the library was built: a binding in another language compares
+ * it with the size of its own copy of the struct before the first call. */
+size_t audiokv_params_size(void);
+
 /* Text for a status code. Never NULL. */
 const char* audiokv_strerror(int status);
 

@@ -61,6 +61,11 @@ def lib() -> ctypes.CDLL:
         L = ctypes.CDLL(LIB_PATH)
         vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
         pp = ctypes.POINTER(audiokv_params)
+        L.audiokv_params_size.restype = sz
+        L.audiokv_params_size.argtypes = []
+        if L.audiokv_params_size() != ctypes.sizeof(audiokv_params):
+            raise RuntimeError(f"audiokv_params is {L.audiokv_params_size()} bytes in {LIB_PATH} and "
+                               f"{ctypes.sizeof(audiokv_params)} in this binding: rebuild the library")
         L.audiokv_strerror.restype = ctypes.c_char_p
         L.audiokv_strerror.argtypes = [ctypes.c_int]
         L.audiokv_budget_from_ratio.restype = i64

@@ -562,6 +562,8 @@ int do_select_gather(audiokv_ctx* ctx, const float* smoothed, const int32_t* bud
 
 extern "C" {
 
+size_t audiokv_params_size(void) { return sizeof(audiokv_params); }
+
 const char* audiokv_strerror(int status) {
   switch (status) {
     case AUDIOKV_OK: return "ok";

@@ -28,6 +28,14 @@ def test_exports_every_declared_symbol(B):
         assert hasattr(L, n), f"{n} declared in audiokv.h but not exported"
 
 
+def test_params_struct_matches_the_library(B):
+    import ctypes
+    assert B.lib().audiokv_params_size() == ctypes.sizeof(B.audiokv_params)
+    # field offsets follow the C layout rules: the last field ends the struct (up to alignment padding)
+    last = B.audiokv_params.page_table_stride
+    assert last.offset + last.size == ctypes.sizeof(B.audiokv_params)
+
+
 def test_budget_from_ratio(B):
     assert B.audiokv_budget_from_ratio(0.4, 112, 8192, 32) == int(0.4 * 112 * 8192)
     assert B.audiokv_budget_from_ratio(0.0, 10, 100, 8) == 80          # never below the windows
