@@ -227,8 +227,14 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
 
 /* Same pass with every buffer in HOST memory (pageable or pinned): copies the inputs to
  * the device (into the workspace, which must have been sized with
- * audiokv_workspace_bytes_host), runs audiokv_evict, copies kept_idx, budgets, cu_kept,
- * k_out and v_out back and waits for the stream. q/k/v extents are given in elements. */
+ * audiokv_workspace_bytes_host), runs the pass, copies kept_idx, budgets, cu_kept,
+ * k_out and v_out back and waits for the stream. q/k/v extents are given in elements.
+ * One bf16 request whose K and V are laid out layer by layer (kv_elems = n_layers *
+ * kv_stride_layer) is processed in chunks of layers on three streams of the context, so
+ * that copies in, kernels and copies out overlap; when v is pinned memory the device can
+ * address, the kept V rows are read from it in place and the rest of V is never copied.
+ * Results do not depend on the route taken. Paged K/V (page_size != 0) is not accepted
+ * here (AUDIOKV_EUNSUPPORTED): the page table is device data. */
 int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, int64_t q_elems, const void* k,
                        const void* v, int64_t kv_elems, const float* head_scores, const int64_t* total_budget,
                        void* k_out, void* v_out, int32_t* kept_idx, int32_t* budgets, int32_t* cu_kept,
