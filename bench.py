@@ -316,12 +316,17 @@ def run_e2e(B, ctx, prob, w, spec, tb, rows, TH, es, barrier, world, args):
 
     step_host()
     barrier()
+    # three groups of up to five calls, the median group: the host side of this leg (pinned-memory traffic, the link)
+    # is shared with whatever else runs on the machine, and one disturbed group should not be the number
     n_e2e = max(1, min(args.steps, 5))
-    t0 = time.perf_counter()
-    for _ in range(n_e2e):
-        step_host()
-    barrier()
-    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / n_e2e, world, "cuda")
+    groups = []
+    for _ in range(3):
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            step_host()
+        barrier()
+        groups.append(max_over_ranks((time.perf_counter() - t0) * 1e3 / n_e2e, world, "cuda"))
+    e2e_ms = sorted(groups)[1]
     # V is pinned: the gather fetches its kept rows from the host buffer itself, the other rows never cross the link
     h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hS)) + hvo.numel() * hvo.element_size()
     d2h = sum(x.numel() * x.element_size() for x in (hko, hvo, hkept, hb, hcu))
