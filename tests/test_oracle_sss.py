@@ -8,8 +8,8 @@ import oracle
 
 
 def _sizes():
-    # every n up to 64 (primes, odd, even), then a spread up to 512 incl. primes and prime squares
-    return list(range(1, 65)) + [97, 121, 127, 128, 169, 210, 243, 256, 257, 289, 360, 385, 499, 509, 510, 511, 512]
+    # every n up to 512: all primes, prime powers, odd and even lengths in that range
+    return list(range(1, 513))
 
 
 @pytest.mark.parametrize("n", _sizes())
@@ -36,10 +36,14 @@ def test_dft_of_a_shifted_impulse():
     assert np.abs(oracle.rfft(x, direct=True) - want).max() < 1e-14
 
 
-@pytest.mark.parametrize("n", [8160, 992, 4099])
+# the prefix lengths of the workloads: L - 32 for L = 8192, 1024, 16384, 32768 (W = 16, 32), and the ragged batch's
+# lengths (among them the odd prime 15227 and lengths with a large prime factor), plus a prime above 4096
+@pytest.mark.parametrize("n", [8160, 992, 4099, 16352, 32736, 32752, 11536, 8572, 15227, 4753, 19192, 5644, 9081, 11878])
 def test_full_size_fast_dft_against_numpy(n):
     x = np.random.default_rng(0).standard_normal(n)
-    assert np.abs(oracle.rfft(x) - np.fft.rfft(x)).max() < 1e-9
+    F = np.fft.rfft(x)
+    assert np.abs(oracle.rfft(x) - F).max() < 1e-9
+    assert np.abs(oracle.irfft(F, n) - x).max() < 1e-11
 
 
 @pytest.mark.parametrize("n", [31, 32, 257, 600])
