@@ -225,6 +225,12 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
                   const float* head_scores, const int64_t* total_budget, void* k_out, void* v_out,
                   int32_t* kept_idx, int32_t* budgets, int32_t* cu_kept, audiokv_stream stream);
 
+/* The cut-offs k* of step 2 as the last audiokv_evict / audiokv_evict_budgeted / audiokv_reevict call on
+ * this context found them (Section 3.3, the smallest k with E(k) >= rho E(n/2); 0 for the pooling
+ * variants): a copy of the context's own record, ordered on `stream` behind that call.
+ * kstar: device int32 [total heads]. AUDIOKV_EINVAL before the first pass on the context. */
+int audiokv_evict_kstar(audiokv_ctx* ctx, int32_t* kstar, audiokv_stream stream);
+
 /* Same pass with every buffer in HOST memory (pageable or pinned): copies the inputs to
  * the device (into the workspace, which must have been sized with
  * audiokv_workspace_bytes_host), runs the pass, copies kept_idx, budgets, cu_kept,

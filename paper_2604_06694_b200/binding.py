@@ -98,6 +98,8 @@ def lib() -> ctypes.CDLL:
         L.audiokv_allocate.argtypes = [vp, pp, vp, ctypes.POINTER(i64), vp, vp, vp]
         L.audiokv_select_gather.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.audiokv_evict.argtypes = [vp, pp, vp, vp, vp, vp, ctypes.POINTER(i64), vp, vp, vp, vp, vp, vp]
+        L.audiokv_evict_kstar.argtypes = [vp, vp, vp]
+        L.audiokv_evict_kstar.restype = ctypes.c_int
         L.audiokv_evict_budgeted.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.audiokv_evict_budgeted.restype = ctypes.c_int
         L.audiokv_reevict_workspace_bytes.restype = sz
@@ -299,6 +301,11 @@ def audiokv_evict(ctx: Context, prob: Problem, q_win, k, v, head_scores, total_b
                                    _dev(head_scores, "head_scores"), _budget_array(total_budget), _dev(k_out, "k_out"),
                                    _dev(v_out, "v_out"), _dev(kept_idx, "kept_idx"), _dev(budgets, "budgets"),
                                    _dev(cu_kept, "cu_kept"), _stream()), "audiokv_evict")
+
+
+def audiokv_evict_kstar(ctx: Context, kstar: torch.Tensor) -> None:
+    """kstar: CUDA int32 [total heads], receives the cut-offs of the context's last pass."""
+    ctx._check(lib().audiokv_evict_kstar(ctx.h, _dev(kstar, "kstar"), _stream()), "audiokv_evict_kstar")
 
 
 def audiokv_evict_budgeted(ctx: Context, prob: Problem, q_win, k, v, budgets, k_out, v_out, kept_idx, cu_kept) -> None:

@@ -797,6 +797,16 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
   return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, s);
 }
 
+int audiokv_evict_kstar(audiokv_ctx* ctx, int32_t* kstar, audiokv_stream stream) {
+  if (!ctx || !kstar) return AUDIOKV_EINVAL;
+  if (!ctx->plan.valid || !ctx->plan_uploaded) return AUDIOKV_EINVAL;  // no pass has run on this context yet
+  cudaError_t e = cudaSetDevice(ctx->device);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  e = cudaMemcpyAsync(kstar, ctx->ws + ctx->plan.lay.kstar, sizeof(int32_t) * ctx->plan.sh.total_heads,
+                      cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
+}
+
 int audiokv_evict_budgeted(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, const void* k, const void* v,
                            const int32_t* budgets, void* k_out, void* v_out, int32_t* kept_idx, int32_t* cu_kept,
                            audiokv_stream stream) {

@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(kThreads) score_simt_kernel(Shape sh, const Re
   float* rowA = Zt + kTile * (kTile + 1);  // sweep 1: running max; sweep 2: max + log2 sum
   float* rowB = rowA + sh.window * sh.group;  // sweep 1: running sum; sweep 2: partial column sums [4][kTile]
 
-  const int u = blockIdx.y, slab = blockIdx.x;
+  const int u = blockIdx.x / n_slab, slab = blockIdx.x - u * n_slab;  // one block per (head, slab), heads outermost
   const HeadCoord hc = head_coord(sh, u);
   const ReqDesc rq = reqs[hc.r];
   const int R = sh.window * sh.group, G = sh.group;
@@ -210,7 +210,8 @@ cudaError_t launch_typed(const Shape& sh, const ReqDesc* d_reqs, const void* q, 
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-  dim3 grid(n_slab, sh.total_heads);
+  if (static_cast<int64_t>(n_slab) * sh.total_heads > 0x7fffffffLL) return cudaErrorNotSupported;
+  dim3 grid(static_cast<unsigned>(n_slab) * static_cast<unsigned>(sh.total_heads));
   k1<<<grid, kThreads, smem, ln.stream>>>(sh, d_reqs, (const T*)q, (const T*)k, scores, stats_ws, n_slab, slab_keys);
   ln.done("score_simt_stats");
   k2<<<grid, kThreads, smem, ln.stream>>>(sh, d_reqs, (const T*)q, (const T*)k, scores, stats_ws, n_slab, slab_keys);
@@ -262,6 +263,16 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 std::mutex g_noalloc_mu;
 void* g_noalloc_ptr[kNoAllocMaxDevices] = {};  // device address of the array, per device ordinal
 
+// The request table reaches the scratch as a kernel argument (2.5 KB, copied at launch): no host
+// buffer has to outlive the call.
+constexpr int kNoAllocMaxReq = 64;
+struct NoAllocTable {
+  ReqDesc r[kNoAllocMaxReq];
+};
+__global__ void noalloc_table_kernel(const NoAllocTable t, int n, ReqDesc* dst) {
+  if (threadIdx.x < n) dst[threadIdx.x] = t.r[threadIdx.x];
+}
+
 // The array's name is only a host-side handle; kernels need the address the runtime reports
 // for the current device.
 cudaError_t noalloc_scratch(int device, void** out) {
@@ -286,13 +297,13 @@ extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const 
   if (device < 0 || device >= kNoAllocMaxDevices) return AUDIOKV_EINVAL;
   if (p->dtype != AUDIOKV_F32 && p->dtype != AUDIOKV_BF16) return AUDIOKV_EINVAL;
   if (p->n_layers < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads) return AUDIOKV_EINVAL;
-  constexpr int kNoAllocMaxReq = 64;  // the request table has a fixed slot in the static scratch
   if (p->n_req < 1 || p->n_req > kNoAllocMaxReq || p->window < 1) return AUDIOKV_EINVAL;
   if (p->head_dim != 64 && p->head_dim != 128 && p->head_dim != 256) return AUDIOKV_EUNSUPPORTED;
   if (p->page_size != 0) return AUDIOKV_EUNSUPPORTED;  // contiguous K only
   const int G = p->n_q_heads / p->n_kv_heads;
   const int64_t R = static_cast<int64_t>(p->window) * G;
   if (R > 1024) return AUDIOKV_EUNSUPPORTED;
+  if (static_cast<int64_t>(p->n_layers) * p->n_kv_heads > 2048) return AUDIOKV_EUNSUPPORTED;  // as audiokv_score
   const int per16 = p->dtype == AUDIOKV_F32 ? 4 : 8;
   const int64_t strides[] = {p->q_stride_req, p->q_stride_layer, p->q_stride_tok, p->q_stride_head,
                              p->kv_stride_layer, p->kv_stride_tok, p->kv_stride_head};
@@ -323,7 +334,8 @@ extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const 
   sh.softmax_scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(static_cast<float>(p->head_dim));
   sh.scale_log2e = static_cast<float>(static_cast<double>(sh.softmax_scale) * 1.4426950408889634);
 
-  ReqDesc reqs[kNoAllocMaxReq];
+  NoAllocTable table{};
+  ReqDesc* reqs = table.r;
   int max_L = 0;
   int64_t score_off = 0;
   for (int r = 0; r < p->n_req; ++r) {
@@ -348,9 +360,8 @@ extern "C" int audiokv_score_noalloc(int device, const audiokv_params* p, const 
   void* base = nullptr;
   if (noalloc_scratch(device, &base) != cudaSuccess) return AUDIOKV_ECUDA;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // The table is staged by the runtime before this returns, so the local array may go out of scope.
-  if (cudaMemcpyAsync(base, reqs, sizeof(ReqDesc) * p->n_req, cudaMemcpyHostToDevice, s) != cudaSuccess)
-    return AUDIOKV_ECUDA;
+  noalloc_table_kernel<<<1, kNoAllocMaxReq, 0, s>>>(table, p->n_req, static_cast<ReqDesc*>(base));
+  if (cudaGetLastError() != cudaSuccess) return AUDIOKV_ECUDA;
   int64_t launches = 0;
   Launch ln{s, &launches, nullptr};
   // Sweep 1 writes every statistics entry that sweep 2 reads, so nothing has to start at zero.

@@ -64,6 +64,52 @@ def test_score_parity(B, name, make):
     assert ctx.last_device_status() == 0
 
 
+# The long lengths, one layer each: 256 key tiles per head at L = 32768 (G = 7, so 224 query rows per head, and
+# W = 64 with 448), a d = 256 head at L = 19224 (the longest request of the ragged batch), and L = 131072.
+LONG_SCORE_CASES = [
+    ("c3_L32768_w32", lambda: wl.generate(wl.config(2), layers=1)),
+    ("c3_L32768_w64", lambda: wl.generate(dataclasses.replace(wl.config(2), window=64, n_kv_heads=2, n_q_heads=14), layers=1)),
+    ("c4_L16384_sinks", lambda: wl.generate(wl.config(3), layers=1)),
+    ("d256_L19224", lambda: wl.generate(dataclasses.replace(wl.config(4), seq_lens=(19224,), audio_frac=(0.9,)), layers=1)),
+    ("L131072_one_head", lambda: wl.generate(dataclasses.replace(wl.config(1), seq_lens=(131072,), audio_frac=(0.9,),
+                                                                 n_q_heads=7, n_kv_heads=1), layers=1)),
+]
+
+
+@pytest.mark.parametrize("name,make", LONG_SCORE_CASES, ids=[c[0] for c in LONG_SCORE_CASES])
+def test_score_and_smooth_parity_at_full_length(B, name, make):
+    """Element by element at the lengths the fused tests only see through kept sets: the scores against the oracle's,
+    then audiokv_smooth on the GPU's own scores against the oracle's smoothing of the same vector."""
+    w = make()
+    s = w.spec
+    prob = B.Problem.from_workload(w)
+    ctx = B.Context(prob)
+    scores = torch.full((B.audiokv_scores_len(prob),), float("nan"), device="cuda")
+    B.audiokv_score(ctx, prob, to_dev(w, w.q), to_dev(w, w.k), scores)
+    out = torch.empty_like(scores)
+    kstar = torch.full((prob.total_heads,), -1, dtype=torch.int32, device="cuda")
+    B.audiokv_smooth(ctx, prob, scores, out, kstar)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    g, gs, gk = scores.cpu().numpy(), out.cpu().numpy(), kstar.cpu().numpy()
+    o, wm = oracle_scores(w, 0)
+    P = s.seq_lens[0] - s.window
+    G = s.n_q_heads // s.n_kv_heads
+    worst = 0.0
+    for h in range(s.n_kv_heads):
+        gh = g[h * P:(h + 1) * P]
+        worst = max(worst, rel_err(gh, o[0, h]))
+        assert rel_err(gh, o[0, h]) <= REL_TOL, (name, h)
+        assert abs(gh.sum(dtype=np.float64) + wm[0, h] - s.window * G) <= 2e-4 * s.window * G
+        rho, alpha = float(np.float32(s.rho)), float(np.float32(s.alpha))
+        want, ko, margin = oracle.sss(gh.astype(np.float64), rho, alpha, s.transition_bins)
+        if gk[h] != ko:
+            assert margin < KSTAR_TIE, (name, h, gk[h], ko, margin)
+            want, _, _ = oracle.sss(gh.astype(np.float64), rho, alpha, s.transition_bins, force_kstar=int(gk[h]))
+        assert rel_err(gs[h * P:(h + 1) * P], want) <= REL_TOL, (name, h)
+    print(f"{name}: worst score error {worst:.2e}")
+
+
 def _score_like(rng, n, kind):
     if kind == "lognormal":
         x = np.exp(rng.standard_normal(n)) * 0.02

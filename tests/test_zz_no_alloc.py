@@ -1,4 +1,4 @@
-"""The allocation-free scoring entry point against the regular one.
+"""The allocation-free scoring entry point against the regular one and against the CPU oracle.
 
 audiokv_score_noalloc serves callers that are not allowed to allocate device memory while they run
 (a serving process whose memory pool is frozen, a plug-in without an allocator); its scratch is a
@@ -10,7 +10,7 @@ import pytest
 import torch
 
 from paper_2604_06694_b200 import workloads as wl
-from helpers import REL_TOL, rel_err, to_dev
+from helpers import REL_TOL, oracle_scores, rel_err, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -45,10 +45,13 @@ def test_two_calls_in_a_row_match_the_regular_entry_point(B):
         assert np.isfinite(got).all()
         s = w.spec
         off = 0
-        for L in s.seq_lens:
+        for r, L in enumerate(s.seq_lens):
             P = L - s.window
-            for _ in range(s.n_layers * s.n_kv_heads):
+            want, _ = oracle_scores(w, r)              # the CPU oracle's scores of this request, fp64
+            want = want.reshape(-1, P)
+            for u in range(s.n_layers * s.n_kv_heads):
                 assert rel_err(got[off:off + P], ref[off:off + P]) <= REL_TOL
+                assert rel_err(got[off:off + P], want[u]) <= REL_TOL
                 off += P
         assert off == got.size
 
