@@ -151,8 +151,9 @@ int audiokv_create(audiokv_ctx** ctx, int device, size_t workspace_bytes);
 /* Frees the workspace. The caller makes sure no call on this context is still running. */
 int audiokv_destroy(audiokv_ctx* ctx);
 
-/* The status word the kernels write (0, AUDIOKV_ETIMEOUT or AUDIOKV_EDEVICE). Synchronises
- * with the work of earlier calls by a blocking copy on `stream`. */
+/* The status word the kernels write (0, AUDIOKV_ETIMEOUT, AUDIOKV_EDEVICE or, from
+ * audiokv_evict_budgeted, AUDIOKV_EINVAL). Synchronises with the work of earlier calls by a
+ * blocking copy on `stream`; a non-zero status is reported once and the word is cleared. */
 int audiokv_last_device_status(audiokv_ctx* ctx, audiokv_stream stream);
 
 /* Text of the last CUDA error a call on this context met (empty string if none). */
@@ -160,6 +161,21 @@ const char* audiokv_last_cuda_error(const audiokv_ctx* ctx);
 
 /* Kernels launched by calls on this context since it was created (for accounting). */
 int64_t audiokv_launch_count(const audiokv_ctx* ctx);
+
+/* Which kernels the last scoring on this context ran on (audiokv_score, or step 1 inside audiokv_evict and
+ * its variants): "tcgen05" = the tensor-core kernels (bf16 inputs), "fma" = the fp32 FMA kernels (fp32
+ * inputs, which are never rounded to TF32; a GQA group of more than 256 query heads; row strides the copy
+ * engine cannot express), "none" before the first scoring. Never NULL. */
+const char* audiokv_last_score_path(const audiokv_ctx* ctx);
+
+/* Limit of the waits inside the tensor-core scoring kernels (the paper has no counterpart: this is the
+ * library's guard against a wait that never ends). Every wait of a warp on a barrier of its CTA gives up
+ * after `cycles` SM clock cycles (default 2e9, about a second): the CTA then stops, lets its copies and
+ * tensor-core operations in flight finish, releases its tensor memory, and the kernel writes
+ * AUDIOKV_ETIMEOUT to the status word; the call's outputs are then undefined and the context stays usable.
+ * Process-wide, read at each launch; cycles <= 0 restores the default. Returns the previous limit. Meant for
+ * deployments that want a shorter guard and for the test that makes a wait run out. */
+int64_t audiokv_set_wait_limit(int64_t cycles);
 
 /* Per-kernel timing of audiokv_evict, for benchmarks. While enabled, every audiokv_evict call
  * on this context records a CUDA event on its stream after each kernel it launches (creating

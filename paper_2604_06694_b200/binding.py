@@ -83,6 +83,10 @@ def lib() -> ctypes.CDLL:
         L.audiokv_last_cuda_error.argtypes = [vp]
         L.audiokv_launch_count.restype = i64
         L.audiokv_launch_count.argtypes = [vp]
+        L.audiokv_last_score_path.argtypes = [vp]
+        L.audiokv_last_score_path.restype = ctypes.c_char_p
+        L.audiokv_set_wait_limit.argtypes = [i64]
+        L.audiokv_set_wait_limit.restype = i64
         L.audiokv_profile_enable.argtypes = [vp, ctypes.c_int]
         L.audiokv_profile_enable.restype = ctypes.c_int
         L.audiokv_profile_count.argtypes = [vp]
@@ -184,6 +188,11 @@ def audiokv_budget_from_ratio(c: float, n_heads_total: int, seq_len: int, window
     return int(lib().audiokv_budget_from_ratio(c, n_heads_total, seq_len, window))
 
 
+def audiokv_set_wait_limit(cycles: int) -> int:
+    """Limit (SM clock cycles) of the waits inside the scoring kernels; <= 0 restores the default. Returns the old one."""
+    return int(lib().audiokv_set_wait_limit(int(cycles)))
+
+
 def audiokv_scores_len(prob: Problem) -> int:
     return int(lib().audiokv_scores_len(prob.ref))
 
@@ -248,6 +257,10 @@ class Context:
         n = lib().audiokv_profile_count(self.h)
         return [(lib().audiokv_profile_name(self.h, i).decode(), float(lib().audiokv_profile_ms(self.h, i)))
                 for i in range(n)]
+
+    def last_score_path(self) -> str:
+        """"tcgen05", "fma" or "none": the kernels the last scoring on this context ran on."""
+        return lib().audiokv_last_score_path(self.h).decode()
 
     def last_device_status(self) -> int:
         return int(lib().audiokv_last_device_status(self.h, _stream()))

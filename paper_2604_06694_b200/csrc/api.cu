@@ -19,11 +19,12 @@ constexpr int kSssSmemComplex = 25600;  // 200 KB of float2: the largest work bu
 constexpr int kSlabKeys = 256;          // keys per slab of the softmax statistics (two K tiles of the tensor-core kernel)
 constexpr int kMaxRows = 1024;          // W * G
 constexpr int kMaxHeadsPerReq = 2048;
+constexpr int kHostChunks = 8;          // the host-buffer call evicts one request in at most this many runs of layers
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {  // byte offsets inside the workspace
-  size_t status, reqs, plans, tables, units, order, stats, fft_scratch, scores, kstar, aux, end;
+  size_t status, reqs, plans, tables, units, ctas, order, stats, fft_scratch, scores, kstar, aux, end;
 };
 
 struct Plan {
@@ -34,9 +35,10 @@ struct Plan {
   Shape sh{};
   std::vector<ReqDesc> reqs;
   std::vector<FftPlan> fft;
-  std::vector<ScoreUnit> units;   // sweep 1 (all keys, ascending) then sweep 2 (prefix keys, descending)
-  int n_units1 = 0, n_units2 = 0;
-  std::vector<int> unit_pre1, unit_pre2;  // [n_req + 1]: units of the requests before r, per sweep
+  std::vector<ScoreUnit> units;          // runs of the tensor-core scoring: both sweeps of every schedule
+  std::vector<int32_t> score_ctas;       // per-CTA run offsets of every (schedule, sweep)
+  std::vector<ScoreSchedule> schedules;  // one per run of requests, plus one per chunk of layers of a single request
+  int score_parts = 1;                   // statistics slots per head of the tensor-core scoring
   std::vector<int32_t> sss_order;  // heads in the order the smoothing blocks take them (see build_plan); -1 = none
   int64_t table_len = 0;        // float2 elements
   int64_t scores_len = 0;
@@ -68,10 +70,11 @@ struct audiokv_ctx {
   cudaStream_t side = nullptr;            // audiokv_evict runs the allocation here, beside the scoring
   cudaEvent_t fork = nullptr, join = nullptr;
   // audiokv_evict_host: copies in on `side`, kernels on the caller's stream, copies out on `out`, chunk by chunk
-  static constexpr int kMaxChunks = 8;
+  static constexpr int kMaxChunks = kHostChunks;
   cudaStream_t out = nullptr;
   cudaEvent_t chunk_in[kMaxChunks] = {}, chunk_done[kMaxChunks] = {}, copies_out = nullptr;
   int64_t launches = 0;
+  int score_path = 0;  // route of the last scoring: 0 none yet, 1 tensor cores, 2 fp32 FMA
   Profiler prof;
   std::string cuda_error;
   ReevictArrays re;  // audiokv_reevict: the per-head problem it hands to the eviction pass
@@ -242,6 +245,106 @@ void build_fft_plan(int n, FftPlan* fp, int64_t* table_len) {
   }
 }
 
+int host_chunks(int n_layers) { return n_layers < kHostChunks ? n_layers : kHostChunks; }
+int host_chunk_layer(int n_layers, int c) { return static_cast<int>(static_cast<int64_t>(n_layers) * c / host_chunks(n_layers)); }
+
+// Schedules of the tensor-core scoring. A schedule covers a set of heads; the key tiles of those heads, in the order
+// the sweep walks them, are dealt out evenly over the CTAs, CTA c taking tiles [c T / grid, (c + 1) T / grid): a few
+// runs of consecutive tiles of one head. Sweep 1 walks the heads in order over all L keys (the runs of a head number
+// its statistics slots); sweep 2 walks them backwards over the prefix keys (the heads sweep 1 touched last are the
+// ones still in L2).
+void build_score_schedules(const audiokv_params* p, Plan* pl) {
+  const Shape& sh = pl->sh;
+  pl->units.clear();
+  pl->score_ctas.clear();
+  pl->schedules.clear();
+  pl->score_parts = 1;
+  if (!score_umma_takes(sh)) return;
+  // a head whose W * G query rows exceed the kernel's Q tile is scored in chunks of window rows (runs of their own)
+  const int w_chunk = score_window_chunk(sh);
+  const int n_wchunks = (p->window + w_chunk - 1) / w_chunk;
+  std::vector<int32_t> parts_of(static_cast<size_t>(sh.total_heads) * n_wchunks, 0);
+  auto add = [&](bool whole, int r_begin, int r_end, int head_begin, int head_end) {
+    ScoreSchedule sc{};
+    sc.whole_requests = whole ? 1 : 0;
+    sc.r_begin = r_begin;
+    sc.r_end = r_end;
+    sc.head_begin = head_begin;
+    sc.head_end = head_end;
+    struct Q {
+      int u, r, hr, ch;
+    };
+    std::vector<Q> qs;  // the (head, window chunk) pairs of this schedule, in sweep-1 order
+    for (int r = r_begin; r < r_end; ++r)
+      for (int hr = whole ? 0 : head_begin; hr < (whole ? sh.heads_per_req : head_end); ++hr)
+        for (int ch = 0; ch < n_wchunks; ++ch) qs.push_back(Q{pl->reqs[r].head_base + hr, r, hr, ch});
+    for (int sweep = 1; sweep <= 2; ++sweep) {
+      if (sweep == 2) std::reverse(qs.begin(), qs.end());
+      int64_t total = 0;
+      for (const Q& x : qs) {
+        const int range = sweep == 1 ? pl->reqs[x.r].L : pl->reqs[x.r].P;
+        total += (range + 127) / 128;
+      }
+      const int grid = static_cast<int>(total < kScoreCtas ? total : kScoreCtas);
+      sc.unit_off[sweep - 1] = static_cast<int32_t>(pl->units.size());
+      sc.cta_off[sweep - 1] = static_cast<int32_t>(pl->score_ctas.size());
+      sc.grid[sweep - 1] = grid;
+      const size_t first = pl->units.size();
+      int64_t tile = 0;  // tiles before the current head in the sweep's sequence
+      int c = 0;         // CTA whose range holds the next tile
+      pl->score_ctas.push_back(0);
+      for (const Q& x : qs) {
+        const ReqDesc& d = pl->reqs[x.r];
+        const int range = sweep == 1 ? d.L : d.P;
+        const int n_tiles = (range + 127) / 128;
+        int t = 0, part = 0;
+        while (t < n_tiles) {
+          // the CTA that owns tile `tile + t`, and how far its range reaches into this head
+          while (c + 1 < grid && (static_cast<int64_t>(c + 1) * total) / grid <= tile + t) {
+            ++c;
+            pl->score_ctas.push_back(static_cast<int32_t>(pl->units.size() - first));
+          }
+          const int64_t c_end = (static_cast<int64_t>(c + 1) * total) / grid;
+          const int take = static_cast<int>(std::min<int64_t>(n_tiles - t, c_end - (tile + t)));
+          ScoreUnit un{};
+          un.u = x.u;
+          un.r = x.r;
+          un.l = x.hr / p->n_kv_heads;
+          un.h = x.hr % p->n_kv_heads;
+          un.part = part++;
+          un.kt0 = t * 128;
+          un.n_tiles = take;
+          un.P = d.P;
+          un.score_base = d.score_offset + static_cast<int64_t>(x.hr) * d.P;
+          un.w0 = x.ch * w_chunk;
+          un.wn = p->window - un.w0 < w_chunk ? p->window - un.w0 : w_chunk;
+          un.qid = x.u * n_wchunks + x.ch;
+          un.head_parts = 0;  // set below
+          pl->units.push_back(un);
+          t += take;
+        }
+        if (sweep == 1) {
+          parts_of[static_cast<size_t>(x.u) * n_wchunks + x.ch] = part;
+          pl->score_parts = part > pl->score_parts ? part : pl->score_parts;
+        }
+        tile += n_tiles;
+      }
+      while (static_cast<int>(pl->score_ctas.size()) - sc.cta_off[sweep - 1] < grid + 1)
+        pl->score_ctas.push_back(static_cast<int32_t>(pl->units.size() - first));
+      for (size_t i = first; i < pl->units.size(); ++i) pl->units[i].head_parts = parts_of[pl->units[i].qid];
+    }
+    pl->schedules.push_back(sc);
+  };
+  const int cap = score_map_chunk(p->n_req);
+  for (int r0 = 0; r0 < p->n_req; r0 += cap) add(true, r0, r0 + cap < p->n_req ? r0 + cap : p->n_req, 0, 0);
+  if (p->n_req == 1 && p->n_layers > 1) {
+    // the host-buffer call evicts one request in chunks of layers
+    const int n_chunks = host_chunks(p->n_layers);
+    for (int c = 0; c < n_chunks; ++c)
+      add(false, 0, 1, host_chunk_layer(p->n_layers, c) * p->n_kv_heads, host_chunk_layer(p->n_layers, c + 1) * p->n_kv_heads);
+  }
+}
+
 int build_plan(const audiokv_params* p, Plan* pl) {
   int rc = check_params(p);
   if (rc) return rc;
@@ -318,43 +421,10 @@ int build_plan(const audiokv_params* p, Plan* pl) {
     d.fft_plan = it->second;
   }
   pl->n_slab = (pl->max_L + kSlabKeys - 1) / kSlabKeys;
-  // Schedule of the tensor-core scoring: sweep 1 walks the heads in order; sweep 2 walks them backwards, since the
-  // heads sweep 1 touched last are the ones still in L2.
-  pl->units.clear();
-  for (int sweep = 1; sweep <= 2; ++sweep) {
-    const size_t first = pl->units.size();
-    std::vector<int>& pre = sweep == 1 ? pl->unit_pre1 : pl->unit_pre2;
-    pre.assign(p->n_req + 1, 0);
-    for (int r = 0; r < p->n_req; ++r) {
-      const ReqDesc& d = pl->reqs[r];
-      pre[r] = static_cast<int>(pl->units.size() - first);
-      const int range = sweep == 1 ? d.L : d.P;
-      const int slabs = (range + kSlabKeys - 1) / kSlabKeys;
-      for (int hr = 0; hr < sh.heads_per_req; ++hr)
-        for (int sl = 0; sl < slabs; ++sl) {
-          ScoreUnit un{};
-          un.u = d.head_base + hr;
-          un.r = r;
-          un.l = hr / p->n_kv_heads;
-          un.h = hr % p->n_kv_heads;
-          un.slab = sl;
-          un.kt0 = sl * kSlabKeys;
-          const int end = range < un.kt0 + kSlabKeys ? range : un.kt0 + kSlabKeys;
-          un.n_tiles = (end - un.kt0 + 127) / 128;
-          un.P = d.P;
-          un.score_base = d.score_offset + static_cast<int64_t>(hr) * d.P;
-          un.head_slabs = (d.L + kSlabKeys - 1) / kSlabKeys;
-          pl->units.push_back(un);
-        }
-    }
-    pre[p->n_req] = static_cast<int>(pl->units.size() - first);
-    if (sweep == 1) pl->n_units1 = static_cast<int>(pl->units.size());
-    else {
-      pl->n_units2 = static_cast<int>(pl->units.size() - first);
-      std::reverse(pl->units.begin() + first, pl->units.end());
-    }
-  }
-  pl->sss_grid = sh.total_heads < 148 ? sh.total_heads : 148;
+  build_score_schedules(p, pl);
+  // one block per head at a time, as many blocks as the planning SM count (the plan, and with it the workspace size,
+  // does not depend on the device)
+  pl->sss_grid = sh.total_heads < kScoreCtas ? sh.total_heads : kScoreCtas;
   {
     // Block b of the smoothing kernel takes entries b, b + grid, b + 2 grid, ... of this list. Heads are sorted by an
     // estimate of their transform's cost and dealt out in a snake (left to right, then right to left), so that
@@ -402,8 +472,13 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   L.plans = off;       off = align_up(off + sizeof(FftPlan) * pl->fft.size());
   L.tables = off;      off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->table_len));
   L.units = off;       off = align_up(off + sizeof(ScoreUnit) * pl->units.size());
+  L.ctas = off;        off = align_up(off + sizeof(int32_t) * pl->score_ctas.size());
   L.order = off;       off = align_up(off + sizeof(int32_t) * pl->sss_order.size());
-  L.stats = off;       off = align_up(off + sizeof(float2) * static_cast<size_t>(sh.total_heads) * pl->n_slab * sh.window * sh.group);
+  {
+    // softmax statistics: [head][slab][row] for the FMA kernels, [head][part][group][row] for the tensor-core ones
+    const size_t slots = std::max<size_t>(pl->n_slab, static_cast<size_t>(pl->score_parts) * 2);
+    L.stats = off;     off = align_up(off + sizeof(float2) * static_cast<size_t>(sh.total_heads) * slots * sh.window * sh.group);
+  }
   L.fft_scratch = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->scratch_per_block) * pl->sss_grid);
   L.scores = off;      off = align_up(off + sizeof(float) * static_cast<size_t>(pl->scores_len));
   L.kstar = off;       off = align_up(off + sizeof(int32_t) * static_cast<size_t>(sh.total_heads));
@@ -451,8 +526,11 @@ int prepare(audiokv_ctx* ctx, const audiokv_params* p, cudaStream_t stream) {
     if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.plans, pl.fft.data(), sizeof(FftPlan) * pl.fft.size(),
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess)
       return cuda_fail(ctx, e);
-    if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.units, pl.units.data(), sizeof(ScoreUnit) * pl.units.size(),
-                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+    if (!pl.units.empty() &&
+        ((e = cudaMemcpyAsync(ctx->ws + pl.lay.units, pl.units.data(), sizeof(ScoreUnit) * pl.units.size(),
+                              cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+         (e = cudaMemcpyAsync(ctx->ws + pl.lay.ctas, pl.score_ctas.data(), sizeof(int32_t) * pl.score_ctas.size(),
+                              cudaMemcpyHostToDevice, stream)) != cudaSuccess))
       return cuda_fail(ctx, e);
     if ((e = cudaMemcpyAsync(ctx->ws + pl.lay.order, pl.sss_order.data(), sizeof(int32_t) * pl.sss_order.size(),
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess)
@@ -492,14 +570,19 @@ int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cuda
   cudaError_t e = cudaErrorNotSupported;
   if (score_umma_takes(pl.sh))
   {
-    const ScoreUnit* units = reinterpret_cast<const ScoreUnit*>(ctx->ws + pl.lay.units);
-    e = launch_score_umma(pl.sh, pl.reqs.data(), units, pl.unit_pre1.data(), units + pl.n_units1, pl.unit_pre2.data(),
-                          q, k, scores, stats, pl.n_slab, kSlabKeys, d_status(ctx), ln, head_begin, head_end,
-                          &ctx->score_maps, ctx->plan_id);
+    e = launch_score_umma(pl.sh, pl.reqs.data(), reinterpret_cast<const ScoreUnit*>(ctx->ws + pl.lay.units),
+                          reinterpret_cast<const int32_t*>(ctx->ws + pl.lay.ctas), pl.schedules.data(),
+                          static_cast<int>(pl.schedules.size()), q, k, scores, stats, pl.score_parts, d_status(ctx), ln,
+                          head_begin, head_end, &ctx->score_maps, ctx->plan_id);
   }
   if (head_end >= 0 && e != cudaSuccess) return cuda_fail(ctx, e);  // no head ranges in the FMA kernel
-  if (e == cudaErrorNotSupported)  // fp32 inputs, W * G above 256, or strides the copy engine cannot take
+  ctx->score_path = 1;
+  if (e == cudaErrorNotSupported) {
+    // fp32 inputs (which must not be rounded to TF32), a GQA group above 256 query heads, or strides the copy
+    // engine cannot take; audiokv_last_score_path tells the caller which route ran
+    ctx->score_path = 2;
     e = launch_score_simt(pl.sh, d_reqs(ctx), q, k, scores, stats, pl.n_slab, kSlabKeys, ln);
+  }
   return e == cudaSuccess ? AUDIOKV_OK : cuda_fail(ctx, e);
 }
 
@@ -686,6 +769,7 @@ int audiokv_last_device_status(audiokv_ctx* ctx, audiokv_stream stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemcpyAsync(&st, ctx->ws, sizeof(int), cudaMemcpyDeviceToHost, s);  // first word of the workspace
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e == cudaSuccess && st != 0) e = cudaMemsetAsync(ctx->ws, 0, sizeof(int), s);  // reported once, then clean again
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return st;
 }
@@ -693,6 +777,17 @@ int audiokv_last_device_status(audiokv_ctx* ctx, audiokv_stream stream) {
 const char* audiokv_last_cuda_error(const audiokv_ctx* ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
 
 int64_t audiokv_launch_count(const audiokv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* audiokv_last_score_path(const audiokv_ctx* ctx) {
+  if (!ctx || ctx->score_path == 0) return "none";
+  return ctx->score_path == 1 ? "tcgen05" : "fma";
+}
+
+int64_t audiokv_set_wait_limit(int64_t cycles) {
+  const int64_t before = score_wait_cycles();
+  set_score_wait_cycles(cycles);
+  return before;
+}
 
 int audiokv_profile_enable(audiokv_ctx* ctx, int on) {
   if (!ctx) return AUDIOKV_EINVAL;
@@ -982,7 +1077,7 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
                        p->kv_stride_layer > 0 && kv_elems == static_cast<int64_t>(NL) * p->kv_stride_layer &&
                        p->kv_stride_layer >= p->kv_stride_tok * pl.reqs[0].L && p->kv_stride_layer >= p->kv_stride_head * Hkv;
   if (layered) {
-    const int n_chunks = NL < audiokv_ctx::kMaxChunks ? NL : audiokv_ctx::kMaxChunks;
+    const int n_chunks = host_chunks(NL);
     int32_t* d_budgets = reinterpret_cast<int32_t*>(db);
     int32_t* d_cu = reinterpret_cast<int32_t*>(dcu);
     AKV_CP(dq, q_win, q_elems * es, cudaMemcpyHostToDevice);
@@ -1012,8 +1107,7 @@ int audiokv_evict_host(audiokv_ctx* ctx, const audiokv_params* p, const void* q_
         cudaGetLastError();  // pageable memory is reported as an error by older drivers: not one of this call's
     }
     for (int c = 0; c < n_chunks; ++c) {
-      const int l0 = static_cast<int>(static_cast<int64_t>(NL) * c / n_chunks);
-      const int l1 = static_cast<int>(static_cast<int64_t>(NL) * (c + 1) / n_chunks);
+      const int l0 = host_chunk_layer(NL, c), l1 = host_chunk_layer(NL, c + 1);
       const size_t off = l0 * layer_bytes, len = (l1 - l0) * layer_bytes;
       AKV_CP_ON(ctx->side, dk + off, static_cast<const char*>(k) + off, len, cudaMemcpyHostToDevice);
       if (v_src == dv) AKV_CP_ON(ctx->side, dv + off, static_cast<const char*>(v) + off, len, cudaMemcpyHostToDevice);

@@ -94,6 +94,19 @@ struct FftPlan {
 // float2 slots of a shared-memory work buffer of `len` elements: element i sits at i + (i >> 4) (see SkewBuf in sss.cu)
 __host__ __device__ inline int sss_padded(int len) { return len + (len >> 4) + 1; }
 
+// SMs of the current device, asked once per device (grids of the bandwidth-bound kernels are sized by it).
+inline int device_sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 1;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 // ---- launchers (one per source file) ---------------------------------------------------
 // Optional per-kernel timing: an event after every kernel launch of one call.
 struct Profiler {
@@ -145,21 +158,46 @@ cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t
 cudaError_t launch_score_simt(const Shape& sh, const ReqDesc* d_reqs, const void* q, const void* k, float* scores,
                               float2* stats_ws, int n_slab, int slab_keys, Launch ln);
 
-// One unit of work of the tensor-core scoring kernel: one slab of one head. The schedule of each sweep is a
-// table of these, built on the host in processing order, so that no role of the kernel divides to find its work.
+// One run of work of the tensor-core scoring kernel: consecutive key tiles of one head (of one chunk of its window
+// rows) that one CTA processes. The schedule of each sweep is a table of these, built on the host in processing
+// order, so that no role of the kernel divides to find its work.
 struct ScoreUnit {
   int32_t u, r, l, h;              // flat head, request, layer, KV head
-  int32_t slab, kt0, n_tiles, P;   // slab number, first key, K tiles of 128 keys, prefix length of the request
+  int32_t part, kt0, n_tiles, P;   // statistics slot of the run (sweep 1), first key, K tiles of 128 keys, prefix length
   int64_t score_base;              // element offset of the head's scores in a packed score buffer
-  int32_t head_slabs;              // slabs of this head in the statistics buffer (all keys, window included)
-  int32_t pad;
+  int32_t head_parts;              // runs sweep 1 made of this head (statistics slots that sweep 2 merges)
+  int32_t w0, wn;                  // window rows [w0, w0 + wn) of the head: the query rows this run works on
+  int32_t qid;                     // u * (window chunks per head) + chunk: changes whenever another Q tile is needed
 };
 
-// score_umma.cu: bf16 scoring on the tcgen05 tensor cores (same statistics buffer). score_umma_takes says
-// whether the shape fits the kernel; the launcher returns cudaErrorNotSupported when the strides
-// cannot be described to the copy engine, and the caller then scores with launch_score_simt.
-// h_reqs: host copy of the request table (the tensor maps are encoded on the host).
+// One launch of the two sweeps: the heads it covers and where its runs lie in the device tables. CTA c of sweep s
+// takes the runs cta[c] .. cta[c + 1] - 1, cta = the grid[s] + 1 entries at cta_off[s] of the CTA table.
+struct ScoreSchedule {
+  int32_t whole_requests;          // 1: all heads of requests [r_begin, r_end); 0: heads [head_begin, head_end) of request 0
+  int32_t r_begin, r_end;
+  int32_t head_begin, head_end;
+  int32_t unit_off[2], cta_off[2], grid[2];
+};
+
+// CTAs the tiles of a launch are dealt out over (the SM count of the part this library is built for; fewer when there
+// are fewer tiles). A device with more SMs leaves some idle, one with fewer runs the CTAs in turn: no CTA waits for another.
+constexpr int kScoreCtas = 148;
+
+// Window rows per run of the tensor-core scoring: the largest share of the window whose W_c * G query rows fit the
+// kernel (256 rows; 128 at head_dim 256, where only a 128-row Q tile leaves room for two K stages), 0 if G alone
+// does not fit. A head whose W * G is larger is scored in ceil(W / W_c) chunks of window rows.
+int score_window_chunk(const Shape& sh);
+// Requests whose tensor maps travel with one launch (8 for a small batch, 120 for a long one).
+int score_map_chunk(int n_req);
+
+// score_umma.cu: bf16 scoring on the tcgen05 tensor cores. score_umma_takes says whether the shape fits the kernel;
+// the launcher returns cudaErrorNotSupported when the strides cannot be described to the copy engine, and the caller
+// then scores with launch_score_simt. h_reqs: host copy of the request table (the tensor maps are encoded on the host).
 bool score_umma_takes(const Shape& sh);
+// Limit, in SM clock cycles, of the waits on mbarriers inside the tensor-core scoring kernels (about one second by
+// default). A wait that runs out stops its CTA and the kernel reports AUDIOKV_ETIMEOUT. cycles <= 0 restores the default.
+void set_score_wait_cycles(long long cycles);
+long long score_wait_cycles();
 // The encoded tensor maps of the last call, kept by the context: encoding a few hundred maps costs more host time than
 // the kernels take on a short cache, and a serving loop calls with the same buffers and the same plan again and again.
 struct ScoreMapCache {
@@ -167,16 +205,16 @@ struct ScoreMapCache {
   const void* k = nullptr;
   uint64_t plan_id = 0;   // changes whenever the plan is rebuilt
   int page_size = -1;
-  std::vector<unsigned char> packs;  // one argument pack per launch chunk
+  std::vector<unsigned char> packs;   // one argument pack per run of requests
+  std::vector<unsigned char> encoded; // which of them hold maps of these buffers
 };
-// units1 / units2: device tables of the two sweeps (build_score_units gives their host form).
-// unit_pre1 / unit_pre2: host arrays [n_req + 1], units of the requests before r in either sweep.
-// head_begin / head_end (single request only): score the heads [head_begin, head_end) alone; -1 = all heads.
-cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
-                              const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
-                              float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
-                              int head_begin = 0, int head_end = -1, ScoreMapCache* cache = nullptr,
-                              uint64_t plan_id = 0);
+// d_units / d_cta: device tables of runs and per-CTA offsets (both sweeps of every schedule). scheds: host.
+// head_end < 0: every whole-request schedule in turn; else the schedule made for heads [head_begin, head_end).
+// stats_ws: float2 [total heads][max_parts][2][W * G].
+cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* d_units, const int32_t* d_cta,
+                              const ScoreSchedule* scheds, int n_sched, const void* q, const void* k, float* scores,
+                              float2* stats_ws, int max_parts, int* status, Launch ln, int head_begin = 0,
+                              int head_end = -1, ScoreMapCache* cache = nullptr, uint64_t plan_id = 0);
 
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);

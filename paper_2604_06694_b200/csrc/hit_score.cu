@@ -51,7 +51,8 @@ cudaError_t launch_hit_score(const float* attn, int n_steps, int n_heads, int64_
   cudaError_t e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * n_heads, ln.stream);
   if (e != cudaSuccess) return e;
   const int64_t n_pairs = static_cast<int64_t>(n_steps) * n_heads;
-  const int grid = static_cast<int>(n_pairs < 148 * 2 ? n_pairs : 148 * 2);
+  const int max_grid = device_sm_count() * 2;
+  const int grid = static_cast<int>(n_pairs < max_grid ? n_pairs : max_grid);
   hit_count_kernel<<<grid, kSelThreads, 0, ln.stream>>>(attn, n_steps, n_heads, row_stride, row_len, span, top_k, counts,
                                                         status);
   ln.done("hit_count");

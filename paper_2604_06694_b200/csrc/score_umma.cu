@@ -4,15 +4,27 @@
 // head, of softmax probabilities. A column sum mixes rows with different normalisers,
 // so the keys are swept twice:
 //   sweep 1  D[row][key]  = Q K^T  (query rows on the TMEM lanes): every thread owns one
-//            row and keeps its running maximum and sum of exp2 over the keys of a slab;
-//            one (max, sum) pair per (head, slab, row) goes to the statistics buffer.
+//            row (two, when W * G exceeds 128) and keeps a reference and a sum of exp2 over
+//            the keys of its tiles; one pair per (head, part, group, row) goes to the
+//            statistics buffer.
 //   sweep 2  D[key][row]  = K Q^T  (keys on the TMEM lanes): every thread owns one key
-//            and adds exp2(z - max - log2 sum) over the rows; no cross-thread reduction.
-// Both sweeps are one persistent kernel (one CTA per SM) with three roles:
-//   warp 16   TMA producer: the Q tile of a head once, K tiles of 128 keys through a ring;
-//   warp 17   MMA issuer: tcgen05.mma, bf16 x bf16 -> fp32 in TMEM, two accumulator buffers;
-//   warps 0-15 four groups of 128 threads that read the accumulators (tcgen05.ld) and do the
-//             softmax arithmetic.
+//            and adds exp2(z - max - log2 sum) over all rows; no cross-thread reduction.
+// Both sweeps are one persistent kernel with three roles:
+//   warps 0-7  two epilogue groups of four warps (one warp per TMEM lane quarter). The groups take the
+//              tiles of the CTA in turn (group g the tiles with parity g), each through accumulator
+//              buffers of its own, so that they depend on nothing but the MMA thread: no barrier
+//              joins them, nothing is exchanged through shared memory, and while one group waits,
+//              loads or stores, the other keeps the special-function unit busy;
+//   warp 8     TMA producer: the Q tile of a head once, K tiles of 128 keys through a ring;
+//   warps 9-10 MMA issuers, one thread per epilogue group: tcgen05.mma, bf16 x bf16 -> fp32 in TMEM. With one issuer
+//              for both groups the tiles were issued in order, and a group that had handed its buffers back waited
+//              for the MMAs of the other group's tile to be let in first.
+// A tile is processed in one or two parts (sweep 1: blocks of 128 query rows; sweep 2: halves of
+// the query rows), each with an accumulator buffer of 128 TMEM columns that goes back to the MMA
+// thread as soon as its last chunk is in registers: the MMAs of the group's next tile run under
+// the arithmetic of this one.
+// The work of a launch is dealt out tile by tile: CTA c takes the tiles [c T / grid, (c + 1) T / grid)
+// of the launch's tile sequence, as a few runs of consecutive tiles of one head (host-built table).
 // Q and K tiles are K-major with the 128-byte swizzle, so the same shared-memory tile is
 // the A operand of one sweep and the B operand of the other.
 // Every wait on an mbarrier is bounded: when one runs out the CTA stops, the kernel
@@ -20,20 +32,22 @@
 #include <cuda.h>
 #include <stddef.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace akv {
 namespace {
 
 constexpr int kTileKeys = 128;    // keys per K tile (UMMA M in sweep 2, N in sweep 1)
-constexpr int kEpiWarps = 16;      // four epilogue groups of four warps (one warp per TMEM lane quarter)
+constexpr int kEpiWarps = 8;      // two epilogue groups of four warps (one warp per TMEM lane quarter)
 constexpr int kProducerWarp = kEpiWarps;
-constexpr int kMmaWarp = kEpiWarps + 1;
-constexpr int kThreads = (kEpiWarps + 2) * 32;
-constexpr int kAccCols = 256;     // TMEM columns of one accumulator buffer
-constexpr uint32_t kTmemCols = 512;
+constexpr int kMmaWarp = kEpiWarps + 1;  // and the next one: an MMA thread per epilogue group
+constexpr int kThreads = (kEpiWarps + 3) * 32;
+constexpr uint32_t kTmemCols = 512;  // four accumulator buffers of 128 columns: [group][buffer]
 constexpr int kMaxStages = 8;
-constexpr long long kWaitCycles = 2000000000LL;  // about one second
+constexpr long long kWaitCycles = 2000000000LL;  // about one second: default limit of every wait on an mbarrier
+constexpr long long kDrainCycles = 200000000LL;  // limit of the waits of the stop path (copies and MMAs still in flight)
 constexpr int kSmemLimit = 232448;               // 227 KB
 
 // Tensor maps travel as kernel arguments, CAP requests' worth per launch. Two sizes: 8 for the usual small batch (the
@@ -49,30 +63,29 @@ struct TmapPack {
 
 struct UmmaArgs {
   Shape sh;
-  const ScoreUnit* units;  // this sweep's schedule, in processing order
+  const ScoreUnit* units;    // this sweep's runs, in processing order
+  const int32_t* cta_begin;  // [grid + 1]: CTA c takes the runs cta_begin[c] .. cta_begin[c + 1] - 1
   float2* stats;
   float* scores;
   int* status;
-  int n_slab;     // slabs per head in the statistics buffer
-  int slab_keys;  // keys per slab, a multiple of kTileKeys
-  int n_units;    // (head, slab) units of this sweep
+  int max_parts;  // statistics slots per head: [head][part][group][row]
   int q_rows;     // rows of the Q tile in shared memory: 128 or 256
-  int r_pad;      // W * G rounded up to 16
+  int r_pad;      // query rows of a Q tile rounded up to 16
   int n_stages;   // K ring depth
   int r0;         // first request of this launch: request r uses maps q[r - r0], k[r - r0]
+  int w_chunk;    // window rows of a run's Q tile (the whole window, or a share of it when W * G exceeds the tile)
+  int accumulate; // sweep 2: the head is scored in several chunks of window rows, whose column sums add up in `scores`
+  long long wait_cycles;  // limit of a wait on an mbarrier, in SM clock cycles
 };
 
 struct Small {
-  alignas(16) float negc[2][256];     // sweep 2: -(max + log2 sum) per row, by head parity (read 16 bytes at a time)
-  alignas(16) float2 mrg[2][3][128];  // sweep 1: partial statistics of the groups that share a row, by unit parity
-  alignas(16) float part[4][3][128];  // sweep 2: partial column sums of groups 1-3, by tile number mod 4
+  alignas(16) float negc[2][2][256];  // sweep 2: -(max + log2 sum) per row: [group][head parity][row]
   alignas(8) uint64_t k_full[kMaxStages];
   uint64_t k_empty[kMaxStages];
   uint64_t q_full, q_empty;
-  uint64_t acc_full[2][2], acc_empty[2][2];  // [group][buffer]: each epilogue group has its own accumulator stream
-  uint64_t all_bar;     // all epilogue threads (512 arrivals)
-  uint64_t part_full[4];  // sweep 2: the twelve warps of groups 1-3 have written part[i]
-  uint64_t drain;       // stop path only: the MMAs still in flight
+  uint64_t acc_full[2][2], acc_empty[2][2];  // [group][buffer]
+  uint64_t grp_bar[2];  // the 128 threads of a group (sweep 2: the rows' normalisers of a new head are in place)
+  uint64_t drain[2];    // stop path only: the MMAs of either issuer still in flight
   uint32_t tmem_base;
   int abort;
 };
@@ -91,6 +104,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// May suspend the thread, for a time of the hardware's choosing, until the phase completes. (An explicit suspend-time
+// hint was measured and made the sweeps a fifth slower: the default wake-up is the quicker one.)
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -104,14 +119,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait. Returns false when the CTA is stopping (this or another wait ran out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort,
-                                          long long limit = kWaitCycles) {
-  if (mbar_try_wait(bar, parity)) return true;
+// The same question without suspending the thread.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait. Returns false when the CTA is stopping (this or another wait ran out). try_wait may suspend the
+// thread for a time of the hardware's choosing before it answers, which is what a long wait wants; with a limit
+// shorter than such a suspension the barrier is polled instead, so that the limit is what ends the wait.
+constexpr long long kPollBelow = 1000000LL;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, long long limit) {
+  const bool poll = limit < kPollBelow;
+  if (poll ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 63u) == 0) {
+  while (!(poll ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity))) {
+    if (poll || (++spins & 15u) == 0) {  // a try_wait that comes back empty-handed has slept a while already
       if (*abort) return false;
       if (clock64() - t0 > limit) {
         *abort = 1;
@@ -120,6 +152,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
   return true;
+}
+// Wait of the stop path: the CTA is already stopping, so the flag is not consulted; bounded all the same.
+__device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity))
+    if (clock64() - t0 > kDrainCycles) return;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
@@ -201,6 +239,18 @@ __device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16
       : "r"(taddr)
       : "memory");
 }
+// The same for 16 columns, into the low half of a 32-register buffer.
+__device__ __forceinline__ void tmem_ld16_issue_lo(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+      : AKV_R8(r, 0), AKV_R8(r, 8)
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_lo(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" : AKV_RW8(r, 0), AKV_RW8(r, 8)::"memory");
+}
 __device__ __forceinline__ void tmem_wait(uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;\n" : AKV_RW8(r, 0), AKV_RW8(r, 8), AKV_RW8(r, 16), AKV_RW8(r, 24)::"memory");
 }
@@ -257,97 +307,155 @@ __device__ __forceinline__ float hsum(f32x2 a, f32x2 b, f32x2 c, f32x2 d) {
   return x + y;
 }
 
-// Sweep 1: N = NH * 32 logits of this thread's row (columns col0 .. col0 + N - 1 of the tile). Updates the
-// row's running maximum (raw dot products) and its sum of exp2 relative to that maximum.
-template <int NH>
-__device__ __forceinline__ void stats_part(uint32_t (&r)[NH][32], bool masked, int col0, int last_col, float sl,
-                                           float& m_run, float& Z) {
-  constexpr int N = NH * 32;
-  if (masked) {
-#pragma unroll
-    for (int i = 0; i < N; ++i)
-      if (col0 + i > last_col) r[i >> 5][i & 31] = 0xff800000u;  // -inf
-  }
-  float cm = __uint_as_float(r[0][0]);
-#pragma unroll
-  for (int i = 1; i + 1 < N; i += 2)
-    cm = max3(cm, __uint_as_float(r[i >> 5][i & 31]), __uint_as_float(r[(i + 1) >> 5][(i + 1) & 31]));
-  cm = fmaxf(cm, __uint_as_float(r[NH - 1][31]));
-  if (cm == -INFINITY) return;  // fully masked: adds nothing
-  const float m_new = fmaxf(m_run, cm);
-  const float rescale = ex2((m_run - m_new) * sl);  // first time: exp2(-inf) = 0
-  m_run = m_new;
-  const float nb = -m_new * sl;
-  const f32x2 sl2 = pack2(sl, sl), nb2 = pack2(nb, nb);
-  f32x2 a0 = pack2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
-#pragma unroll
-  for (int i = 0; i < N; i += 8) {
-    a0 = add2(a0, ex2_2(fma2(pack2(r[i >> 5][i & 31], r[i >> 5][(i & 31) + 1]), sl2, nb2)));
-    a1 = add2(a1, ex2_2(fma2(pack2(r[i >> 5][(i & 31) + 2], r[i >> 5][(i & 31) + 3]), sl2, nb2)));
-    a2 = add2(a2, ex2_2(fma2(pack2(r[i >> 5][(i & 31) + 4], r[i >> 5][(i & 31) + 5]), sl2, nb2)));
-    a3 = add2(a3, ex2_2(fma2(pack2(r[i >> 5][(i & 31) + 6], r[i >> 5][(i & 31) + 7]), sl2, nb2)));
-  }
-  Z = fmaf(Z, rescale, hsum(a0, a1, a2, a3));
+// exp2 on the FMA pipe, for a share of the exponentials: the special-function unit delivers 16 exp2 per clock and
+// SM and bounds both sweeps, while the FMA pipe has room. With t = round(x) + 1.5 * 2^23 (the integer lands in the low
+// mantissa bits), n = t - 1.5 * 2^23 and f = x - n in [-1/2, 1/2]: 2^x = 2^n p(f), p the cubic that minimises the
+// maximum relative error of 2^f on that interval (7.5e-5; rms 5e-5, well inside the 1e-3 the scores are held to),
+// and 2^n is an integer add into the exponent field. x must lie in [-125, 2^22).
+constexpr float kMagic = 12582912.f;  // 1.5 * 2^23
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
 }
-// One tile of sweep 1, NCH chunks of 32 columns: the next chunk's TMEM load runs under the arithmetic of this one.
-template <int NCH>
-__device__ __forceinline__ void stats_tile(uint32_t taddr, bool live, bool masked, int col0, int last_col, float sl,
-                                           float& m_run, float& Z) {
-  uint32_t ra[1][32], rb[1][32];
-  tmem_ld32_issue(taddr, ra[0]);
+// x and t = round(x) + kMagic, both halves
+__device__ __forceinline__ f32x2 ex2_poly(f32x2 x, f32x2 t) {
+  const f32x2 f = sub2(x, sub2(t, pack2(kMagic, kMagic)));
+  f32x2 p = fma2(f, pack2(5.5171664930e-02f, 5.5171664930e-02f), pack2(2.4261112188e-01f, 2.4261112188e-01f));
+  p = fma2(p, f, pack2(6.9326098622e-01f, 6.9326098622e-01f));
+  p = fma2(p, f, pack2(9.9992807358e-01f, 9.9992807358e-01f));
+  uint32_t tl, th, pl, ph;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(tl), "=r"(th) : "l"(t));
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(pl), "=r"(ph) : "l"(p));
+  return pack2(pl + (tl << 23), ph + (th << 23));
+}
+// Of every eight pairs of exponentials, this many go to the FMA pipe. Measured on the epilogue arithmetic alone, two
+// warps per scheduler: the column sums of sweep 2 take 2314 cycles per 128 columns with none, 1955 with two, 2052 with
+// three; the row statistics of sweep 1, whose maxima already load the other pipes, 2399, 2481 and 3025: none there.
+#ifndef AKV_POLY_S1
+#define AKV_POLY_S1 0
+#endif
+#ifndef AKV_POLY_S2
+#define AKV_POLY_S2 2
+#endif
+constexpr int kPolyS1 = AKV_POLY_S1, kPolyS2 = AKV_POLY_S2;
+
+// Sweep 1 works on 64 accumulator columns of a row at a time (two register buffers of 32).
+__device__ __forceinline__ float max32(const uint32_t (&r)[32]) {
+  float c0 = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+  float c1 = max3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
+  float c2 = max3(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
+  float c3 = max3(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
 #pragma unroll
-  for (int c = 0; c < NCH; c += 2) {
-    tmem_wait(ra[0]);
-    if (c + 1 < NCH) tmem_ld32_issue(taddr + (c + 1) * 32, rb[0]);
-    if (live) stats_part<1>(ra, masked, col0 + c * 32, last_col, sl, m_run, Z);  // padding rows only take part in the loads
-    __syncwarp();  // a warp may hold live and padding rows: rejoin before the warp-wide TMEM instructions
-    if (c + 1 < NCH) {
-      tmem_wait(rb[0]);
-      if (c + 2 < NCH) tmem_ld32_issue(taddr + (c + 2) * 32, ra[0]);
-      if (live) stats_part<1>(rb, masked, col0 + (c + 1) * 32, last_col, sl, m_run, Z);
-      __syncwarp();
+  for (int i = 12; i + 7 < 32; i += 8) {
+    c0 = max3(c0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+    c1 = max3(c1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+    c2 = max3(c2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+    c3 = max3(c3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+  }
+  c0 = max3(c0, __uint_as_float(r[28]), __uint_as_float(r[29]));
+  c1 = max3(c1, __uint_as_float(r[30]), __uint_as_float(r[31]));
+  return fmaxf(max3(c0, c1, c2), c3);
+}
+// Adds exp2(r * sl - m) of 32 logits into four pairs of partial sums; m is a whole number of octaves.
+__device__ __forceinline__ void exp_sum32(const uint32_t (&r)[32], float sl, float inv_sl, float m, f32x2& a0, f32x2& a1,
+                                          f32x2& a2, f32x2& a3) {
+  const float nb = -m;
+  const float r_min = (m - 120.f) * inv_sl;  // logits below this add less than 2^-120 each: held there for the polynomial
+  const f32x2 sl2 = pack2(sl, sl), nb2 = pack2(nb, nb), nbm2 = pack2(nb + kMagic, nb + kMagic);
+#pragma unroll
+  for (int i = 0; i < 32; i += 16) {
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+      const uint32_t x0 = r[i + 2 * p], x1 = r[i + 2 * p + 1];
+      f32x2 e;
+      if (p < kPolyS1) {
+        const f32x2 v = pack2(fmaxf(__uint_as_float(x0), r_min), fmaxf(__uint_as_float(x1), r_min));
+        e = ex2_poly(fma2(v, sl2, nb2), fma2(v, sl2, nbm2));  // nb is an integer: nb + kMagic is exact
+      } else {
+        e = ex2_2(fma2(pack2(x0, x1), sl2, nb2));
+      }
+      if ((p & 3) == 0) a0 = add2(a0, e);
+      else if ((p & 3) == 1) a1 = add2(a1, e);
+      else if ((p & 3) == 2) a2 = add2(a2, e);
+      else a3 = add2(a3, e);
     }
   }
 }
+// The next whole octave at or above x: adding 1.5 * 2^23 rounded upwards leaves ceil(x) in the low mantissa bits
+// (FMA-pipe operations; ceilf would queue behind the exponentials in the special-function unit).
+__device__ __forceinline__ float ceil_octave(float x) { return __fadd_ru(x, kMagic) - kMagic; }
 
+// Sweep 1: 64 logits of this thread's row (columns col0 .. col0 + 63 of the tile, in two buffers). Updates the row's
+// reference m_ref (a whole number of octaves, so that changing it rescales the sum exactly) and its sum Z of exp2
+// relative to that reference. The exponentials are taken against the reference the row had BEFORE these columns
+// and the maximum of the columns is found beside them, not before them: a reference up to 60 octaves below the
+// maximum loses nothing in fp32, so only the first columns of a run, or a jump of more than 60 octaves, have to
+// wait for their maximum (and then take the exponentials once more).
+__device__ __forceinline__ void stats_step(uint32_t (&ra)[32], uint32_t (&rb)[32], bool masked, int col0, int last_col,
+                                           float sl, float inv_sl, float& m_ref, float& Z) {
+  if (masked) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      if (col0 + i > last_col) ra[i] = 0xff800000u;  // -inf
+      if (col0 + 32 + i > last_col) rb[i] = 0xff800000u;
+    }
+  }
+  if (m_ref == -INFINITY) {
+    const float cm = fmaxf(max32(ra), max32(rb));
+    if (cm == -INFINITY) return;  // fully masked: adds nothing
+    m_ref = ceil_octave(cm * sl);
+  }
+  f32x2 a0 = pack2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
+  exp_sum32(ra, sl, inv_sl, m_ref, a0, a1, a2, a3);
+  exp_sum32(rb, sl, inv_sl, m_ref, a0, a1, a2, a3);
+  const float cm = fmaxf(max32(ra), max32(rb));
+  const float d = ceil_octave(cm * sl) - m_ref;  // -inf when the columns are all masked
+  if (d > 60.f) {
+    const float m_new = m_ref + d;
+    a0 = a1 = a2 = a3 = pack2(0.f, 0.f);
+    exp_sum32(ra, sl, inv_sl, m_new, a0, a1, a2, a3);
+    exp_sum32(rb, sl, inv_sl, m_new, a0, a1, a2, a3);
+    Z = fmaf(Z, ex2(m_ref - m_new), hsum(a0, a1, a2, a3));
+    m_ref = m_new;
+  } else {
+    Z += hsum(a0, a1, a2, a3);
+    if (d > 0.f) {  // keep the reference at or above the running maximum: later columns then stay in range
+      Z *= ex2(-d);
+      m_ref += d;
+    }
+  }
+}
 // Sweep 2: N logits of this thread's key against N query rows; nc = their -(max + log2 sum), 16-byte aligned.
-// Adds exp2(z * sl + nc[row]) into four pairs of partial sums.
+// Adds exp2(z * sl + nc[row]) into four pairs of partial sums. The arguments are at most 0 (up to rounding).
 template <int N>
-__device__ __forceinline__ void colsum_part(const uint32_t (&r)[N], const float* __restrict__ nc, f32x2 sl2, f32x2& a0,
+__device__ __forceinline__ void colsum_part(const uint32_t (&r)[32], const float* __restrict__ nc, f32x2 sl2, f32x2& a0,
                                             f32x2& a1, f32x2& a2, f32x2& a3) {
   const ulonglong2* nc2 = reinterpret_cast<const ulonglong2*>(nc);
+  const f32x2 magic2 = pack2(kMagic, kMagic);
 #pragma unroll
   for (int j = 0; j < N; j += 8) {
     const ulonglong2 v = nc2[j >> 2], w = nc2[(j >> 2) + 1];
-    a0 = add2(a0, ex2_2(fma2(pack2(r[j], r[j + 1]), sl2, v.x)));
-    a1 = add2(a1, ex2_2(fma2(pack2(r[j + 2], r[j + 3]), sl2, v.y)));
-    a2 = add2(a2, ex2_2(fma2(pack2(r[j + 4], r[j + 5]), sl2, w.x)));
-    a3 = add2(a3, ex2_2(fma2(pack2(r[j + 6], r[j + 7]), sl2, w.y)));
-  }
-}
-// One tile of sweep 2: this group's n_u (<= 4) units of 16 TMEM columns starting at taddr; nc points at the
-// first of its query rows. Chunks of 32 columns and a last one of 16; the other warps of the scheduler cover
-// the load latency.
-__device__ __forceinline__ float colsum_tile(uint32_t taddr, int n_u, const float* __restrict__ nc, float sl) {
-  const int n32 = n_u >> 1;
-  const bool tail = (n_u & 1) != 0;
-  uint32_t ra[32], rt[16];
-  if (tail) tmem_ld16_issue(taddr + n32 * 32, rt);
-  const f32x2 sl2 = pack2(sl, sl);
-  f32x2 a0 = pack2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
+    const int n_poly = (j & 8) ? kPolyS2 / 2 : (kPolyS2 + 1) / 2;  // of every 4 pairs, alternately: 1 and 1 make 2 of 8
+    f32x2 x[4] = {fma2(pack2(r[j], r[j + 1]), sl2, v.x), fma2(pack2(r[j + 2], r[j + 3]), sl2, v.y),
+                  fma2(pack2(r[j + 4], r[j + 5]), sl2, w.x), fma2(pack2(r[j + 6], r[j + 7]), sl2, w.y)};
+    f32x2 e[4];
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    if (c < n32) {
-      tmem_ld32_issue(taddr + c * 32, ra);
-      tmem_wait(ra);
-      colsum_part<32>(ra, nc + c * 32, sl2, a0, a1, a2, a3);
+    for (int p = 0; p < 4; ++p) {
+      if (p < n_poly) {
+        float lo, hi;
+        unpack2(x[p], lo, hi);
+        const f32x2 c = pack2(fmaxf(lo, -120.f), fmaxf(hi, -120.f));  // padding rows carry -inf
+        e[p] = ex2_poly(c, add2(c, magic2));
+      } else {
+        e[p] = ex2_2(x[p]);
+      }
     }
+    a0 = add2(a0, e[0]);
+    a1 = add2(a1, e[1]);
+    a2 = add2(a2, e[2]);
+    a3 = add2(a3, e[3]);
   }
-  if (tail) {
-    tmem_wait(rt);
-    colsum_part<16>(rt, nc + n32 * 32, sl2, a0, a1, a2, a3);
-  }
-  return hsum(a0, a1, a2, a3);
 }
 
 template <int SWEEP, int D, int CAP>
@@ -365,10 +473,17 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
   volatile int* abort = &sm->abort;
 
   const Shape& sh = a.sh;
-  const int R = sh.window * sh.group, G = sh.group;
-  const bool both = SWEEP == 1 && R > 128;   // sweep 1 with two row blocks: each group reads its own block of every tile
+  const int G = sh.group, R = a.w_chunk * G;  // query rows of a run's Q tile; Rt: of the head (statistics layout)
+  const int Rt = sh.window * G;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = a.n_stages;
+  const long long wl = a.wait_cycles;
+  // Parts of a tile, each with an accumulator buffer of its own.
+  //   sweep 1: blocks of 128 query rows (M = 128 rows, N = 128 keys);
+  //   sweep 2: the query rows in one piece (up to 128) or in two halves of whole 16s (M = 128 keys, N = the rows).
+  const int n_parts = SWEEP == 1 ? (R > 128 ? 2 : 1) : (a.r_pad > 128 ? 2 : 1);
+  const int cols0 = SWEEP == 1 ? kTileKeys : (n_parts == 2 ? ((a.r_pad >> 4) + 1) / 2 * 16 : a.r_pad);
+  const int cols1 = SWEEP == 1 ? kTileKeys : a.r_pad - cols0;
 
   // ---- set-up ----
   if (threadIdx.x == 0) {
@@ -377,16 +492,16 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
       mbar_init(smem_u32(&sm->k_empty[s]), 1);
     }
     mbar_init(smem_u32(&sm->q_full), 1);
-    mbar_init(smem_u32(&sm->q_empty), 1);
+    mbar_init(smem_u32(&sm->q_empty), 2);  // both MMA threads are done with the Q tile
     for (int g = 0; g < 2; ++g) {
       for (int b = 0; b < 2; ++b) {
         mbar_init(smem_u32(&sm->acc_full[g][b]), 1);
-        mbar_init(smem_u32(&sm->acc_empty[g][b]), 8);  // the two epilogue groups that share the stream
+        mbar_init(smem_u32(&sm->acc_empty[g][b]), 4);  // the four warps of the group
       }
+      mbar_init(smem_u32(&sm->grp_bar[g]), 128);
     }
-    mbar_init(smem_u32(&sm->all_bar), kEpiWarps * 32);
-    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sm->part_full[i]), 12);
-    mbar_init(smem_u32(&sm->drain), 1);
+    mbar_init(smem_u32(&sm->drain[0]), 1);
+    mbar_init(smem_u32(&sm->drain[1]), 1);
     sm->abort = 0;
     fence_barrier_init();
   }
@@ -413,18 +528,7 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
   chain_release();
   const uint32_t tmem_base = sm->tmem_base;
 
-  const int unit_begin = static_cast<int>(static_cast<int64_t>(blockIdx.x) * a.n_units / gridDim.x);
-  const int unit_end = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * a.n_units / gridDim.x);
-
-  // Every tile is split between the two epilogue groups, and each group gets its share through its own
-  // pair of accumulator buffers (TMEM columns (2 b + g) * 128 ..), filled by its own MMAs: the groups
-  // then run half a tile apart instead of in step, and one group's exponentials cover the other's
-  // loads and maxima.
-  //   sweep 1, two row blocks: group g = row block g, all 128 keys;
-  //   sweep 1, one row block:  group g = keys 64 g .. 64 g + 63 of every row;
-  //   sweep 2: group 0 = the first half of the query rows (in units of 16), group 1 = the rest.
-  const int n16 = a.r_pad >> 4, u_split = (n16 + 1) >> 1;
-  auto share_units = [&](int g) { return g == 0 ? u_split : n16 - u_split; };  // sweep 2: units of 16 rows
+  const int unit_begin = __ldg(a.cta_begin + blockIdx.x), unit_end = __ldg(a.cta_begin + blockIdx.x + 1);
 
   if (warp == kProducerWarp) {
     // ---- TMA producer ----
@@ -444,7 +548,7 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
       ScoreUnit Unext = a.units[unit_begin < unit_end ? unit_begin : 0];
       for (int n = unit_begin; n < unit_end && ok; ++n) {
         const ScoreUnit U = Unext;
-        if (n + 1 < unit_end) Unext = a.units[n + 1];  // the next descriptor arrives under this unit's work
+        if (n + 1 < unit_end) Unext = a.units[n + 1];  // the next descriptor arrives under this run's work
         for (int t = 0; t < U.n_tiles; ++t, ++it) {
           const uint32_t bar = smem_u32(&sm->k_full[s]);
           int page_y = 0;
@@ -461,18 +565,19 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
           }
           bool mine = true;
           if (lane == 0) {
-            if (t == 0 && U.u != prev_u) {
-              if (heads > 0) mine = mbar_wait(smem_u32(&sm->q_empty), (heads - 1) & 1, abort);  // MMAs on the old Q are done
+            if (t == 0 && U.qid != prev_u) {
+              if (heads > 0) mine = mbar_wait(smem_u32(&sm->q_empty), (heads - 1) & 1, abort, wl);  // MMAs on the old Q are done
               if (mine) {
+                // the box is w_chunk window rows; rows of a last, shorter chunk beyond the window arrive as zeros
                 const uint32_t qbar = smem_u32(&sm->q_full);
                 mbar_expect_tx(qbar, static_cast<uint32_t>(R) * D * 2);
                 for (int kb = 0; kb < KB; ++kb)
-                  tma_load_4d(smem_u32(q_s + kb * q_blk), &tm.q[U.r - a.r0], qbar, kb * 64, U.h * G, 0, U.l);
-                prev_u = U.u;
+                  tma_load_4d(smem_u32(q_s + kb * q_blk), &tm.q[U.r - a.r0], qbar, kb * 64, U.h * G, U.w0, U.l);
+                prev_u = U.qid;
                 ++heads;
               }
             }
-            if (mine) mine = mbar_wait(smem_u32(&sm->k_empty[s]), ph ^ 1, abort);
+            if (mine) mine = mbar_wait(smem_u32(&sm->k_empty[s]), ph ^ 1, abort, wl);
             if (mine) mbar_expect_tx(bar, kKStage);
           }
           ok = __shfl_sync(lanes, mine, 0);
@@ -502,116 +607,101 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
         }
       }
       if (lane == 0 && *abort) {  // let the copies still in flight land before the CTA goes away
-        const long long short_limit = 200000000LL;
-        for (int j = it > S ? it - S : 0; j < it; ++j)
-          mbar_wait(smem_u32(&sm->k_full[j % S]), (j / S) & 1, abort, short_limit);
-        if (heads > 0) mbar_wait(smem_u32(&sm->q_full), (heads - 1) & 1, abort, short_limit);
+        for (int j = it > S ? it - S : 0; j < it; ++j) mbar_wait_drain(smem_u32(&sm->k_full[j % S]), (j / S) & 1);
+        if (heads > 0) mbar_wait_drain(smem_u32(&sm->q_full), (heads - 1) & 1);
       }
     }
-  } else if (warp == kMmaWarp) {
+  } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
     if (lane == 0) {
-      // ---- MMA issuer ----
-      int it = 0, heads = 0, prev_u = -1, s = 0;
-      uint32_t ph = 0;
+      // ---- MMA issuer of group g ----
+      // Tile `it` of the CTA belongs to group it & 1 and sits in stage it % S of the K ring. Its parts go to the
+      // group's buffers in turn: part number qc of the group uses buffer qc & 1, in phase (qc >> 1) & 1 of the
+      // buffer's barriers.
+      const int g = warp - kMmaWarp;
+      int it = 0, heads = 0, prev_u = -1, qc = 0;
       bool ok = true;
-      const uint32_t idesc1 = both ? umma_idesc(128, kTileKeys) : umma_idesc(128, kTileKeys / 2);
       ScoreUnit Unext = a.units[unit_begin < unit_end ? unit_begin : 0];
       for (int n = unit_begin; n < unit_end && ok; ++n) {
         const ScoreUnit U = Unext;
-        if (n + 1 < unit_end) Unext = a.units[n + 1];  // the next descriptor arrives under this unit's work
-        if (U.u != prev_u) {
-          if (prev_u != -1) umma_commit(smem_u32(&sm->q_empty));
-          ok = mbar_wait(smem_u32(&sm->q_full), heads & 1, abort);
+        if (n + 1 < unit_end) Unext = a.units[n + 1];  // the next descriptor arrives under this run's work
+        if (U.qid != prev_u) {
+          if (prev_u != -1) umma_commit(smem_u32(&sm->q_empty));  // this thread's MMAs on the old Q tile are done
+          ok = mbar_wait(smem_u32(&sm->q_full), heads & 1, abort, wl);
           if (!ok) break;
           tc_fence_after();
-          prev_u = U.u;
+          prev_u = U.qid;
           ++heads;
         }
         for (int t = 0; t < U.n_tiles && ok; ++t, ++it) {
-          ok = mbar_wait(smem_u32(&sm->k_full[s]), ph, abort);
+          if ((it & 1) != g) continue;  // the other thread's tile
+          const int s = it % S;
+          ok = mbar_wait(smem_u32(&sm->k_full[s]), (it / S) & 1, abort, wl);
           if (!ok) break;
-          const int b = it & 1;
           const uint32_t k_addr = smem_u32(k_s + s * kKStage);
           const uint32_t q_addr = smem_u32(q_s);
-          for (int g = 0; g < 2; ++g) {
-            if (SWEEP == 2 && share_units(g) == 0) continue;
-            ok = mbar_wait(smem_u32(&sm->acc_empty[g][b]), ((it >> 1) & 1) ^ 1, abort);
+          for (int p = 0; p < n_parts; ++p) {
+            const int b = qc & 1;
+            ok = mbar_wait(smem_u32(&sm->acc_empty[g][b]), ((qc >> 1) & 1) ^ 1, abort, wl);
             if (!ok) break;
+            ++qc;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (2 * b + g) * 128;
-            // byte offsets of the group's share inside the Q tile / the K tile (multiples of 1024: whole 8-row groups)
-            const uint32_t q_off = SWEEP == 1 ? (both ? g * (128 * 128) : 0) : (g == 0 ? 0 : u_split * 16 * 128);
-            const uint32_t k_off = SWEEP == 1 && !both ? g * (64 * 128) : 0;
-            const uint32_t idesc = SWEEP == 1 ? idesc1 : umma_idesc(kTileKeys, share_units(g) * 16);
+            const uint32_t d_tmem = tmem_base + (2 * g + b) * 128;
+            // byte offset of the part inside the Q tile (a multiple of 1024: whole 8-row groups)
+            const uint32_t q_off = SWEEP == 1 ? p * (128 * 128) : (p == 0 ? 0 : cols0 * 128);
+            const uint32_t idesc = SWEEP == 1 ? umma_idesc(128, kTileKeys) : umma_idesc(kTileKeys, p == 0 ? cols0 : cols1);
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
 #pragma unroll
               for (int ks = 0; ks < 4; ++ks) {
                 const uint64_t dq = umma_desc(q_addr + kb * q_blk + q_off + ks * 32);
-                const uint64_t dk = umma_desc(k_addr + kb * kKBlk + k_off + ks * 32);
+                const uint64_t dk = umma_desc(k_addr + kb * kKBlk + ks * 32);
                 if (SWEEP == 1) umma_bf16(d_tmem, dq, dk, idesc, (kb | ks) != 0);
                 else umma_bf16(d_tmem, dk, dq, idesc, (kb | ks) != 0);
               }
             }
             umma_commit(smem_u32(&sm->acc_full[g][b]));
           }
-          umma_commit(smem_u32(&sm->k_empty[s]));
-          if (++s == S) {
-            s = 0;
-            ph ^= 1;
-          }
+          if (ok) umma_commit(smem_u32(&sm->k_empty[s]));
         }
       }
       if (*abort) {  // TMEM must not be released under MMAs that are still running
-        umma_commit(smem_u32(&sm->drain));
-        mbar_wait(smem_u32(&sm->drain), 0, abort, 200000000LL);
+        umma_commit(smem_u32(&sm->drain[g]));
+        mbar_wait_drain(smem_u32(&sm->drain[g]), 0);
       }
     }
   } else {
-    // ---- epilogue: four groups of four warps; warp w reads TMEM lanes 32 (w % 4) .. +31 ----
-    // Groups 2 st and 2 st + 1 share accumulator stream st and split its columns in two:
-    //   sweep 1, two row blocks: stream = row block, group = 64 of its 128 key columns;
-    //   sweep 1, one row block:  stream = 64 key columns, group = 32 of them;
-    //   sweep 2: stream = half of the query rows (units of 16), group = half of those; groups 1-3 hand their
-    //            partial column sums to group 0 through shared memory.
-    // Four warps per scheduler keep the special-function unit fed while others load, reduce or wait.
-    const int g4 = warp >> 2, quarter = warp & 3;
-    const int st = g4 >> 1, sub = g4 & 1;
+    // ---- epilogue: two groups of four warps; warp w reads TMEM lanes 32 (w % 4) .. +31 ----
+    const int g = warp >> 2, quarter = warp & 3;
     const int gl = quarter * 32 + lane;  // thread index inside the group = TMEM lane
-    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-    const float sl = sh.scale_log2e;
-    int it = 0, prev_u = -1, n_done = 0, heads = 0;
-    uint32_t all_phase = 0;
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + 2 * g * 128;
+    const float sl = sh.scale_log2e, inv_sl = 1.0f / sl;
+    int it = 0, prev_u = -1, heads = 0, qc = 0;
+    uint32_t grp_phase = 0;
     bool ok = true;
-    const int row = (both ? st * 128 : 0) + gl;                // sweep 1: this thread's query row
-    const int col0 = both ? sub * 64 : st * 64 + sub * 32;     // sweep 1: first key column (of the tile) of its share
-    const int tcol1 = both ? sub * 64 : sub * 32;              // ... and that column inside the stream's accumulator
-    const int win_i = row / G;                                 // window row of that query row
-    const bool live = row < R;
-    // sweep 2: the stream's units of 16 query rows, and this group's part of them
-    const int st_u0 = st == 0 ? 0 : u_split, st_n = share_units(st);
-    const int half_n = (st_n + 1) >> 1;
-    const int my_u0 = sub == 0 ? 0 : half_n, my_n = sub == 0 ? half_n : st_n - half_n;
+    uint32_t ra[32], rb[32];
     if (SWEEP == 2) chain_wait();  // the statistics of sweep 1 are complete and visible
     ScoreUnit Unext = a.units[unit_begin < unit_end ? unit_begin : 0];
-    for (int n = unit_begin; n < unit_end && ok; ++n, ++n_done) {
+    for (int n = unit_begin; n < unit_end && ok; ++n) {
       const ScoreUnit U = Unext;
       if (n + 1 < unit_end) Unext = a.units[n + 1];
-      if (SWEEP == 2 && U.u != prev_u) {
-        // Merge the slabs' statistics of this head: negc[row] = -(max + log2 sum); padding rows get -inf.
-        // One row per thread of the first two groups, eight independent loads in flight at a time.
-        const int slabs = U.head_slabs;
-        const int rr = g4 * 128 + gl;
-        if (rr < 256) {
+      const int live_rows = U.wn * G;  // query rows of this run (the Q tile may hold more: padding, a short last chunk)
+      if (SWEEP == 2 && U.qid != prev_u) {
+        // Merge the parts' statistics of this head: negc[row] = -(max + log2 sum); padding rows get -inf. Each group
+        // keeps a copy of its own (two rows per thread), in two versions by head parity: a warp of the group that is
+        // still on the head before reads the other version, and none can be two heads behind the barrier below.
+        float* dst = sm->negc[g][heads & 1];
+        for (int rr = gl; rr < 256; rr += 128) {
           float c = -INFINITY;
-          if (rr < R) {
-            const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.n_slab * R + rr;
+          if (rr < live_rows) {
+            const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.max_parts * 2 * Rt + U.w0 * G + rr;
             float M = -INFINITY, Zt = 0.f;
-            for (int s0 = 0; s0 < slabs; s0 += 8) {
+            const int n_ent = U.head_parts * 2;
+            for (int s0 = 0; s0 < n_ent; s0 += 8) {
               float2 sv[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i)
-                sv[i] = s0 + i < slabs ? __ldg(hs + static_cast<int64_t>(s0 + i) * R) : make_float2(-INFINITY, 0.f);
+                sv[i] = s0 + i < n_ent ? __ldcg(hs + static_cast<int64_t>(s0 + i) * Rt)  // written by the kernel before
+                                       : make_float2(-INFINITY, 0.f);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 if (sv[i].y > 0.f) {
@@ -623,85 +713,109 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
             }
             c = -(M + log2f(Zt));
           }
-          // two copies by head parity: a slower warp may still read the previous head's
-          sm->negc[heads & 1][rr] = c;
+          dst[rr] = c;
         }
         ++heads;
-        mbar_arrive(smem_u32(&sm->all_bar));
-        ok = mbar_wait(smem_u32(&sm->all_bar), all_phase, abort);
-        all_phase ^= 1;
+        mbar_arrive(smem_u32(&sm->grp_bar[g]));
+        ok = mbar_wait(smem_u32(&sm->grp_bar[g]), grp_phase, abort, wl);
+        grp_phase ^= 1;
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
-      prev_u = U.u;
-      float m_run = -INFINITY, Z = 0.f;  // sweep 1: this thread's row (its share of the columns)
+      prev_u = U.qid;
+      if (SWEEP == 1 && a.accumulate && U.w0 == 0) {
+        // a head scored in several chunks of window rows: sweep 2 adds each chunk's column sums into the score buffer,
+        // so the first chunk's run clears the entries of its keys (sweep 2 starts after this kernel has ended)
+        const int k_end = U.kt0 + U.n_tiles * kTileKeys < U.P ? U.kt0 + U.n_tiles * kTileKeys : U.P;
+        for (int key = U.kt0 + static_cast<int>(threadIdx.x); key < k_end; key += kEpiWarps * 32)
+          a.scores[U.score_base + key] = 0.f;
+      }
+      // sweep 1: this thread's rows gl and 128 + gl: reference, in whole octaves, and sum of exp2 relative to it
+      float m_ref[2] = {-INFINITY, -INFINITY}, Z[2] = {0.f, 0.f};
+      const float* nc = SWEEP == 2 ? sm->negc[g][(heads - 1) & 1] : nullptr;
       for (int t = 0; t < U.n_tiles; ++t, ++it) {
-        const int b = it & 1;
-        const bool stream_on = SWEEP == 1 || st_n > 0;  // the MMA thread skips a stream without rows
-        if (stream_on) {
-          ok = mbar_wait(smem_u32(&sm->acc_full[st][b]), (it >> 1) & 1, abort);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          tc_fence_after();
-        }
+        if ((it & 1) != g) continue;  // the other group's tile
         const int kt = U.kt0 + t * kTileKeys;
-        const uint32_t taddr = lane_addr + (2 * b + st) * 128;
-        if (SWEEP == 1) {
-          const bool masked = kt + kTileKeys - 1 > U.P;  // the tile reaches into the window: causal mask, end of request
-          const int last_col = U.P + win_i - kt;         // last visible key of this row, relative to the tile
-          if (both) stats_tile<2>(taddr + tcol1, live, masked, col0, last_col, sl, m_run, Z);
-          else stats_tile<1>(taddr + tcol1, live, masked, col0, last_col, sl, m_run, Z);
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[st][b]));
-        } else {
-          float acc = 0.f;
-          if (stream_on) {
-            if (my_n > 0) acc = colsum_tile(taddr + my_u0 * 16, my_n, sm->negc[(heads - 1) & 1] + (st_u0 + my_u0) * 16, sl);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[st][b]));
+        const f32x2 sl2 = pack2(sl, sl);
+        f32x2 a0 = pack2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;  // sweep 2: this key's sums over the rows
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+          if (p >= n_parts || !ok) continue;
+          const int b = qc & 1;
+          ok = mbar_wait(smem_u32(&sm->acc_full[g][b]), (qc >> 1) & 1, abort, wl);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) continue;
+          ++qc;
+          tc_fence_after();
+          const uint32_t taddr = lane_addr + b * 128;
+          const uint32_t ebar = smem_u32(&sm->acc_empty[g][b]);
+          // Steps of 64 accumulator columns (two register buffers of 32; the last one may hold 16 in sweep 2): the loads of
+          // a step land within tens of cycles, so nothing is prefetched, and the arithmetic of a step is one long block
+          // of independent work for the scheduler. The accumulator buffer goes back to the MMA thread as soon as its
+          // last step is in registers.
+          const int cols = p == 0 ? cols0 : cols1;
+          const int n_ch = (cols + 31) >> 5;
+          const bool tail = (cols & 16) != 0;
+          const int row = p * 128 + gl;                       // sweep 1: this thread's query row in the part
+          const bool live = row < live_rows;
+          const bool masked = kt + kTileKeys - 1 > U.P;       // sweep 1: the tile reaches into the window: causal mask
+          const int last_col = U.P + U.w0 + row / G - kt;     // sweep 1: last visible key of this row, relative to the tile
+          const float* ncp = SWEEP == 2 ? nc + (p == 0 ? 0 : cols0) : nullptr;
+#pragma unroll
+          for (int st = 0; st < 2; ++st) {
+            const int c0 = 2 * st;  // first chunk of 32 columns of this step
+            if (c0 < n_ch) {
+              const bool has_b = c0 + 1 < n_ch;
+              const bool a_half = tail && c0 == n_ch - 1, b_half = tail && c0 + 1 == n_ch - 1;
+              if (a_half) tmem_ld16_issue_lo(taddr + c0 * 32, ra);
+              else tmem_ld32_issue(taddr + c0 * 32, ra);
+              if (has_b) {
+                if (b_half) tmem_ld16_issue_lo(taddr + (c0 + 1) * 32, rb);
+                else tmem_ld32_issue(taddr + (c0 + 1) * 32, rb);
+              }
+              if (a_half) tmem_wait_lo(ra);
+              else tmem_wait(ra);
+              if (has_b) {
+                if (b_half) tmem_wait_lo(rb);
+                else tmem_wait(rb);
+              }
+              if (c0 + 2 >= n_ch) {  // the part is in registers: its buffer goes back to the MMA thread
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(ebar);
+              }
+              if constexpr (SWEEP == 1) {
+                if (live) stats_step(ra, rb, masked, c0 * 32, last_col, sl, inv_sl, m_ref[p], Z[p]);  // padding rows only load
+                __syncwarp();  // a warp may hold live and padding rows: rejoin before the warp-wide TMEM instructions
+              } else {
+                if (a_half) colsum_part<16>(ra, ncp + c0 * 32, sl2, a0, a1, a2, a3);
+                else colsum_part<32>(ra, ncp + c0 * 32, sl2, a0, a1, a2, a3);
+                if (has_b) {
+                  if (b_half) colsum_part<16>(rb, ncp + (c0 + 1) * 32, sl2, a0, a1, a2, a3);
+                  else colsum_part<32>(rb, ncp + (c0 + 1) * 32, sl2, a0, a1, a2, a3);
+                }
+              }
+            }
           }
-          const int slot = it & 3;
-          if (g4 != 0) {
-            sm->part[slot][g4 - 1][gl] = acc;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm->part_full[slot]));
-          } else {
-            // Slot it & 3 is written again four tiles on. By then the MMAs of tile it + 4 have been issued,
-            // so this group has released the buffer of tile it + 2, which it does after the read below.
-            ok = mbar_wait(smem_u32(&sm->part_full[slot]), (it >> 2) & 1, abort);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const int key = kt + gl;
-            if (key < U.P)
-              a.scores[U.score_base + key] = (acc + sm->part[slot][0][gl]) + (sm->part[slot][1][gl] + sm->part[slot][2][gl]);
+        }
+        if (!ok) break;
+        if (SWEEP == 2) {
+          const int key = kt + gl;
+          if (key < U.P) {
+            const float sum = hsum(a0, a1, a2, a3);
+            if (a.accumulate) atomicAdd(a.scores + U.score_base + key, sum);  // the buffer was cleared by sweep 1
+            else a.scores[U.score_base + key] = sum;
           }
         }
       }
       if (!ok) break;
       if (SWEEP == 1) {
-        // the groups that share a row hand their statistics to the first of them
-        float2* out = a.stats + (static_cast<int64_t>(U.u) * a.n_slab + U.slab) * R;
-        float2(*mg)[128] = sm->mrg[n_done & 1];
-        const bool writer = both ? sub == 0 : g4 == 0;
-        if (!writer) mg[both ? st : g4 - 1][gl] = make_float2(m_run, Z);
-        mbar_arrive(smem_u32(&sm->all_bar));
-        ok = mbar_wait(smem_u32(&sm->all_bar), all_phase, abort);
-        all_phase ^= 1;
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (writer && live) {
-          const int s0 = both ? st : 0, ns_ = both ? 1 : 3;
-          float M = m_run;
-          for (int o = 0; o < ns_; ++o) M = fmaxf(M, mg[s0 + o][gl].x);
-          float Zt = Z > 0.f ? Z * ex2((m_run - M) * sl) : 0.f;
-          for (int o = 0; o < ns_; ++o) {
-            const float2 pz = mg[s0 + o][gl];
-            if (pz.y > 0.f) Zt += pz.y * ex2((pz.x - M) * sl);
-          }
-          out[row] = make_float2(M * sl, Zt);
-        }
+        // this group's share of the run (every second tile): one entry per row, merged by sweep 2 with the other
+        // group's and the other parts'; a group without a tile in the run writes an empty entry
+        float2* out = a.stats + ((static_cast<int64_t>(U.u) * a.max_parts + U.part) * 2 + g) * Rt + U.w0 * G;
+#pragma unroll
+        for (int p = 0; p < 2; ++p)
+          if (p < n_parts && p * 128 + gl < live_rows) out[p * 128 + gl] = make_float2(m_ref[p], Z[p]);
       }
     }
   }
@@ -754,95 +868,124 @@ cudaError_t launch_sweep(const TmapPack<CAP>& tm, const UmmaArgs& args, int grid
 }
 
 template <int CAP>
-cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
-                                  const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
-                                  float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
-                                  int head_begin, int head_end, ScoreMapCache* cache, uint64_t plan_id);
+cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* d_units, const int32_t* d_cta,
+                                  const ScoreSchedule& sc, int slot, const void* q, const void* k, float* scores,
+                                  float2* stats_ws, int max_parts, int* status, Launch ln, ScoreMapCache* cache,
+                                  uint64_t plan_id);
 
 }  // namespace
 
-bool score_umma_takes(const Shape& sh) {
-  if (sh.dtype != AUDIOKV_BF16) return false;
-  const int R = sh.window * sh.group;
-  if (R > 256 || sh.group > 256 || sh.window > 256) return false;
-  const int q_rows = R > 128 ? 256 : 128;
-  const int q_bytes = q_rows * sh.head_dim * 2, stage = kTileKeys * sh.head_dim * 2;
-  const int room = kSmemLimit - 1024 - static_cast<int>(sizeof(Small)) - q_bytes;
-  return room >= 2 * stage;
+int score_window_chunk(const Shape& sh) {
+  if (sh.group < 1 || sh.window < 1) return 0;
+  const int stage = kTileKeys * sh.head_dim * 2;
+  for (int q_rows = 256; q_rows >= 128; q_rows -= 128) {
+    const int room = kSmemLimit - 1024 - static_cast<int>(sizeof(Small)) - q_rows * sh.head_dim * 2;
+    if (room < 2 * stage) continue;  // the K ring needs two stages
+    const int w_max = q_rows / sh.group;
+    if (w_max < 1) return 0;
+    if (w_max >= sh.window) return sh.window;
+    const int n_chunks = (sh.window + w_max - 1) / w_max;
+    return (sh.window + n_chunks - 1) / n_chunks;  // chunks of equal size (the last one may be shorter)
+  }
+  return 0;
 }
 
-cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
-                              const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
-                              float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
-                              int head_begin, int head_end, ScoreMapCache* cache, uint64_t plan_id) {
-  if (sh.n_req <= kMapChunkSmall)
-    return launch_score_umma_cap<kMapChunkSmall>(sh, h_reqs, units1, unit_pre1, units2, unit_pre2, q, k, scores, stats_ws,
-                                                 n_slab, slab_keys, status, ln, head_begin, head_end, cache, plan_id);
-  return launch_score_umma_cap<kMapChunkLarge>(sh, h_reqs, units1, unit_pre1, units2, unit_pre2, q, k, scores, stats_ws,
-                                               n_slab, slab_keys, status, ln, head_begin, head_end, cache, plan_id);
+static std::atomic<long long> g_wait_cycles{kWaitCycles};
+long long score_wait_cycles() { return g_wait_cycles.load(); }
+void set_score_wait_cycles(long long cycles) { g_wait_cycles.store(cycles > 0 ? cycles : kWaitCycles); }
+
+bool score_umma_takes(const Shape& sh) {
+  if (sh.dtype != AUDIOKV_BF16) return false;
+  const int wc = score_window_chunk(sh);
+  return wc >= 1 && wc <= 256 && sh.group <= 256;
+}
+
+int score_map_chunk(int n_req) { return n_req <= kMapChunkSmall ? kMapChunkSmall : kMapChunkLarge; }
+
+cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* d_units, const int32_t* d_cta,
+                              const ScoreSchedule* scheds, int n_sched, const void* q, const void* k, float* scores,
+                              float2* stats_ws, int max_parts, int* status, Launch ln, int head_begin, int head_end,
+                              ScoreMapCache* cache, uint64_t plan_id) {
+  if (!score_umma_takes(sh)) return cudaErrorNotSupported;
+  // every schedule that covers whole requests, in order; or the one schedule made for this range of heads
+  bool any = false;
+  for (int i = 0; i < n_sched; ++i) {
+    const ScoreSchedule& sc = scheds[i];
+    if (head_end < 0 ? !sc.whole_requests : (sc.whole_requests || sc.head_begin != head_begin || sc.head_end != head_end))
+      continue;
+    any = true;
+    // the maps of a head range are those of its (single) request: slot 0; whole-request schedules come one per slot
+    const int slot = sc.whole_requests ? sc.r_begin / score_map_chunk(sh.n_req) : 0;
+    cudaError_t e = sh.n_req <= kMapChunkSmall
+                        ? launch_score_umma_cap<kMapChunkSmall>(sh, h_reqs, d_units, d_cta, sc, slot, q, k, scores, stats_ws,
+                                                                max_parts, status, ln, cache, plan_id)
+                        : launch_score_umma_cap<kMapChunkLarge>(sh, h_reqs, d_units, d_cta, sc, slot, q, k, scores, stats_ws,
+                                                                max_parts, status, ln, cache, plan_id);
+    if (e != cudaSuccess) return e;
+  }
+  return any ? cudaSuccess : cudaErrorInvalidValue;
 }
 
 namespace {
 
 template <int CAP>
-cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* units1, const int* unit_pre1,
-                                  const ScoreUnit* units2, const int* unit_pre2, const void* q, const void* k,
-                                  float* scores, float2* stats_ws, int n_slab, int slab_keys, int* status, Launch ln,
-                                  int head_begin, int head_end, ScoreMapCache* cache, uint64_t plan_id) {
-  constexpr int kMapChunk = CAP;
+cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* d_units, const int32_t* d_cta,
+                                  const ScoreSchedule& sc, int slot, const void* q, const void* k, float* scores,
+                                  float2* stats_ws, int max_parts, int* status, Launch ln, ScoreMapCache* cache,
+                                  uint64_t plan_id) {
   using Pack = TmapPack<CAP>;
-  if (!score_umma_takes(sh) || slab_keys % kTileKeys) return cudaErrorNotSupported;
-  if (head_end >= 0 && sh.n_req != 1) return cudaErrorInvalidValue;  // head ranges: one request only
   EncodeTiledFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
-  const int R = sh.window * sh.group, d = sh.head_dim;
+  const int w_chunk = score_window_chunk(sh);
+  const int R = w_chunk * sh.group, d = sh.head_dim;  // query rows of one Q tile
 
   UmmaArgs args{};
   args.sh = sh;
   args.stats = stats_ws;
   args.scores = scores;
   args.status = status;
-  args.n_slab = n_slab;
-  args.slab_keys = slab_keys;
+  args.max_parts = max_parts;
   args.q_rows = R > 128 ? 256 : 128;
   args.r_pad = (R + 15) / 16 * 16;
+  args.w_chunk = w_chunk;
+  args.accumulate = w_chunk < sh.window ? 1 : 0;
+  args.wait_cycles = score_wait_cycles();
   const int q_bytes = args.q_rows * d * 2, stage = kTileKeys * d * 2;
   const int room = kSmemLimit - 1024 - static_cast<int>(sizeof(Small)) - q_bytes;
   args.n_stages = room / stage < kMaxStages ? room / stage : kMaxStages;
   const size_t smem = 1024 + static_cast<size_t>(q_bytes) + static_cast<size_t>(args.n_stages) * stage + sizeof(Small);
 
-  int dev = 0, n_sm = 0;
-  cudaError_t e;
-  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-  if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-
-  // Tensor maps are kernel arguments, CAP requests' worth per launch: a longer batch takes both sweeps chunk
-  // by chunk. Sweep 1 lists the units by ascending request, sweep 2 by descending request, so a chunk of requests
-  // is one contiguous run of either list.
-  const int n_units2 = unit_pre2[sh.n_req];
-  const int n_chunks = (sh.n_req + kMapChunk - 1) / kMapChunk;
-  // the maps depend on the buffers, the request table and the strides: the same buffers under the same plan reuse them
+  // Tensor maps are kernel arguments, CAP requests' worth per launch: one pack per run of CAP requests. They depend
+  // on the buffers, the request table and the strides: the same buffers under the same plan reuse them.
+  const int n_slots = (sh.n_req + CAP - 1) / CAP;
   std::vector<unsigned char> local;
   std::vector<unsigned char>& packs = cache ? cache->packs : local;
-  const size_t pack_bytes = sizeof(Pack) * static_cast<size_t>(n_chunks) + 64;  // + room to align to 64 bytes
-  const bool reuse = cache && cache->q == q && cache->k == k && cache->plan_id == plan_id &&
-                     cache->page_size == sh.page_size && packs.size() == pack_bytes;
-  if (!reuse) {
-    if (cache) cache->q = nullptr;  // stays invalid if the encoding below fails half way
+  const size_t pack_bytes = sizeof(Pack) * static_cast<size_t>(n_slots) + 64;  // + room to align to 64 bytes
+  const bool same = cache && cache->q == q && cache->k == k && cache->plan_id == plan_id &&
+                    cache->page_size == sh.page_size && packs.size() == pack_bytes &&
+                    cache->encoded.size() == static_cast<size_t>(n_slots);
+  if (!same) {
     packs.assign(pack_bytes, 0);
+    if (cache) {
+      cache->encoded.assign(n_slots, 0);
+      cache->q = q;
+      cache->k = k;
+      cache->plan_id = plan_id;
+      cache->page_size = sh.page_size;
+    }
   }
   unsigned char* pack0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(packs.data()) + 63) & ~uintptr_t(63));
-  for (int r0 = 0; r0 < sh.n_req; r0 += kMapChunk) {
-    const int r1 = r0 + kMapChunk < sh.n_req ? r0 + kMapChunk : sh.n_req;
-    Pack& tm = *reinterpret_cast<Pack*>(pack0 + sizeof(Pack) * static_cast<size_t>(r0 / kMapChunk));
-    for (int r = r0; r < r1 && !reuse; ++r) {
+  Pack& tm = *reinterpret_cast<Pack*>(pack0 + sizeof(Pack) * static_cast<size_t>(slot));
+  const int r0 = slot * CAP, r1 = r0 + CAP < sh.n_req ? r0 + CAP : sh.n_req;
+  if (!(cache && cache->encoded[slot])) {
+    for (int r = r0; r < r1; ++r) {
       {
         const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(sh.n_q_heads),
                                     static_cast<cuuint64_t>(sh.window), static_cast<cuuint64_t>(sh.n_layers)};
         const int64_t es[3] = {sh.q_stride_head, sh.q_stride_tok, sh.q_stride_layer};
         cuuint64_t strides[3];
         if (!fill_strides(4, dims, es, strides)) return cudaErrorNotSupported;
-        const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(sh.group), static_cast<cuuint32_t>(sh.window), 1u};
+        const cuuint32_t box[4] = {64u, static_cast<cuuint32_t>(sh.group), static_cast<cuuint32_t>(w_chunk), 1u};
         const cuuint32_t ones[4] = {1u, 1u, 1u, 1u};
         void* base = const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(q) + h_reqs[r].q_offset);
         if (enc(&tm.q[r - r0], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, ones,
@@ -867,44 +1010,29 @@ cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorNotSupported;
     }
-    args.r0 = r0;
-    const ScoreUnit* u1 = units1 + unit_pre1[r0];
-    int n1 = unit_pre1[r1] - unit_pre1[r0];
-    const ScoreUnit* u2 = units2 + (n_units2 - unit_pre2[r1]);
-    int n2 = unit_pre2[r1] - unit_pre2[r0];
-    if (head_end >= 0) {
-      // one request: every head has the same number of slabs in a sweep, and its units are consecutive
-      const int s1 = n1 / sh.heads_per_req, s2 = n2 / sh.heads_per_req;
-      u1 += head_begin * s1;
-      n1 = (head_end - head_begin) * s1;
-      u2 += (sh.heads_per_req - head_end) * s2;  // sweep 2 lists the heads backwards
-      n2 = (head_end - head_begin) * s2;
-    }
-
-#define AKV_SWEEP(SW, DD, UNITS, N)                                                  \
-  args.n_units = (N);                                                                \
-  args.units = (UNITS);                                                              \
-  e = launch_sweep<SW, DD>(tm, args, (N) < n_sm ? (N) : n_sm, smem, ln.stream);      \
-  if (e != cudaSuccess) return e;                                                    \
-  ln.done(SW == 1 ? "score_umma_stats" : "score_umma_colsum")
-    if (d == 64) {
-      AKV_SWEEP(1, 64, u1, n1);
-      AKV_SWEEP(2, 64, u2, n2);
-    } else if (d == 128) {
-      AKV_SWEEP(1, 128, u1, n1);
-      AKV_SWEEP(2, 128, u2, n2);
-    } else {
-      AKV_SWEEP(1, 256, u1, n1);
-      AKV_SWEEP(2, 256, u2, n2);
-    }
+    if (cache) cache->encoded[slot] = 1;
+  }
+  args.r0 = r0;
+  cudaError_t e;
+#define AKV_SWEEP(SW, DD)                                                              \
+  args.units = d_units + sc.unit_off[SW - 1];                                          \
+  args.cta_begin = d_cta + sc.cta_off[SW - 1];                                         \
+  if (sc.grid[SW - 1] > 0) {                                                           \
+    e = launch_sweep<SW, DD>(tm, args, sc.grid[SW - 1], smem, ln.stream);              \
+    if (e != cudaSuccess) return e;                                                    \
+    ln.done(SW == 1 ? "score_umma_stats" : "score_umma_colsum");                      \
+  }
+  if (d == 64) {
+    AKV_SWEEP(1, 64);
+    AKV_SWEEP(2, 64);
+  } else if (d == 128) {
+    AKV_SWEEP(1, 128);
+    AKV_SWEEP(2, 128);
+  } else {
+    AKV_SWEEP(1, 256);
+    AKV_SWEEP(2, 256);
+  }
 #undef AKV_SWEEP
-  }
-  if (cache && !reuse) {
-    cache->q = q;
-    cache->k = k;
-    cache->plan_id = plan_id;
-    cache->page_size = sh.page_size;
-  }
   return cudaSuccess;
 }
 

@@ -102,7 +102,8 @@ cudaError_t launch_select(const Shape& sh, const ReqDesc* d_reqs, const float* s
   const size_t smem = static_cast<size_t>(smem_keys) * sizeof(uint32_t);
   cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int grid = sh.total_heads < 148 * 4 ? sh.total_heads : 148 * 4;
+  const int max_grid = device_sm_count() * 4;
+  const int grid = sh.total_heads < max_grid ? sh.total_heads : max_grid;
   select_kernel<<<grid, kSelThreads, smem, ln.stream>>>(sh, d_reqs, smoothed, budgets, cu_kept, kept_idx, smem_keys,
                                                         status);
   ln.done("select");
@@ -117,7 +118,7 @@ cudaError_t launch_gather(const Shape& sh, const ReqDesc* d_reqs, const int32_t*
   const int chunks_per_row = sh.head_dim / elems_per_chunk;  // 8 .. 64: head_dim is 64, 128 or 256
   int log2_chunks = 0;
   while ((1 << log2_chunks) < chunks_per_row) ++log2_chunks;
-  gather_kernel<<<dim3(148 * 8), dim3(256), 0, ln.stream>>>(sh, d_reqs, cu_kept, kept_idx, (const uint4*)k, (const uint4*)v,
+  gather_kernel<<<dim3(device_sm_count() * 8), dim3(256), 0, ln.stream>>>(sh, d_reqs, cu_kept, kept_idx, (const uint4*)k, (const uint4*)v,
                                                          (uint4*)k_out, (uint4*)v_out, log2_chunks, elems_per_chunk,
                                                          head_begin, head_end);
   cudaError_t e = cudaGetLastError();

@@ -20,6 +20,8 @@ from __future__ import annotations
 
 import dataclasses
 import math
+import os
+from concurrent.futures import ThreadPoolExecutor
 from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
@@ -137,11 +139,12 @@ def _ar1_inplace(x: np.ndarray, rho: float) -> None:
 
 
 def generate(spec: WorkloadSpec, seed: int = 0, layers: Optional[int] = None,
-             layer_range: Optional[Tuple[int, int]] = None) -> Workload:
+             layer_range: Optional[Tuple[int, int]] = None, workers: Optional[int] = None) -> Workload:
     """Draw one workload. `layers` truncates the stack (the first `layers` layers) for small parity cases;
     budgets are then computed for the truncated stack. `layer_range` = (l0, l1) draws only layers l0..l1-1 of
     that stack, bit-identical to the same layers of the full draw (a layer shard of a multi-GPU run): q, k, v hold
-    l1 - l0 layers, while head_scores and total_budget stay those of the whole stack, which the allocation needs."""
+    l1 - l0 layers, while head_scores and total_budget stay those of the whole stack, which the allocation needs.
+    `workers`: threads drawing (request, layer) pairs side by side (the result does not depend on it)."""
     if layers is not None:
         spec = dataclasses.replace(spec, n_layers=int(layers))
     NL, Hq, Hkv, d, W = spec.n_layers, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.window
@@ -158,28 +161,39 @@ def generate(spec: WorkloadSpec, seed: int = 0, layers: Optional[int] = None,
     v = np.zeros((l1 - l0, Hkv, sumL, d), dtype=st)
     q = np.zeros((len(lens), l1 - l0, W, Hq, d), dtype=st)
     S = np.zeros((len(lens), NL, Hkv), dtype=np.float32)
-    for r, L in enumerate(lens):
+    def draw_layer(r: int, l: int) -> None:
+        # every (request, layer) has a generator of its own, so the draw does not depend on the order of the calls
+        L = lens[r]
         n_audio = int(round(spec.audio_frac[r] * L))
+        rng = np.random.Generator(np.random.Philox(key=[seed, (r << 20) + l + 1]))
+        for h in range(Hkv):
+            rho = spec.ar_rho if spec.ar_rho_range is None else float(rng.uniform(*spec.ar_rho_range))
+            for dst, is_k in ((k, True), (v, False)):
+                x = rng.standard_normal(size=(L, d), dtype=np.float32)
+                _ar1_inplace(x[:n_audio], rho)
+                if is_k and spec.n_sink:
+                    x[: spec.n_sink] *= 8.0
+                dst[l - l0, h, cu[r]:cu[r] + L] = _store(x, spec.dtype)
+            # window queries of this KV head's group; window tokens inside the audio segment continue an AR(1) chain
+            xq = rng.standard_normal(size=(W, G * d), dtype=np.float32)
+            n_aw = max(0, min(W, n_audio - (L - W)))
+            _ar1_inplace(xq[:n_aw], rho)
+            q[r, l - l0, :, h * G:(h + 1) * G, :] = _store(xq, spec.dtype).reshape(W, G, d)
+
+    for r, L in enumerate(lens):
         rng_s = np.random.Generator(np.random.Philox(key=[seed, 1000 + r]))
         if spec.head_score_dist == "uniform":
             S[r] = rng_s.uniform(0.0, 1.0, size=(NL, Hkv)).astype(np.float32)
         else:
             S[r] = rng_s.beta(0.5, 2.0, size=(NL, Hkv)).astype(np.float32)
-        for l in range(l0, l1):
-            rng = np.random.Generator(np.random.Philox(key=[seed, (r << 20) + l + 1]))
-            for h in range(Hkv):
-                rho = spec.ar_rho if spec.ar_rho_range is None else float(rng.uniform(*spec.ar_rho_range))
-                for dst, is_k in ((k, True), (v, False)):
-                    x = rng.standard_normal(size=(L, d), dtype=np.float32)
-                    _ar1_inplace(x[:n_audio], rho)
-                    if is_k and spec.n_sink:
-                        x[: spec.n_sink] *= 8.0
-                    dst[l - l0, h, cu[r]:cu[r] + L] = _store(x, spec.dtype)
-                # window queries of this KV head's group; window tokens inside the audio segment continue an AR(1) chain
-                xq = rng.standard_normal(size=(W, G * d), dtype=np.float32)
-                n_aw = max(0, min(W, n_audio - (L - W)))
-                _ar1_inplace(xq[:n_aw], rho)
-                q[r, l - l0, :, h * G:(h + 1) * G, :] = _store(xq, spec.dtype).reshape(W, G, d)
+    jobs = [(r, l) for r in range(len(lens)) for l in range(l0, l1)]
+    n_workers = min(len(jobs), workers if workers is not None else min(16, os.cpu_count() or 1))
+    if n_workers > 1:
+        with ThreadPoolExecutor(n_workers) as pool:
+            list(pool.map(lambda rl: draw_layer(*rl), jobs))
+    else:
+        for rl in jobs:
+            draw_layer(*rl)
     B = np.array([kept_total(spec, L) for L in lens], dtype=np.int64)
     base = base_per_head(spec, min(lens))
     if layer_range is None:

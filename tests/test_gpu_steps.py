@@ -33,6 +33,10 @@ SCORE_CASES = [
     ("bf16_d256_g4_w32", lambda: wl.generate(_small_spec("bf16", 8, 2, 256, [1111], 32))),
     ("bf16_d128_g8_w33_short", lambda: wl.generate(_small_spec("bf16", 8, 1, 128, [34, 35, 97], 33))),
     ("bf16_d128_g7_w64", lambda: wl.generate(_small_spec("bf16", 7, 1, 128, [2100], 64))),
+    # more query rows than one Q tile holds: the window is scored in chunks of rows whose column sums add up
+    ("bf16_d128_g7_w48_two_chunks", lambda: wl.generate(_small_spec("bf16", 14, 2, 128, [1300, 411], 48, layers=2))),
+    ("bf16_d256_g4_w64_two_chunks", lambda: wl.generate(_small_spec("bf16", 8, 2, 256, [900], 64))),
+    ("bf16_d64_g8_w100_four_chunks", lambda: wl.generate(_small_spec("bf16", 8, 1, 64, [1777], 100))),
 ]
 
 
@@ -90,7 +94,7 @@ def test_score_and_smooth_parity_at_full_length(B, name, make):
     kstar = torch.full((prob.total_heads,), -1, dtype=torch.int32, device="cuda")
     B.audiokv_smooth(ctx, prob, scores, out, kstar)
     torch.cuda.synchronize()
-    assert ctx.last_device_status() == 0
+    assert ctx.last_device_status() == 0 and ctx.last_score_path() == "tcgen05"
     g, gs, gk = scores.cpu().numpy(), out.cpu().numpy(), kstar.cpu().numpy()
     o, wm = oracle_scores(w, 0)
     P = s.seq_lens[0] - s.window
