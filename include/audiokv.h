@@ -144,8 +144,8 @@ int audiokv_create(audiokv_ctx** ctx, int device, size_t workspace_bytes);
  * Stream capture: every device-buffer entry point may be recorded into a CUDA graph, once the
  * context has seen its params in a call OUTSIDE capture (the first call with a new shape copies
  * the plan up from pageable memory and waits for it; inside a capture it returns AUDIOKV_ECUDA
- * and says so in audiokv_last_cuda_error). audiokv_evict forks to a stream of the context for the
- * allocation and joins back, which a capture follows. The host-buffer call waits on the host and
+ * and says so in audiokv_last_cuda_error). Every kernel of audiokv_evict goes to the caller's stream
+ * (some as programmatic dependents of the one before). The host-buffer call waits on the host and
  * cannot be captured. */
 
 /* Frees the workspace. The caller makes sure no call on this context is still running. */

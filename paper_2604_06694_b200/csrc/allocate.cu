@@ -35,6 +35,7 @@ __global__ void __launch_bounds__(kAllocThreads)
 allocate_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restrict__ head_scores, BudgetArgs args,
                 int32_t* __restrict__ budgets, int32_t* __restrict__ cu_kept, int* __restrict__ status) {
   extern __shared__ long long sm[];
+  chain_release();  // the first scoring sweep, which needs nothing from here, may start beside this kernel
   const int N = sh.heads_per_req;
   long long* Sq = sm;            // [N] quantised scores
   long long* tk = Sq + N;        // [N] share above the floor
@@ -169,6 +170,7 @@ budget_prefix_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const int32_t* 
                      int32_t* __restrict__ budgets, int32_t* __restrict__ cu_kept, int* __restrict__ status) {
   __shared__ long long warp_sum[32];
   __shared__ long long carry;
+  chain_release();  // the first scoring sweep, which needs nothing from here, may start beside this kernel
   if (threadIdx.x == 0) carry = 0;
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

@@ -476,7 +476,7 @@ int build_plan(const audiokv_params* p, Plan* pl) {
   L.order = off;       off = align_up(off + sizeof(int32_t) * pl->sss_order.size());
   {
     // softmax statistics: [head][slab][row] for the FMA kernels, [head][part][group][row] for the tensor-core ones
-    const size_t slots = std::max<size_t>(pl->n_slab, static_cast<size_t>(pl->score_parts) * 2);
+    const size_t slots = std::max<size_t>(pl->n_slab, static_cast<size_t>(pl->score_parts) * score_stat_sets());
     L.stats = off;     off = align_up(off + sizeof(float2) * static_cast<size_t>(sh.total_heads) * slots * sh.window * sh.group);
   }
   L.fft_scratch = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(pl->scratch_per_block) * pl->sss_grid);
@@ -563,7 +563,7 @@ int* d_status(audiokv_ctx* c) { return reinterpret_cast<int*>(c->ws + c->plan.la
 
 // head_end >= 0 (one request, tensor-core path only): the heads [head_begin, head_end) alone.
 int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cudaStream_t stream, int head_begin = 0,
-             int head_end = -1) {
+             int head_end = -1, bool beside = false) {
   Plan& pl = ctx->plan;
   Launch ln{stream, &ctx->launches, &ctx->prof};
   float2* stats = reinterpret_cast<float2*>(ctx->ws + pl.lay.stats);
@@ -573,7 +573,7 @@ int do_score(audiokv_ctx* ctx, const void* q, const void* k, float* scores, cuda
     e = launch_score_umma(pl.sh, pl.reqs.data(), reinterpret_cast<const ScoreUnit*>(ctx->ws + pl.lay.units),
                           reinterpret_cast<const int32_t*>(ctx->ws + pl.lay.ctas), pl.schedules.data(),
                           static_cast<int>(pl.schedules.size()), q, k, scores, stats, pl.score_parts, d_status(ctx), ln,
-                          head_begin, head_end, &ctx->score_maps, ctx->plan_id);
+                          head_begin, head_end, &ctx->score_maps, ctx->plan_id, beside);
   }
   if (head_end >= 0 && e != cudaSuccess) return cuda_fail(ctx, e);  // no head ranges in the FMA kernel
   ctx->score_path = 1;
@@ -870,21 +870,14 @@ int audiokv_evict(audiokv_ctx* ctx, const audiokv_params* p, const void* q_win, 
   float* ws_scores = reinterpret_cast<float*>(ctx->ws + pl.lay.scores);
   int32_t* ws_kstar = reinterpret_cast<int32_t*>(ctx->ws + pl.lay.kstar);
   profile_begin(ctx, s);
-  // The budgets depend on nothing the GPU computes, and only the selection needs them: the allocation
-  // runs on the context's side stream beside the scoring (on the caller's stream while per-kernel
-  // timing is on, so that every kernel is timed alone).
-  const bool beside = !ctx->prof.on;
-  cudaError_t e;
-  if (beside) {
-    if ((e = cudaEventRecord(ctx->fork, s)) != cudaSuccess) return cuda_fail(ctx, e);
-    if ((e = cudaStreamWaitEvent(ctx->side, ctx->fork, 0)) != cudaSuccess) return cuda_fail(ctx, e);
-  }
-  rc = do_allocate(ctx, head_scores, total_budget, budgets, cu_kept, beside ? ctx->side : s);
-  // recorded even after a failed launch, so that the side stream always rejoins the caller's
-  if (beside && (e = cudaEventRecord(ctx->join, ctx->side)) != cudaSuccess) return cuda_fail(ctx, e);
-  if (!rc) rc = do_score(ctx, q_win, k, ws_scores, s);
-  // the selection is the first reader of the budgets: the scoring sweeps do not wait for them
-  if (beside && (e = cudaStreamWaitEvent(s, ctx->join, 0)) != cudaSuccess) return cuda_fail(ctx, e);
+  // The budgets depend on nothing the GPU computes, and only the selection needs them. The allocation kernel is
+  // launched the ordinary way (everything earlier on the stream is then complete when it starts) and lets its
+  // dependents in at once; the first scoring sweep, a programmatic dependent, runs beside it and waits for it at its
+  // own end, so that the smoothing and selection, two chained kernels later, find the budgets complete. With per-kernel
+  // timing on, every kernel waits for the one before it.
+  const bool beside = !ctx->prof.on && score_umma_takes(pl.sh);
+  rc = do_allocate(ctx, head_scores, total_budget, budgets, cu_kept, s);
+  if (!rc) rc = do_score(ctx, q_win, k, ws_scores, s, 0, -1, beside);
   if (rc) return rc;
   // the pooling variants hand their result to the selection through the score buffer itself
   float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
@@ -919,7 +912,7 @@ int audiokv_evict_budgeted(audiokv_ctx* ctx, const audiokv_params* p, const void
   Launch ln{s, &ctx->launches, &ctx->prof};
   cudaError_t e = launch_budget_prefix(pl.sh, d_reqs(ctx), budgets, ws_budgets, cu_kept, d_status(ctx), ln);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
-  if ((rc = do_score(ctx, q_win, k, ws_scores, s))) return rc;
+  if ((rc = do_score(ctx, q_win, k, ws_scores, s, 0, -1, !ctx->prof.on && score_umma_takes(pl.sh)))) return rc;
   float* ws_smoothed = pl.sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL ? ws_scores : nullptr;
   if ((rc = do_smooth(ctx, ws_scores, ws_smoothed, ws_kstar, ws_budgets, cu_kept, kept_idx, s))) return rc;
   return do_gather(ctx, cu_kept, kept_idx, k, v, k_out, v_out, s);

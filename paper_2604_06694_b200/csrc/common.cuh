@@ -187,6 +187,8 @@ constexpr int kScoreCtas = 148;
 // kernel (256 rows; 128 at head_dim 256, where only a 128-row Q tile leaves room for two K stages), 0 if G alone
 // does not fit. A head whose W * G is larger is scored in ceil(W / W_c) chunks of window rows.
 int score_window_chunk(const Shape& sh);
+// Statistics entries sweep 1 of the tensor-core scoring writes per part of a head (its epilogue groups and sets).
+int score_stat_sets();
 // Requests whose tensor maps travel with one launch (8 for a small batch, 120 for a long one).
 int score_map_chunk(int n_req);
 
@@ -210,11 +212,13 @@ struct ScoreMapCache {
 };
 // d_units / d_cta: device tables of runs and per-CTA offsets (both sweeps of every schedule). scheds: host.
 // head_end < 0: every whole-request schedule in turn; else the schedule made for heads [head_begin, head_end).
-// stats_ws: float2 [total heads][max_parts][2][W * G].
+// stats_ws: float2 [total heads][max_parts][score_stat_sets()][W * G].
+// beside: the kernel launched just before on the stream is the library's own budget kernel (ordinary launch, calls
+// chain_release at once): the first sweep then runs beside it instead of after it.
 cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* d_units, const int32_t* d_cta,
                               const ScoreSchedule* scheds, int n_sched, const void* q, const void* k, float* scores,
                               float2* stats_ws, int max_parts, int* status, Launch ln, int head_begin = 0,
-                              int head_end = -1, ScoreMapCache* cache = nullptr, uint64_t plan_id = 0);
+                              int head_end = -1, ScoreMapCache* cache = nullptr, uint64_t plan_id = 0, bool beside = false);
 
 // sss.cu
 cudaError_t launch_fft_tables(int n_plans, float2* d_tables, const FftPlan* d_plans, Launch ln);

@@ -40,10 +40,15 @@ namespace akv {
 namespace {
 
 constexpr int kTileKeys = 128;    // keys per K tile (UMMA M in sweep 2, N in sweep 1)
-constexpr int kEpiWarps = 8;      // two epilogue groups of four warps (one warp per TMEM lane quarter)
-constexpr int kProducerWarp = kEpiWarps;
-constexpr int kMmaWarp = kEpiWarps + 1;  // and the next one: an MMA thread per epilogue group
-constexpr int kThreads = (kEpiWarps + 3) * 32;
+// Epilogue warps: two groups of one or two sets of four warps (one warp per TMEM lane quarter). Sweep 1 runs two sets
+// per group, which split the key columns of every part (measured: 92 us against 104 with one set; its maxima leave
+// the special-function unit idle often enough for a second pair of warps per scheduler to pay); sweep 2 runs one set
+// (88 us against 91: with one set a thread keeps all the registers it wants and part of the exponentials goes to the FMA
+// pipe). After the epilogue warps come the producer warp and the two MMA warps.
+constexpr int epi_sets(int sweep) { return sweep == 1 ? 2 : 1; }
+constexpr int epi_warps(int sweep) { return 8 * epi_sets(sweep); }
+constexpr int n_threads(int sweep) { return (epi_warps(sweep) + 3) * 32; }
+constexpr int kStatSets = 2 * epi_sets(1);  // statistics entries sweep 1 writes per part: [group][set]
 constexpr uint32_t kTmemCols = 512;  // four accumulator buffers of 128 columns: [group][buffer]
 constexpr int kMaxStages = 8;
 constexpr long long kWaitCycles = 2000000000LL;  // about one second: default limit of every wait on an mbarrier
@@ -75,6 +80,7 @@ struct UmmaArgs {
   int r0;         // first request of this launch: request r uses maps q[r - r0], k[r - r0]
   int w_chunk;    // window rows of a run's Q tile (the whole window, or a share of it when W * G exceeds the tile)
   int accumulate; // sweep 2: the head is scored in several chunks of window rows, whose column sums add up in `scores`
+  int beside;     // sweep 1 runs beside the kernel launched before it (see launch_score_umma) and waits for it at its end
   long long wait_cycles;  // limit of a wait on an mbarrier, in SM clock cycles
 };
 
@@ -459,7 +465,7 @@ __device__ __forceinline__ void colsum_part(const uint32_t (&r)[32], const float
 }
 
 template <int SWEEP, int D, int CAP>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(n_threads(SWEEP), 1)
 score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -475,6 +481,8 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
   const Shape& sh = a.sh;
   const int G = sh.group, R = a.w_chunk * G;  // query rows of a run's Q tile; Rt: of the head (statistics layout)
   const int Rt = sh.window * G;
+  constexpr int kSets = epi_sets(SWEEP), kEpiWarps = epi_warps(SWEEP), kThreads = n_threads(SWEEP);
+  constexpr int kProducerWarp = kEpiWarps, kMmaWarp = kEpiWarps + 1;  // and kEpiWarps + 2: an MMA thread per group
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = a.n_stages;
   const long long wl = a.wait_cycles;
@@ -496,9 +504,9 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
     for (int g = 0; g < 2; ++g) {
       for (int b = 0; b < 2; ++b) {
         mbar_init(smem_u32(&sm->acc_full[g][b]), 1);
-        mbar_init(smem_u32(&sm->acc_empty[g][b]), 4);  // the four warps of the group
+        mbar_init(smem_u32(&sm->acc_empty[g][b]), 4 * kSets);  // the warps of the group
       }
-      mbar_init(smem_u32(&sm->grp_bar[g]), 128);
+      mbar_init(smem_u32(&sm->grp_bar[g]), 128 * kSets);
     }
     mbar_init(smem_u32(&sm->drain[0]), 1);
     mbar_init(smem_u32(&sm->drain[1]), 1);
@@ -524,7 +532,10 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
   // and Q) and only then lets sweep 2 be brought in. A CTA of sweep 2 therefore starts on inputs that are
   // final: its copies and MMAs begin as soon as a CTA of sweep 1 has left the SM, and only its epilogue waits
   // (below) for sweep 1 to finish, since only the statistics come from there.
-  if (SWEEP == 1) chain_wait();
+  // When the kernel before sweep 1 is the library's own budget kernel, launched the ordinary way (so that everything
+  // earlier on the stream is complete) and needing nothing sweep 1 touches, sweep 1 runs beside it and waits for it
+  // only at its end: the kernels after it then find the budgets complete through the chain of waits.
+  if (SWEEP == 1 && !a.beside) chain_wait();
   chain_release();
   const uint32_t tmem_base = sm->tmem_base;
 
@@ -670,9 +681,9 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
       }
     }
   } else {
-    // ---- epilogue: two groups of four warps; warp w reads TMEM lanes 32 (w % 4) .. +31 ----
-    const int g = warp >> 2, quarter = warp & 3;
-    const int gl = quarter * 32 + lane;  // thread index inside the group = TMEM lane
+    // ---- epilogue: two groups of kSets sets of four warps; warp w reads TMEM lanes 32 (w % 4) .. +31 ----
+    const int g = warp / (4 * kSets), set = (warp >> 2) % kSets, quarter = warp & 3;
+    const int gl = quarter * 32 + lane;  // TMEM lane
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + 2 * g * 128;
     const float sl = sh.scale_log2e, inv_sl = 1.0f / sl;
     int it = 0, prev_u = -1, heads = 0, qc = 0;
@@ -687,15 +698,15 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
       const int live_rows = U.wn * G;  // query rows of this run (the Q tile may hold more: padding, a short last chunk)
       if (SWEEP == 2 && U.qid != prev_u) {
         // Merge the parts' statistics of this head: negc[row] = -(max + log2 sum); padding rows get -inf. Each group
-        // keeps a copy of its own (two rows per thread), in two versions by head parity: a warp of the group that is
-        // still on the head before reads the other version, and none can be two heads behind the barrier below.
+        // keeps a copy of its own, in two versions by head parity: a warp of the group that is still on the head before
+        // reads the other version, and none can be two heads behind the barrier below.
         float* dst = sm->negc[g][heads & 1];
-        for (int rr = gl; rr < 256; rr += 128) {
+        for (int rr = set * 128 + gl; rr < 256; rr += 128 * kSets) {
           float c = -INFINITY;
           if (rr < live_rows) {
-            const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.max_parts * 2 * Rt + U.w0 * G + rr;
+            const float2* hs = a.stats + static_cast<int64_t>(U.u) * a.max_parts * kStatSets * Rt + U.w0 * G + rr;
             float M = -INFINITY, Zt = 0.f;
-            const int n_ent = U.head_parts * 2;
+            const int n_ent = U.head_parts * kStatSets;
             for (int s0 = 0; s0 < n_ent; s0 += 8) {
               float2 sv[8];
 #pragma unroll
@@ -761,8 +772,15 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
           const bool masked = kt + kTileKeys - 1 > U.P;       // sweep 1: the tile reaches into the window: causal mask
           const int last_col = U.P + U.w0 + row / G - kt;     // sweep 1: last visible key of this row, relative to the tile
           const float* ncp = SWEEP == 2 ? nc + (p == 0 ? 0 : cols0) : nullptr;
+          if (kSets == 2 && 2 * set >= n_ch) {  // this set has no columns in the part
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ebar);
+          }
+          // one set: both steps of the part, unrolled; two sets: each takes one step (one copy of the code)
 #pragma unroll
-          for (int st = 0; st < 2; ++st) {
+          for (int i = 0; i < (kSets == 2 ? 1 : 2); ++i) {
+            const int st = kSets == 2 ? set : i;
             const int c0 = 2 * st;  // first chunk of 32 columns of this step
             if (c0 < n_ch) {
               const bool has_b = c0 + 1 < n_ch;
@@ -779,7 +797,7 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
                 if (b_half) tmem_wait_lo(rb);
                 else tmem_wait(rb);
               }
-              if (c0 + 2 >= n_ch) {  // the part is in registers: its buffer goes back to the MMA thread
+              if (kSets == 2 || c0 + 2 >= n_ch) {  // this warp's columns of the part are in registers: its buffer goes back
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(ebar);
@@ -812,7 +830,7 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
       if (SWEEP == 1) {
         // this group's share of the run (every second tile): one entry per row, merged by sweep 2 with the other
         // group's and the other parts'; a group without a tile in the run writes an empty entry
-        float2* out = a.stats + ((static_cast<int64_t>(U.u) * a.max_parts + U.part) * 2 + g) * Rt + U.w0 * G;
+        float2* out = a.stats + ((static_cast<int64_t>(U.u) * a.max_parts + U.part) * kStatSets + g * kSets + set) * Rt + U.w0 * G;
 #pragma unroll
         for (int p = 0; p < 2; ++p)
           if (p < n_parts && p * 128 + gl < live_rows) out[p * 128 + gl] = make_float2(m_ref[p], Z[p]);
@@ -821,6 +839,7 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
   }
 
   // ---- teardown ----
+  if (SWEEP == 1 && a.beside) chain_wait();
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && sm->abort) atomicExch(a.status, AUDIOKV_ETIMEOUT);
@@ -864,14 +883,14 @@ cudaError_t launch_sweep(const TmapPack<CAP>& tm, const UmmaArgs& args, int grid
   auto kern = score_umma_kernel<SWEEP, D, CAP>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  return launch_chained(kern, dim3(grid), dim3(kThreads), smem, stream, tm, args);
+  return launch_chained(kern, dim3(grid), dim3(n_threads(SWEEP)), smem, stream, tm, args);
 }
 
 template <int CAP>
 cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* d_units, const int32_t* d_cta,
                                   const ScoreSchedule& sc, int slot, const void* q, const void* k, float* scores,
                                   float2* stats_ws, int max_parts, int* status, Launch ln, ScoreMapCache* cache,
-                                  uint64_t plan_id);
+                                  uint64_t plan_id, bool beside);
 
 }  // namespace
 
@@ -900,15 +919,17 @@ bool score_umma_takes(const Shape& sh) {
   return wc >= 1 && wc <= 256 && sh.group <= 256;
 }
 
+int score_stat_sets() { return kStatSets; }
+
 int score_map_chunk(int n_req) { return n_req <= kMapChunkSmall ? kMapChunkSmall : kMapChunkLarge; }
 
 cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* d_units, const int32_t* d_cta,
                               const ScoreSchedule* scheds, int n_sched, const void* q, const void* k, float* scores,
                               float2* stats_ws, int max_parts, int* status, Launch ln, int head_begin, int head_end,
-                              ScoreMapCache* cache, uint64_t plan_id) {
+                              ScoreMapCache* cache, uint64_t plan_id, bool beside) {
   if (!score_umma_takes(sh)) return cudaErrorNotSupported;
   // every schedule that covers whole requests, in order; or the one schedule made for this range of heads
-  bool any = false;
+  bool any = false, any_before = false;  // only the first launch follows the caller's kernel
   for (int i = 0; i < n_sched; ++i) {
     const ScoreSchedule& sc = scheds[i];
     if (head_end < 0 ? !sc.whole_requests : (sc.whole_requests || sc.head_begin != head_begin || sc.head_end != head_end))
@@ -918,9 +939,10 @@ cudaError_t launch_score_umma(const Shape& sh, const ReqDesc* h_reqs, const Scor
     const int slot = sc.whole_requests ? sc.r_begin / score_map_chunk(sh.n_req) : 0;
     cudaError_t e = sh.n_req <= kMapChunkSmall
                         ? launch_score_umma_cap<kMapChunkSmall>(sh, h_reqs, d_units, d_cta, sc, slot, q, k, scores, stats_ws,
-                                                                max_parts, status, ln, cache, plan_id)
+                                                                max_parts, status, ln, cache, plan_id, beside && !any_before)
                         : launch_score_umma_cap<kMapChunkLarge>(sh, h_reqs, d_units, d_cta, sc, slot, q, k, scores, stats_ws,
-                                                                max_parts, status, ln, cache, plan_id);
+                                                                max_parts, status, ln, cache, plan_id, beside && !any_before);
+    any_before = true;
     if (e != cudaSuccess) return e;
   }
   return any ? cudaSuccess : cudaErrorInvalidValue;
@@ -932,7 +954,7 @@ template <int CAP>
 cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const ScoreUnit* d_units, const int32_t* d_cta,
                                   const ScoreSchedule& sc, int slot, const void* q, const void* k, float* scores,
                                   float2* stats_ws, int max_parts, int* status, Launch ln, ScoreMapCache* cache,
-                                  uint64_t plan_id) {
+                                  uint64_t plan_id, bool beside) {
   using Pack = TmapPack<CAP>;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
@@ -949,6 +971,7 @@ cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const 
   args.r_pad = (R + 15) / 16 * 16;
   args.w_chunk = w_chunk;
   args.accumulate = w_chunk < sh.window ? 1 : 0;
+  args.beside = beside ? 1 : 0;
   args.wait_cycles = score_wait_cycles();
   const int q_bytes = args.q_rows * d * 2, stage = kTileKeys * d * 2;
   const int room = kSmemLimit - 1024 - static_cast<int>(sizeof(Small)) - q_bytes;

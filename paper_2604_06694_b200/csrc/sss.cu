@@ -645,8 +645,11 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
   __shared__ double red[32];
   __shared__ int s_kstar;
   __shared__ SelectSmem ssm;
+  // Launched as a programmatic dependent: the block is brought in while the kernel before it drains, reads its plan
+  // and stages its tables (written when the plan was made, not by the kernels of the pass), and waits for that
+  // kernel only where it first touches the scores.
   chain_release();
-  chain_wait();
+  bool waited = false;
 
   int loaded_plan = -1;  // plan whose tables sit in shared memory
   for (int slot = blockIdx.x; slot < n_order; slot += gridDim.x) {
@@ -691,6 +694,10 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     const float* x = scores + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P;
     float* y = smoothed ? smoothed + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P : nullptr;
 
+    if (!waited) {
+      chain_wait();
+      waited = true;
+    }
     if (sh.smooth_mode >= AUDIOKV_SMOOTH_AVG_POOL) {
       // Variant: local pooling instead of the spectral filter. The sequence is staged first (scores and smoothed
       // may be the same array), pooled over |i - j| <= pool_kernel / 2 (average: zero padding counts in the
@@ -998,11 +1005,11 @@ cudaError_t launch_sss(const Shape& sh, const ReqDesc* d_reqs, const FftPlan* d_
                        Launch ln) {
   cudaError_t e = cudaFuncSetAttribute(sss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   if (e != cudaSuccess) return e;
-  sss_kernel<<<grid, kSssThreads, smem_bytes, ln.stream>>>(sh, d_reqs, d_plans, d_tables, scores, smoothed, kstar,
-                                                           scratch, scratch_per_block, order, n_order, first_head, budgets,
-                                                           cu_kept, kept_idx, status);
+  e = launch_chained(sss_kernel, dim3(grid), dim3(kSssThreads), smem_bytes, ln.stream, sh, d_reqs, d_plans, d_tables, scores,
+                     smoothed, kstar, scratch, scratch_per_block, order, n_order, first_head, budgets, cu_kept, kept_idx,
+                     status);
   ln.done(budgets ? "sss_select" : "sss");
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace akv

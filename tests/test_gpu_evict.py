@@ -110,7 +110,7 @@ def test_evict_config1_full(B):
 def test_evict_config2_three_layers(B):
     w = wl.generate(wl.config(1), layers=3)
     ties = check_against_oracle(w, run_evict(B, w))
-    assert ties <= 8
+    assert ties <= 4          # observed: none
 
 
 def test_evict_config4_one_layer_with_sinks(B):

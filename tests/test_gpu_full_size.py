@@ -26,7 +26,9 @@ def test_config2_all_layers_as_benchmarked(B):
     g = run_evict(B, w)
     assert g["launches"] == 5 + 2          # the pass (5 kernels) after the two table kernels of the first call
     ties = check_against_oracle(w, g)
-    assert ties <= 3 * 112                 # tokens exchanged at near ties, over 112 heads
+    # tokens exchanged at near ties over the 112 heads, and heads whose cut-off had to be handed to the oracle:
+    # observed 4 to 6 and 0 (the bounds leave a margin of a few tokens, not a multiple)
+    assert ties <= 16 and g["forced_kstar_heads"] == 0
 
 
 @pytest.mark.parametrize("keep,W,layers", [(0.4, 32, 4), (0.2, 32, 2), (0.6, 32, 2), (0.4, 16, 2), (0.4, 64, 2)])
@@ -34,13 +36,15 @@ def test_config3_long_context_sweep(B, keep, W, layers):
     spec = dataclasses.replace(wl.config(2), keep=keep, window=W)
     w = wl.generate(spec, layers=layers)
     assert w.spec.seq_lens == [32768]
-    check_against_oracle(w, run_evict(B, w))
+    g = run_evict(B, w)
+    assert check_against_oracle(w, g) <= 16 and g["forced_kstar_heads"] == 0     # observed: up to 6 tokens, no head
 
 
 def test_config4_sinks_L16k(B):
     w = wl.generate(wl.config(3), layers=6)
     assert w.spec.seq_lens == [16384] and w.spec.n_sink == 4
-    check_against_oracle(w, run_evict(B, w))
+    g = run_evict(B, w)
+    assert check_against_oracle(w, g) <= 8 and g["forced_kstar_heads"] <= 1      # observed: 2 tokens, no head
 
 
 def test_config5_ragged_batch_of_eight_in_one_launch(B):
@@ -48,7 +52,7 @@ def test_config5_ragged_batch_of_eight_in_one_launch(B):
     assert len(w.spec.seq_lens) == 8 and min(w.spec.seq_lens) >= 2048 and max(w.spec.seq_lens) <= 32768
     g = run_evict(B, w)
     assert g["launches"] == 5 + 2
-    check_against_oracle(w, g)
+    assert check_against_oracle(w, g) <= 24 and g["forced_kstar_heads"] <= 1     # observed: 10 tokens over 48 heads, no head
 
 
 def test_maximum_sequence_length(B):

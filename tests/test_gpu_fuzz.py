@@ -43,8 +43,8 @@ def test_random_shape(B, case):
     w = wl.generate(spec, seed=case)
     g = run_evict(B, w)
     ties = check_against_oracle(w, g)
-    heads = spec.n_layers * spec.n_kv_heads * len(spec.seq_lens)
-    assert ties <= 4 * heads, (spec, ties)
+    # observed over the 40 cases: no token exchanged at a near tie, one head in one case with a moved cut-off
+    assert ties <= 4 and g["forced_kstar_heads"] <= 2, (spec, ties, g["forced_kstar_heads"])
 
 
 @pytest.mark.parametrize("case", range(12))

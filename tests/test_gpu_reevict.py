@@ -5,6 +5,7 @@ cache every head has its own length, so the oracle side is the same four steps a
 a one-layer, one-KV-head request made of the head's own rows and its group's window queries.
 """
 import dataclasses
+import os
 
 import numpy as np
 import pytest
@@ -80,6 +81,10 @@ def check_heads(c, g, budgets=None, heads=None):
         ties += check_kept(idx, sm, int(budgets[u]) - W, n - W, W, f"head {u}")
         assert np.array_equal(g["k_out"][a:b], c.k[c.cu[u]:c.cu[u + 1]][idx]), f"K rows of head {u}"
         assert np.array_equal(g["v_out"][a:b], c.v[c.cu[u]:c.cu[u + 1]][idx]), f"V rows of head {u}"
+    log = os.environ.get("AUDIOKV_PARITY_LOG")
+    if log:
+        with open(log, "a") as f:
+            f.write(f"reevict {s.name} layers={NL} heads={TH} W={W} tie_tokens={ties}\n")
     return ties
 
 
