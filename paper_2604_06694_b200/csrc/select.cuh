@@ -21,6 +21,7 @@ constexpr int kSelBins = 2048;  // 11-bit digits: three passes (11 + 11 + 10 bit
 struct SelectSmem {
   int hist[kSelBins];
   int wsum[32];
+  int weq[32];
   uint32_t prefix;
   int want;
 };
@@ -49,24 +50,31 @@ __device__ __forceinline__ int block_excl_scan_int(int v, int* wsum, int* total)
 // Writes to `out` the k prefix tokens (of P) with the largest keys, ties to the lower index, in
 // ascending token order, then the W window tokens P .. P+W-1. key_at(j) gives the key of token j.
 // Every thread of the block calls this with the same arguments. Three radix passes (11, 11 and 10 bits) find
-// the k-th largest key; the bin that holds it is located by a block-wide scan over the counts.
+// the k-th largest key; the bin that holds it is located by a block-wide scan over the counts. The compaction
+// gives every warp a contiguous stretch of tokens, 32 neighbours at a time: ballots rank the kept tokens inside
+// the warp, one exchange of the warps' totals ranks the warps.
 template <typename KeyAt>
 __device__ __forceinline__ void select_topk(KeyAt key_at, int P, int W, int k, int32_t* __restrict__ out,
                                             SelectSmem* sm, int* __restrict__ status) {
+  static_assert(kSelBins == 2 * kSelThreads, "every thread owns two bins of the histogram");
   uint32_t thr = 0;  // key of the k-th largest element
   int need_eq = 0;   // how many elements equal to thr are kept (those with the lowest indices)
   if (k > 0 && k < P) {
+    // thread t owns bins 2047 - 2t and 2046 - 2t (descending): `above` counts the keys in higher bins
+    const int b_hi = kSelBins - 1 - 2 * static_cast<int>(threadIdx.x), b_lo = b_hi - 1;
     __syncthreads();
     if (threadIdx.x == 0) {
       sm->prefix = 0u;
       sm->want = k;
     }
+    sm->hist[b_hi] = 0;
+    sm->hist[b_lo] = 0;
+#pragma unroll 1
     for (int pass = 0; pass < 3; ++pass) {
       const int shift = pass == 0 ? 21 : pass == 1 ? 10 : 0;
       const int bits = pass == 2 ? 10 : 11;
       const uint32_t dmask = (1u << bits) - 1u;
-      for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) sm->hist[b] = 0;
-      __syncthreads();
+      __syncthreads();  // the histogram is clear; prefix and want of the pass before are set
       const uint32_t prefix = sm->prefix;
       const int want = sm->want;
       const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + bits));
@@ -75,9 +83,9 @@ __device__ __forceinline__ void select_topk(KeyAt key_at, int P, int W, int k, i
         if ((key & pmask) == prefix) atomicAdd(&sm->hist[(key >> shift) & dmask], 1);
       }
       __syncthreads();
-      // thread t owns bins 2047 - 2t and 2046 - 2t (descending): `above` counts the keys in higher bins
-      const int b_hi = kSelBins - 1 - 2 * static_cast<int>(threadIdx.x), b_lo = b_hi - 1;
       const int c_hi = sm->hist[b_hi], c_lo = sm->hist[b_lo];
+      sm->hist[b_hi] = 0;  // its owner clears a bin for the next pass as soon as it has read it
+      sm->hist[b_lo] = 0;
       int tot;
       const int above = block_excl_scan_int(c_hi + c_lo, sm->wsum, &tot);
       if (above < want && want <= above + c_hi) {
@@ -87,8 +95,8 @@ __device__ __forceinline__ void select_topk(KeyAt key_at, int P, int W, int k, i
         sm->prefix = prefix | (static_cast<uint32_t>(b_lo) << shift);
         sm->want = want - above - c_hi;
       }
-      __syncthreads();
     }
+    __syncthreads();
     thr = sm->prefix;
     need_eq = sm->want;
   } else if (k == P) {
@@ -96,32 +104,56 @@ __device__ __forceinline__ void select_topk(KeyAt key_at, int P, int W, int k, i
     need_eq = P;  // every key is >= 0: keep all
   }
 
-  // ordered compaction: thread t owns the contiguous index range [a, b)
-  const int per = (P + kSelThreads - 1) / kSelThreads;
-  const int a = min(P, static_cast<int>(threadIdx.x) * per), b = min(P, a + per);
-  int n_eq = 0, n_gt = 0;
+  // ordered compaction: warp w owns tokens [w * chunk, (w + 1) * chunk), lane l looks at token j0 + l of each row of 32
+  constexpr int kWarps = kSelThreads / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t lt = (1u << lane) - 1u;
+  const int chunk = ((P + kWarps - 1) / kWarps + 31) & ~31;
+  const int c0 = min(P, warp * chunk), c1 = min(P, c0 + chunk);
+  int n_gt = 0, n_eq = 0;
   if (k > 0) {
-    for (int j = a; j < b; ++j) {
-      const uint32_t key = key_at(j);
-      n_eq += key == thr;
-      n_gt += key > thr;
+    for (int j0 = c0; j0 < c1; j0 += 32) {
+      const int j = j0 + lane;
+      const uint32_t key = j < c1 ? key_at(j) : 0u;
+      n_gt += __popc(__ballot_sync(0xffffffffu, j < c1 && key > thr));
+      n_eq += __popc(__ballot_sync(0xffffffffu, j < c1 && key == thr));
     }
   }
-  int tot;
-  const int eq_before = block_excl_scan_int(n_eq, sm->wsum, &tot);
-  int my_eq_kept = min(n_eq, max(0, need_eq - eq_before));
-  if (k == 0) my_eq_kept = 0;
-  int pos = block_excl_scan_int(n_gt + my_eq_kept, sm->wsum, &tot);
+  __syncthreads();  // wsum is free again
+  if (lane == 0) {
+    sm->wsum[warp] = n_gt;
+    sm->weq[warp] = n_eq;
+  }
+  __syncthreads();
+  // every warp ranks the warps: equal keys before warp w, then kept tokens before warp w
+  const int e = sm->weq[lane];
+  int e_inc = e;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, e_inc, o);
+    if (lane >= o) e_inc += t;
+  }
+  const int kept_w = sm->wsum[lane] + min(e, max(0, need_eq - (e_inc - e)));
+  int k_inc = kept_w;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, k_inc, o);
+    if (lane >= o) k_inc += t;
+  }
+  const int tot = __shfl_sync(0xffffffffu, k_inc, 31);
+  int eq_seen = __shfl_sync(0xffffffffu, e_inc - e, warp);
+  int pos = __shfl_sync(0xffffffffu, k_inc - kept_w, warp);
   if (k > 0) {
-    int eq_seen = eq_before;
-    for (int j = a; j < b; ++j) {
-      const uint32_t key = key_at(j);
-      bool keep = key > thr;
-      if (key == thr) {
-        keep = eq_seen < need_eq;
-        ++eq_seen;
-      }
-      if (keep) out[pos++] = j;
+    for (int j0 = c0; j0 < c1; j0 += 32) {
+      const int j = j0 + lane;
+      const uint32_t key = j < c1 ? key_at(j) : 0u;
+      const bool is_eq = j < c1 && key == thr;
+      const uint32_t b_eq = __ballot_sync(0xffffffffu, is_eq);
+      const bool keep = (j < c1 && key > thr) || (is_eq && eq_seen + __popc(b_eq & lt) < need_eq);
+      const uint32_t b_keep = __ballot_sync(0xffffffffu, keep);
+      if (keep) out[pos + __popc(b_keep & lt)] = j;
+      pos += __popc(b_keep);
+      eq_seen += __popc(b_eq);
     }
   }
   if (tot != k && threadIdx.x == 0) atomicExch(status, AUDIOKV_EDEVICE);

@@ -690,8 +690,12 @@ __device__ __forceinline__ DirectGeom direct_geom(int n, bool packed) {
   g.a = packed ? 2 : 1;
   g.M = n / g.a;
   g.rows = (g.M + kSssThreads - 1) / kSssThreads;
-  g.wt = unit_root_exact(g.a * threadIdx.x, n);
-  g.v = unit_root_exact(1, n);
+  // one accurate rotation per thread, w_1^t; w_1 is the ratio of two neighbours' and w_1^{2t} its square
+  const float2 w = unit_root_exact(threadIdx.x, n);
+  const float2 w_l0 = make_float2(__shfl_sync(0xffffffffu, w.x, 0), __shfl_sync(0xffffffffu, w.y, 0));
+  const float2 w_l1 = make_float2(__shfl_sync(0xffffffffu, w.x, 1), __shfl_sync(0xffffffffu, w.y, 1));
+  g.v = cmulc(w_l1, w_l0);
+  g.wt = packed ? cmul(w, w) : w;
   return g;
 }
 
@@ -775,26 +779,27 @@ __device__ __noinline__ int direct_cutoff(const float* __restrict__ x, int n, bo
     if (lane == 0) ds->part[warp][k] = F;
   }
   __syncthreads();
-  // warp k adds up bin k over the warps' parts (lane w reads warp w's), warp 0 the three sums
-  if (warp < kDirectBins) {
-    double t0 = warp == 0 ? ds->sums[lane][0] : static_cast<double>(ds->part[lane][warp].x);
-    double t1 = warp == 0 ? ds->sums[lane][1] : static_cast<double>(ds->part[lane][warp].y);
-    double t2 = warp == 0 ? ds->sums[lane][2] : 0.0;
+  // warp k adds up bin k over the warps' parts (lane w reads warp w's), warp 0 the three sums. (Rolled loops: this
+  // runs once, and straight-line code costs more in instruction fetches than its arithmetic takes.)
+  if (warp == 0) {
+#pragma unroll 1
+    for (int q = 0; q < 3; ++q) {
+      double t = ds->sums[lane][q];
+#pragma unroll 1
+      for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+      if (lane == 0) ds->tot[q] = t;
+      if (lane == 0 && q == 0) ds->bin[0] = make_float2(static_cast<float>(t), 0.f);
+    }
+  } else if (warp < kDirectBins) {
+    float2 t = ds->part[lane][warp];
+#pragma unroll 1
     for (int o = 16; o > 0; o >>= 1) {
-      t0 += __shfl_xor_sync(0xffffffffu, t0, o);
-      t1 += __shfl_xor_sync(0xffffffffu, t1, o);
-      if (warp == 0) t2 += __shfl_xor_sync(0xffffffffu, t2, o);
+      t.x += __shfl_xor_sync(0xffffffffu, t.x, o);
+      t.y += __shfl_xor_sync(0xffffffffu, t.y, o);
     }
     if (lane == 0) {
-      if (warp == 0) {
-        ds->tot[0] = t0;
-        ds->tot[1] = t1;
-        ds->tot[2] = t2;
-        ds->bin[0] = make_float2(static_cast<float>(t0), 0.f);
-      } else {
-        ds->energy[warp] = t0 * t0 + t1 * t1;
-        ds->bin[warp] = make_float2(static_cast<float>(t0), static_cast<float>(t1));
-      }
+      ds->energy[warp] = static_cast<double>(t.x) * t.x + static_cast<double>(t.y) * t.y;
+      ds->bin[warp] = t;
     }
   }
   __syncthreads();
