@@ -99,7 +99,7 @@ def test_reevict_bf16_two_layers(B):
     assert len(set(np.diff(c.cu).tolist())) > 4          # the heads really differ in length
     g = run_reevict(B, c)
     ties = check_heads(c, g)
-    assert ties <= 8
+    assert ties <= 4          # observed: 0
 
 
 def test_reevict_f32(B):
@@ -116,7 +116,7 @@ def test_reevict_ragged_batch_many_heads(B):
     assert len(c.new_budgets) == 132
     g = run_reevict(B, c)
     assert g["launches"] == 2 + 3 + 4 + 1 + 1      # tables, allocation x3 (64 requests each), sweeps x2 x2, smoothing, gather
-    assert check_heads(c, g) <= 60
+    assert check_heads(c, g) <= 6      # observed: 0 over 112 to 132 heads
 
 
 def test_reevict_keep_all_and_window_only(B):
