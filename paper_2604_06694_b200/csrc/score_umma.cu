@@ -464,6 +464,50 @@ __device__ __forceinline__ void colsum_part(const uint32_t (&r)[32], const float
   }
 }
 
+// Sweep 2, one part of COLS accumulator columns (a multiple of 16, at most 128) for this thread's key: the same
+// steps as the general loop below (64 columns in two register buffers, the buffer handed back once the last step
+// is in registers), with the shape known at compile time: no branch on the number of chunks or on a half-filled
+// last buffer, and the arithmetic of a step is one basic block for the scheduler. (Sweep 2 runs two epilogue warps
+// per scheduler; with the general loop a tenth of their time went to resolving those branches.)
+template <int COLS>
+__device__ __forceinline__ void colsum_cols(uint32_t taddr, const float* __restrict__ ncp, f32x2 sl2, uint32_t ebar, int lane,
+                                            uint32_t (&ra)[32], uint32_t (&rb)[32], f32x2& a0, f32x2& a1, f32x2& a2,
+                                            f32x2& a3) {
+  constexpr int n_ch = (COLS + 31) / 32;
+  constexpr bool tail = (COLS & 16) != 0;
+#pragma unroll
+  for (int st = 0; st < 2; ++st) {
+    const int c0 = 2 * st;
+    if (c0 < n_ch) {
+      const bool has_b = c0 + 1 < n_ch;
+      const bool a_half = tail && c0 == n_ch - 1, b_half = tail && c0 + 1 == n_ch - 1;
+      if (a_half) tmem_ld16_issue_lo(taddr + c0 * 32, ra);
+      else tmem_ld32_issue(taddr + c0 * 32, ra);
+      if (has_b) {
+        if (b_half) tmem_ld16_issue_lo(taddr + (c0 + 1) * 32, rb);
+        else tmem_ld32_issue(taddr + (c0 + 1) * 32, rb);
+      }
+      if (a_half) tmem_wait_lo(ra);
+      else tmem_wait(ra);
+      if (has_b) {
+        if (b_half) tmem_wait_lo(rb);
+        else tmem_wait(rb);
+      }
+      if (c0 + 2 >= n_ch) {  // the part is in registers: its buffer goes back to the MMA thread
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(ebar);
+      }
+      if (a_half) colsum_part<16>(ra, ncp + c0 * 32, sl2, a0, a1, a2, a3);
+      else colsum_part<32>(ra, ncp + c0 * 32, sl2, a0, a1, a2, a3);
+      if (has_b) {
+        if (b_half) colsum_part<16>(rb, ncp + (c0 + 1) * 32, sl2, a0, a1, a2, a3);
+        else colsum_part<32>(rb, ncp + (c0 + 1) * 32, sl2, a0, a1, a2, a3);
+      }
+    }
+  }
+}
+
 template <int SWEEP, int D, int CAP>
 __global__ void __launch_bounds__(n_threads(SWEEP), 1)
 score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
@@ -773,6 +817,15 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
             __syncwarp();
             if (lane == 0) mbar_arrive(ebar);
           }
+          if constexpr (SWEEP == 2 && kSets == 1) {
+            switch (cols) {  // the shapes of a launch: one or two of these
+#define AKV_COLS_CASE(C) case C: colsum_cols<C>(taddr, ncp, sl2, ebar, lane, ra, rb, a0, a1, a2, a3); break;
+              AKV_COLS_CASE(16) AKV_COLS_CASE(32) AKV_COLS_CASE(48) AKV_COLS_CASE(64)
+              AKV_COLS_CASE(80) AKV_COLS_CASE(96) AKV_COLS_CASE(112) AKV_COLS_CASE(128)
+#undef AKV_COLS_CASE
+              default: break;  // r_pad is a multiple of 16 and a part at most 128 columns
+            }
+          } else {
           // one set: both steps of the part, unrolled; two sets: each takes one step (one copy of the code)
 #pragma unroll
           for (int i = 0; i < (kSets == 2 ? 1 : 2); ++i) {
@@ -811,6 +864,7 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
               }
             }
           }
+          }  // general loop
         }
         if (!ok) break;
         if (SWEEP == 2) {
