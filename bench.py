@@ -324,6 +324,8 @@ def run_cuda(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     spec = wl.config(args.config)
+    if args.window or args.keep:  # the keep x window sweep of the long-context configuration (not a bench line)
+        spec = dataclasses.replace(spec, window=args.window or spec.window, keep=args.keep or spec.keep)
     sharded = args.shard == "layers"
     if sharded:
         # one request for the whole job, its layers dealt out over the ranks; no exchange step either: the budgets need
@@ -361,7 +363,8 @@ def run_cuda(args):
         e2e_ms, h2d, d2h = run_e2e(B, case.ctx, case.prob, w, spec, case.tb, case.rows, case.TH, w.torch_dtype(),
                                    barrier, world, args)
     others = []
-    if world == 1 and args.config == 1 and not args.skip_other and not sharded and not args.layers and not args.page_size:
+    if (world == 1 and args.config == 1 and not args.skip_other and not sharded and not args.layers and not args.page_size
+            and not args.window and not args.keep):
         del case
         torch.cuda.empty_cache()
         for idx in (2, 3, 4):
@@ -579,6 +582,8 @@ def main():
                     help="hold K and V in a pool of pages of this many tokens (0 = contiguous, the bench line)")
     ap.add_argument("--layers", type=int, default=None,
                     help="truncate the stack to its first LAYERS layers (small cases for profiler captures; not a bench line)")
+    ap.add_argument("--window", type=int, default=None, help="observation window W instead of the configuration's (not a bench line)")
+    ap.add_argument("--keep", type=float, default=None, help="retention ratio instead of the configuration's (not a bench line)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
