@@ -652,10 +652,11 @@ struct DirectSmem {
   float2 tab[kDirectRows][kDirectBins];          // tab[i][k] = w_k^{a kSssThreads i}
   float2 part[kSssThreads / 32][kDirectBins];    // per warp: bins 1 .. kDirectBins - 1
   double sums[kSssThreads / 32][3];              // per warp: sum x, sum x^2, alternating sum
-  double energy[kDirectBins];                    // |F_k|^2, k >= 1
-  double tot[3];                                 // sum x (= F_0), sum x^2, alternating sum (= F_{n/2} for an even n)
+  double energy[kDirectBins];                    // |F_k|^2 as it counts towards the cumulative energy
+  double tot[3];                                 // F_0 (= sum x), the energy threshold rho E, the margin of a decision
   float2 bin[kDirectBins];                       // F_k
-  int kstar;                                     // -1: not decided here
+  int kstar;                                     // stage 1: k*, -1: left to the transform, -2: the bins decide
+  int k_hi;                                      // last bin to evaluate; after stage 3: k* or -1
 };
 
 // e^{-2 pi i (j k mod n) / n}: the product is reduced exactly in integers, the angle then lies in [-pi, pi] where the
@@ -743,10 +744,59 @@ __device__ __noinline__ int direct_cutoff(const float* __restrict__ x, int n, bo
     for (int o = 16; o > 0; o >>= 1) val += __shfl_xor_sync(0xffffffffu, val, o);
     if (lane == 0) ds->sums[warp][q] = val;
   }
-  __syncthreads();  // the table is complete
+  __syncthreads();  // the table and the warps' sums are complete
+  // Stage 1, from the three sums alone (warp 0): the mean bin F_0 and, by Parseval, the total over the bins
+  // 0 .. floor(n/2). Often that settles the cut-off at bin 0, and only the T bins of the cosine band are needed; it
+  // also tells a head whose mean holds less than half of the energy asked for, which is left to the transform at once
+  // (a matter of time only: both paths compute the same function).
+  if (warp == 0) {
+    double t[3];
+#pragma unroll 1
+    for (int q = 0; q < 3; ++q) {
+      double v = ds->sums[lane][q];
+#pragma unroll 1
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      t[q] = v;
+    }
+    if (lane == 0) {
+      const int Kb = n / 2;
+      const double F0 = t[0], FN = t[2];
+      const double total = 0.5 * (static_cast<double>(n) * t[1] + F0 * F0 + ((n & 1) ? 0.0 : FN * FN));
+      const bool no_mean = smooth_mode == AUDIOKV_SMOOTH_ENERGY_NO_MEAN;
+      const double rest = fmax(total - F0 * F0, 0.0), whole = no_mean ? rest : total;
+      const double thr = static_cast<double>(rho) * whole;
+      // The rotations are good to about 1e-6, so a bin's energy is off by up to 2e-6 |F_k| F_0: a decision is taken
+      // here only when it is clear of the threshold by several times the sum of that over the bins.
+      const double margin = 1e-5 * (whole + fabs(F0) * static_cast<double>(sqrtf(static_cast<float>(rest))));
+      int ks = -2, k_hi = kDirectBins - 1;  // -2: the bins have to decide
+      if (smooth_mode == AUDIOKV_SMOOTH_FIXED_FRACTION) {
+        ks = static_cast<int>(floor(static_cast<double>(kappa) * Kb));
+      } else if (!(whole > 0.0)) {
+        ks = -1;
+      } else if (!no_mean) {
+        if (F0 * F0 >= thr + margin) ks = 0;
+        else if (F0 * F0 < 0.5 * thr) ks = -1;
+      }
+      if (ks >= 0) {
+        k_hi = ks + T;
+        if (k_hi >= kDirectBins || k_hi >= Kb) ks = -1;
+      }
+      ds->tot[0] = F0;
+      ds->tot[1] = thr;
+      ds->tot[2] = margin;
+      ds->bin[0] = make_float2(static_cast<float>(F0), 0.f);
+      ds->energy[0] = no_mean ? 0.0 : F0 * F0;
+      ds->k_hi = k_hi;
+      ds->kstar = ks;
+    }
+  }
+  __syncthreads();
+  if (ds->kstar == -1) return -1;
+  const int k_hi = ds->k_hi;
+  // Stage 2: bins 1 .. k_hi from their definition
   float2 pk = make_float2(1.f, 0.f), vk = pk;
 #pragma unroll 1
-  for (int k = 1; k < kDirectBins; ++k) {
+  for (int k = 1; k <= k_hi; ++k) {
     pk = cmul(pk, g.wt);  // w_k^{a t}
     vk = cmul(vk, g.v);   // w_k
     float2 A0 = make_float2(0.f, 0.f), A1 = A0;  // at most 64 entries per thread: their sums stay in fp32
@@ -779,18 +829,9 @@ __device__ __noinline__ int direct_cutoff(const float* __restrict__ x, int n, bo
     if (lane == 0) ds->part[warp][k] = F;
   }
   __syncthreads();
-  // warp k adds up bin k over the warps' parts (lane w reads warp w's), warp 0 the three sums. (Rolled loops: this
-  // runs once, and straight-line code costs more in instruction fetches than its arithmetic takes.)
-  if (warp == 0) {
-#pragma unroll 1
-    for (int q = 0; q < 3; ++q) {
-      double t = ds->sums[lane][q];
-#pragma unroll 1
-      for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-      if (lane == 0) ds->tot[q] = t;
-      if (lane == 0 && q == 0) ds->bin[0] = make_float2(static_cast<float>(t), 0.f);
-    }
-  } else if (warp < kDirectBins) {
+  // warp k adds up bin k over the warps' parts (lane w reads warp w's). (Rolled loops: this runs once, and
+  // straight-line code costs more in instruction fetches than its arithmetic takes.)
+  if (warp >= 1 && warp <= k_hi) {
     float2 t = ds->part[lane][warp];
 #pragma unroll 1
     for (int o = 16; o > 0; o >>= 1) {
@@ -803,37 +844,27 @@ __device__ __noinline__ int direct_cutoff(const float* __restrict__ x, int n, bo
     }
   }
   __syncthreads();
+  if (ds->kstar >= 0) return ds->kstar;  // settled in stage 1
+  // Stage 3: the first bin at which the cumulative energy reaches the threshold, if it does so clearly
   if (threadIdx.x == 0) {
     const int Kb = n / 2;
-    const double F0 = ds->tot[0], FN = ds->tot[2];
-    // Parseval over the bins 0 .. floor(n/2) of a real sequence
-    const double total = 0.5 * (static_cast<double>(n) * ds->tot[1] + F0 * F0 + ((n & 1) ? 0.0 : FN * FN));
+    const double thr = ds->tot[1], margin = ds->tot[2];
     int ks = -1;
-    if (smooth_mode == AUDIOKV_SMOOTH_FIXED_FRACTION) {
-      ks = static_cast<int>(floor(static_cast<double>(kappa) * Kb));
-    } else {
-      const bool no_mean = smooth_mode == AUDIOKV_SMOOTH_ENERGY_NO_MEAN;
-      const double rest = fmax(total - F0 * F0, 0.0), whole = no_mean ? rest : total;
-      const double thr = static_cast<double>(rho) * whole;
-      // The rotations are good to about 1e-6, so a bin's energy is off by up to 2e-6 |F_k| F_0: the decision is taken
-      // here only when it is clear of the threshold by several times the sum of that over the bins.
-      const double margin = 1e-5 * (whole + fabs(F0) * static_cast<double>(sqrtf(static_cast<float>(rest))));
-      double run = 0.0;
+    double run = 0.0;
 #pragma unroll 1
-      for (int k = 0; k < kDirectBins; ++k) {
-        const double before = run;
-        run += k == 0 ? (no_mean ? 0.0 : F0 * F0) : ds->energy[k];
-        if (run >= thr) {
-          if (run >= thr + margin && (k == 0 || before <= thr - margin) && whole > 0.0) ks = k;
-          break;
-        }
+    for (int k = 0; k < kDirectBins; ++k) {
+      const double before = run;
+      run += ds->energy[k];
+      if (run >= thr) {
+        if (run >= thr + margin && (k == 0 || before <= thr - margin)) ks = k;
+        break;
       }
     }
     if (ks < 0 || ks + T >= kDirectBins || ks + T >= Kb) ks = -1;
-    ds->kstar = ks;
+    ds->k_hi = ks;
   }
   __syncthreads();
-  return ds->kstar;
+  return ds->k_hi;
 }
 
 // The residual mix of every token from the masked bins c_k = mask_k F_k (1 up to k*, raised cosine over the T bins
