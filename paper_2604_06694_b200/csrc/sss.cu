@@ -371,8 +371,8 @@ __device__ __noinline__ void pass_odd(SkewBuf buf, int N, int ns, const float2* 
 // its (at most kPrimeTasks) tasks in registers until every task of the round has read its inputs.
 // The pass twiddles are applied in a sweep of their own (inverse: before, forward: with the
 // write-back).
-constexpr int kPrimeTasks = 2;  // tasks per thread and round
-constexpr int kPrimeOut = 4;    // consecutive c per task: the folded inputs P_s, Q_s are formed once for all of them
+constexpr int kPrimeTasks = 1;  // tasks per thread and round (two were tried: the second slot is mostly empty and costs registers)
+constexpr int kPrimeOut = 5;    // consecutive c per task: the folded inputs P_s, Q_s are formed once for all of them
 
 template <bool INV>
 __device__ __noinline__ void pass_prime(SkewBuf buf, int N, int ns, int p, const float2* tw,
