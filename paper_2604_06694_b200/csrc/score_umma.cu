@@ -425,11 +425,11 @@ __device__ __forceinline__ void stats_step(uint32_t (&ra)[32], uint32_t (&rb)[32
     Z = fmaf(Z, ex2(m_ref - m_new), hsum(a0, a1, a2, a3));
     m_ref = m_new;
   } else {
-    Z += hsum(a0, a1, a2, a3);
-    if (d > 0.f) {  // keep the reference at or above the running maximum: later columns then stay in range
-      Z *= ex2(-d);
-      m_ref += d;
-    }
+    // keep the reference at or above the running maximum, so that later columns stay in range; without a branch
+    // (d = -inf when the columns are all masked: no change)
+    const float dd = fmaxf(d, 0.f);
+    Z = (Z + hsum(a0, a1, a2, a3)) * ex2(-dd);
+    m_ref += dd;
   }
 }
 // Sweep 2: N logits of this thread's key against N query rows; nc = their -(max + log2 sum), 16-byte aligned.
