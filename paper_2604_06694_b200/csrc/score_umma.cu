@@ -40,12 +40,14 @@ namespace akv {
 namespace {
 
 constexpr int kTileKeys = 128;    // keys per K tile (UMMA M in sweep 2, N in sweep 1)
-// Epilogue warps: two groups of one or two sets of four warps (one warp per TMEM lane quarter). Sweep 1 runs two sets
-// per group, which split the key columns of every part (measured: 92 us against 104 with one set; its maxima leave
-// the special-function unit idle often enough for a second pair of warps per scheduler to pay); sweep 2 runs one set
-// (88 us against 91: with one set a thread keeps all the registers it wants and part of the exponentials goes to the FMA
-// pipe). After the epilogue warps come the producer warp and the two MMA warps.
-constexpr int epi_sets(int sweep) { return sweep == 1 ? 2 : 1; }
+// Epilogue warps: two groups of kSets sets of four warps (one warp per TMEM lane quarter); the sets of a group split
+// the columns of every part. Both sweeps run two sets (four epilogue warps per scheduler, 96 registers per thread).
+// Sweep 1: 92 us against 104 with one set (its maxima leave the special-function unit idle often enough for a second
+// pair of warps per scheduler to pay). Sweep 2 ran one set with 168 registers and 64-column steps for a long time
+// (85 us; two sets on the same steps 90: no registers left to schedule with); two sets on 32-column steps, with the
+// same share of the exponentials on the FMA pipe, take 80 us. After the epilogue warps come the producer warp and
+// the two MMA warps.
+constexpr int epi_sets(int sweep) { return 2; }
 constexpr int epi_warps(int sweep) { return 8 * epi_sets(sweep); }
 constexpr int n_threads(int sweep) { return (epi_warps(sweep) + 3) * 32; }
 constexpr int kStatSets = 2 * epi_sets(1);  // statistics entries sweep 1 writes per part: [group][set]
@@ -79,7 +81,7 @@ struct UmmaArgs {
   int n_stages;   // K ring depth
   int r0;         // first request of this launch: request r uses maps q[r - r0], k[r - r0]
   int w_chunk;    // window rows of a run's Q tile (the whole window, or a share of it when W * G exceeds the tile)
-  int accumulate; // sweep 2: the head is scored in several chunks of window rows, whose column sums add up in `scores`
+  int accumulate; // sweep 2 adds into `scores` (cleared by sweep 1): two warp sets per key, or several chunks of window rows
   int beside;     // sweep 1 runs beside the kernel launched before it (see launch_score_umma) and waits for it at its end
   long long wait_cycles;  // limit of a wait on an mbarrier, in SM clock cycles
 };
@@ -464,47 +466,36 @@ __device__ __forceinline__ void colsum_part(const uint32_t (&r)[32], const float
   }
 }
 
-// Sweep 2, one part of COLS accumulator columns (a multiple of 16, at most 128) for this thread's key: the same
-// steps as the general loop below (64 columns in two register buffers, the buffer handed back once the last step
-// is in registers), with the shape known at compile time: no branch on the number of chunks or on a half-filled
-// last buffer, and the arithmetic of a step is one basic block for the scheduler. (Sweep 2 runs two epilogue warps
-// per scheduler; with the general loop a tenth of their time went to resolving those branches.)
-template <int COLS>
-__device__ __forceinline__ void colsum_cols(uint32_t taddr, const float* __restrict__ ncp, f32x2 sl2, uint32_t ebar, int lane,
-                                            uint32_t (&ra)[32], uint32_t (&rb)[32], f32x2& a0, f32x2& a1, f32x2& a2,
-                                            f32x2& a3) {
+// Sweep 2, set SET of two: the chunks 2 SET and 2 SET + 1 of a part of COLS accumulator columns (a multiple of 16, at
+// most 128) for this thread's key, one 32-column buffer at a time; the shape is known at compile time, so the tile
+// loop has no branch on chunk counts or on a half-filled last buffer. The part's buffer is handed back to the MMA
+// thread once this set's last chunk is in registers (at once when the set has no chunk in the part).
+template <int COLS, int SET>
+__device__ __forceinline__ void colsum_cols_set(uint32_t taddr, const float* __restrict__ ncp, f32x2 sl2, uint32_t ebar, int lane,
+                                                uint32_t (&ra)[32], f32x2& a0, f32x2& a1, f32x2& a2, f32x2& a3) {
   constexpr int n_ch = (COLS + 31) / 32;
   constexpr bool tail = (COLS & 16) != 0;
+  constexpr int c_lo = 2 * SET, c_hi = c_lo + 2 < n_ch ? c_lo + 2 : n_ch;  // chunks [c_lo, c_hi)
+  if (c_lo >= n_ch) {
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(ebar);
+    return;
+  }
 #pragma unroll
-  for (int st = 0; st < 2; ++st) {
-    const int c0 = 2 * st;
-    if (c0 < n_ch) {
-      const bool has_b = c0 + 1 < n_ch;
-      const bool a_half = tail && c0 == n_ch - 1, b_half = tail && c0 + 1 == n_ch - 1;
-      if (a_half) tmem_ld16_issue_lo(taddr + c0 * 32, ra);
-      else tmem_ld32_issue(taddr + c0 * 32, ra);
-      if (has_b) {
-        if (b_half) tmem_ld16_issue_lo(taddr + (c0 + 1) * 32, rb);
-        else tmem_ld32_issue(taddr + (c0 + 1) * 32, rb);
-      }
-      if (a_half) tmem_wait_lo(ra);
-      else tmem_wait(ra);
-      if (has_b) {
-        if (b_half) tmem_wait_lo(rb);
-        else tmem_wait(rb);
-      }
-      if (c0 + 2 >= n_ch) {  // the part is in registers: its buffer goes back to the MMA thread
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(ebar);
-      }
-      if (a_half) colsum_part<16>(ra, ncp + c0 * 32, sl2, a0, a1, a2, a3);
-      else colsum_part<32>(ra, ncp + c0 * 32, sl2, a0, a1, a2, a3);
-      if (has_b) {
-        if (b_half) colsum_part<16>(rb, ncp + (c0 + 1) * 32, sl2, a0, a1, a2, a3);
-        else colsum_part<32>(rb, ncp + (c0 + 1) * 32, sl2, a0, a1, a2, a3);
-      }
+  for (int c = c_lo; c < c_hi; ++c) {
+    const bool half = tail && c == n_ch - 1;
+    if (half) tmem_ld16_issue_lo(taddr + c * 32, ra);
+    else tmem_ld32_issue(taddr + c * 32, ra);
+    if (half) tmem_wait_lo(ra);
+    else tmem_wait(ra);
+    if (c == c_hi - 1) {
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(ebar);
     }
+    if (half) colsum_part<16>(ra, ncp + c * 32, sl2, a0, a1, a2, a3);
+    else colsum_part<32>(ra, ncp + c * 32, sl2, a0, a1, a2, a3);
   }
 }
 
@@ -775,8 +766,9 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
       }
       prev_u = U.qid;
       if (SWEEP == 1 && a.accumulate && U.w0 == 0) {
-        // a head scored in several chunks of window rows: sweep 2 adds each chunk's column sums into the score buffer,
-        // so the first chunk's run clears the entries of its keys (sweep 2 starts after this kernel has ended)
+        // Sweep 2 adds a key's column sums into the score buffer from several places (its two warp sets; the chunks
+        // of a window scored in chunks), so the run of the first chunk clears the entries of its keys (sweep 2's
+        // epilogue starts after this kernel has ended)
         const int k_end = U.kt0 + U.n_tiles * kTileKeys < U.P ? U.kt0 + U.n_tiles * kTileKeys : U.P;
         for (int key = U.kt0 + static_cast<int>(threadIdx.x); key < k_end; key += kEpiWarps * 32)
           a.scores[U.score_base + key] = 0.f;
@@ -812,14 +804,18 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
           const bool masked = kt + kTileKeys - 1 > U.P;       // sweep 1: the tile reaches into the window: causal mask
           const int last_col = U.P + U.w0 + row / G - kt;     // sweep 1: last visible key of this row, relative to the tile
           const float* ncp = SWEEP == 2 ? nc + (p == 0 ? 0 : cols0) : nullptr;
-          if (kSets == 2 && 2 * set >= n_ch) {  // this set has no columns in the part
+          if (SWEEP == 1 && kSets == 2 && 2 * set >= n_ch) {  // this set has no columns in the part (never: a part of sweep 1 is 128 columns)
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(ebar);
           }
-          if constexpr (SWEEP == 2 && kSets == 1) {
+          if constexpr (SWEEP == 2 && kSets == 2) {
             switch (cols) {  // the shapes of a launch: one or two of these
-#define AKV_COLS_CASE(C) case C: colsum_cols<C>(taddr, ncp, sl2, ebar, lane, ra, rb, a0, a1, a2, a3); break;
+#define AKV_COLS_CASE(C)                                                                          \
+  case C:                                                                                         \
+    if (set == 0) colsum_cols_set<C, 0>(taddr, ncp, sl2, ebar, lane, ra, a0, a1, a2, a3);         \
+    else colsum_cols_set<C, 1>(taddr, ncp, sl2, ebar, lane, ra, a0, a1, a2, a3);                  \
+    break;
               AKV_COLS_CASE(16) AKV_COLS_CASE(32) AKV_COLS_CASE(48) AKV_COLS_CASE(64)
               AKV_COLS_CASE(80) AKV_COLS_CASE(96) AKV_COLS_CASE(112) AKV_COLS_CASE(128)
 #undef AKV_COLS_CASE
@@ -868,10 +864,13 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
         }
         if (!ok) break;
         if (SWEEP == 2) {
+          // The sets of a group (and the chunks of a window scored in several chunks) hold sums over different rows
+          // of the same key: each adds its own into the score buffer, which sweep 1 cleared. With two addends the
+          // result does not depend on their order.
           const int key = kt + gl;
           if (key < U.P) {
             const float sum = hsum(a0, a1, a2, a3);
-            if (a.accumulate) atomicAdd(a.scores + U.score_base + key, sum);  // the buffer was cleared by sweep 1
+            if (a.accumulate) atomicAdd(a.scores + U.score_base + key, sum);
             else a.scores[U.score_base + key] = sum;
           }
         }
@@ -1020,7 +1019,7 @@ cudaError_t launch_score_umma_cap(const Shape& sh, const ReqDesc* h_reqs, const 
   args.q_rows = R > 128 ? 256 : 128;
   args.r_pad = (R + 15) / 16 * 16;
   args.w_chunk = w_chunk;
-  args.accumulate = w_chunk < sh.window ? 1 : 0;
+  args.accumulate = (w_chunk < sh.window || epi_sets(2) > 1) ? 1 : 0;
   args.beside = beside ? 1 : 0;
   args.wait_cycles = score_wait_cycles();
   const int q_bytes = args.q_rows * d * 2, stage = kTileKeys * d * 2;
