@@ -810,10 +810,12 @@ score_umma_kernel(const __grid_constant__ TmapPack<CAP> tm, const UmmaArgs a) {
             if (lane == 0) mbar_arrive(ebar);
           }
           if constexpr (SWEEP == 2 && kSets == 2) {
+            // the sets take the leading and the trailing chunks of the two parts of a tile in turn: with 112 columns a
+            // part that is 64 against 48 columns, and evens out over the tile
             switch (cols) {  // the shapes of a launch: one or two of these
 #define AKV_COLS_CASE(C)                                                                          \
   case C:                                                                                         \
-    if (set == 0) colsum_cols_set<C, 0>(taddr, ncp, sl2, ebar, lane, ra, a0, a1, a2, a3);         \
+    if ((set ^ p) == 0) colsum_cols_set<C, 0>(taddr, ncp, sl2, ebar, lane, ra, a0, a1, a2, a3);   \
     else colsum_cols_set<C, 1>(taddr, ncp, sl2, ebar, lane, ra, a0, a1, a2, a3);                  \
     break;
               AKV_COLS_CASE(16) AKV_COLS_CASE(32) AKV_COLS_CASE(48) AKV_COLS_CASE(64)
