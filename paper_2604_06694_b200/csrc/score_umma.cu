@@ -8,17 +8,18 @@
 //            the keys of its tiles; one pair per (head, part, group, row) goes to the
 //            statistics buffer.
 //   sweep 2  D[key][row]  = K Q^T  (keys on the TMEM lanes): every thread owns one key
-//            and adds exp2(z - max - log2 sum) over all rows; no cross-thread reduction.
+//            and adds exp2(z - max - log2 sum) over its set's rows; the two sets' sums of a key meet in the score
+//            buffer (atomic adds into a buffer that sweep 1 cleared).
 // Both sweeps are one persistent kernel with three roles:
-//   warps 0-7  two epilogue groups of four warps (one warp per TMEM lane quarter). The groups take the
-//              tiles of the CTA in turn (group g the tiles with parity g), each through accumulator
-//              buffers of its own, so that they depend on nothing but the MMA thread: no barrier
-//              joins them, nothing is exchanged through shared memory, and while one group waits,
-//              loads or stores, the other keeps the special-function unit busy;
-//   warp 8     TMA producer: the Q tile of a head once, K tiles of 128 keys through a ring;
-//   warps 9-10 MMA issuers, one thread per epilogue group: tcgen05.mma, bf16 x bf16 -> fp32 in TMEM. With one issuer
-//              for both groups the tiles were issued in order, and a group that had handed its buffers back waited
-//              for the MMAs of the other group's tile to be let in first.
+//   warps 0-15  two epilogue groups of two sets of four warps (one warp per TMEM lane quarter and set). The groups
+//               take the tiles of the CTA in turn (group g the tiles with parity g), each through accumulator
+//               buffers of its own, so that they depend on nothing but their MMA thread: no barrier joins them,
+//               nothing is exchanged through shared memory, and while one group waits, loads or stores, the other
+//               keeps the special-function unit busy. The two sets of a group split the columns of every part;
+//   warp 16     TMA producer: the Q tile of a head once, K tiles of 128 keys through a ring;
+//   warps 17-18 MMA issuers, one thread per epilogue group: tcgen05.mma, bf16 x bf16 -> fp32 in TMEM. With one issuer
+//               for both groups the tiles were issued in order, and a group that had handed its buffers back waited
+//               for the MMAs of the other group's tile to be let in first.
 // A tile is processed in one or two parts (sweep 1: blocks of 128 query rows; sweep 2: halves of
 // the query rows), each with an accumulator buffer of 128 TMEM columns that goes back to the MMA
 // thread as soon as its last chunk is in registers: the MMAs of the group's next tile run under
