@@ -338,11 +338,11 @@ __device__ __forceinline__ f32x2 ex2_poly(f32x2 x, f32x2 t) {
   asm("mov.b64 {%0, %1}, %2;" : "=r"(pl), "=r"(ph) : "l"(p));
   return pack2(pl + (tl << 23), ph + (th << 23));
 }
-// Of every eight pairs of exponentials, this many go to the FMA pipe. Measured on the epilogue arithmetic alone, two
-// warps per scheduler: the column sums of sweep 2 take 2314 cycles per 128 columns with none, 1955 with two, 2052 with
-// three; the row statistics of sweep 1, whose maxima already load the other pipes, 2399, 2481 and 3025: none there.
+// Of every eight pairs of exponentials, this many go to the FMA pipe. In the kernel as it stands (four epilogue warps
+// per scheduler in both sweeps): sweep 2 takes 87.2 us with none, 80.9 with one, 79.9 with two, 83.8 with three;
+// sweep 1, once its per-step maxima were gone, 86.6 with none, 84.8 with one, 85.5 with two, 88.4 with three.
 #ifndef AKV_POLY_S1
-#define AKV_POLY_S1 0
+#define AKV_POLY_S1 1
 #endif
 #ifndef AKV_POLY_S2
 #define AKV_POLY_S2 2
@@ -397,10 +397,13 @@ __device__ __forceinline__ float ceil_octave(float x) { return __fadd_ru(x, kMag
 
 // Sweep 1: 64 logits of this thread's row (columns col0 .. col0 + 63 of the tile, in two buffers). Updates the row's
 // reference m_ref (a whole number of octaves, so that changing it rescales the sum exactly) and its sum Z of exp2
-// relative to that reference. The exponentials are taken against the reference the row had BEFORE these columns
-// and the maximum of the columns is found beside them, not before them: a reference up to 60 octaves below the
-// maximum loses nothing in fp32, so only the first columns of a run, or a jump of more than 60 octaves, have to
-// wait for their maximum (and then take the exponentials once more).
+// relative to that reference. The exponentials are taken against the reference the row had BEFORE these columns:
+// a reference tens of octaves away from the maximum loses nothing in fp32, so only the first columns of a run
+// look for their maximum first, and only a sum of 2^60 or more (a jump of the maximum by about that much, or an
+// overflow) has the exponentials taken once more. Afterwards the reference is raised by what the SUM of the columns
+// says (it bounds their maximum from above), which needs no maximum over the columns: measured, the 22 three-input
+// maxima per step kept the ALU pipe from taking a share of the exponentials (with them, a polynomial share made
+// the sweep slower; without them, one pair in eight on the FMA pipe brings 87.6 -> 84.8 us).
 __device__ __forceinline__ void stats_step(uint32_t (&ra)[32], uint32_t (&rb)[32], bool masked, int col0, int last_col,
                                            float sl, float inv_sl, float& m_ref, float& Z) {
   if (masked) {
@@ -418,21 +421,23 @@ __device__ __forceinline__ void stats_step(uint32_t (&ra)[32], uint32_t (&rb)[32
   f32x2 a0 = pack2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
   exp_sum32(ra, sl, inv_sl, m_ref, a0, a1, a2, a3);
   exp_sum32(rb, sl, inv_sl, m_ref, a0, a1, a2, a3);
-  const float cm = fmaxf(max32(ra), max32(rb));
-  const float d = ceil_octave(cm * sl) - m_ref;  // -inf when the columns are all masked
-  if (d > 60.f) {
-    const float m_new = m_ref + d;
+  const float s = hsum(a0, a1, a2, a3);  // these columns' sum relative to m_ref: at least their largest term
+  if (!(s < 0x1p60f)) {
+    // a jump of the maximum by tens of octaves (or an overflow): take the exponentials again, against the maximum
+    const float cm = fmaxf(max32(ra), max32(rb));
+    const float m_new = ceil_octave(cm * sl);
     a0 = a1 = a2 = a3 = pack2(0.f, 0.f);
     exp_sum32(ra, sl, inv_sl, m_new, a0, a1, a2, a3);
     exp_sum32(rb, sl, inv_sl, m_new, a0, a1, a2, a3);
     Z = fmaf(Z, ex2(m_ref - m_new), hsum(a0, a1, a2, a3));
     m_ref = m_new;
   } else {
-    // keep the reference at or above the running maximum, so that later columns stay in range; without a branch
-    // (d = -inf when the columns are all masked: no change)
-    const float dd = fmaxf(d, 0.f);
-    Z = (Z + hsum(a0, a1, a2, a3)) * ex2(-dd);
-    m_ref += dd;
+    // Keep the reference above what was seen, so that later columns stay in range: when the sum reaches 1 the
+    // reference goes up by the sum's binary exponent + 1 (a whole number of octaves: the rescaling is exact and is
+    // built from bits, no special function). The sum bounds the maximum from above, so no maximum is needed.
+    const int e = s >= 1.f ? (__float_as_int(s) >> 23) - 126 : 0;            // 0 <= e <= 60
+    Z = (Z + s) * __int_as_float((127 - e) << 23);                            // * 2^-e
+    m_ref += __int_as_float(0x4b000000 | e) - 8388608.f;                      // + e
   }
 }
 // Sweep 2: N logits of this thread's key against N query rows; nc = their -(max + log2 sum), 16-byte aligned.
