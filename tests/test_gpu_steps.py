@@ -68,6 +68,42 @@ def test_score_parity(B, name, make):
     assert ctx.last_device_status() == 0
 
 
+def test_score_reference_jumps(B):
+    """Rows whose logits jump by far more than 60 octaves in the middle of the keys, twice: every window query is the
+    same vector v, and two keys far into the cache are multiples of v (4 v after 3 tiles, 9 v after 9 more), so
+    their logits stand 50 and 110 nats (70 and 160 octaves) above everything before them. The running row sums of the
+    first sweep must follow such jumps (the exponentials are then taken again against the new maximum), and the two
+    keys end up with nearly all of the probability."""
+    w = wl.generate(_small_spec("bf16", 8, 2, 128, (2048 + 64,), 32))
+    d = 128
+    bits = lambda x: torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).view(torch.uint16).numpy()
+    v = np.ones(d, dtype=np.float32)
+    v[1::2] = -1.0
+    w.q[...] = bits(v)                                  # every window row and query head
+    k32 = w.as_torch(w.k).to(torch.float32).numpy() * 0.05
+    k32[:, :, 400, :] = 4.0 * v                         # logit 4 * 128 / sqrt(128) = 45 nats above the small keys
+    k32[:, :, 1500, :] = 9.0 * v                        # and 57 nats above that one
+    w.k[...] = bits(k32)
+    prob = B.Problem.from_workload(w)
+    ctx = B.Context(prob)
+    q, k = to_dev(w, w.q), to_dev(w, w.k)
+    scores = torch.full((B.audiokv_scores_len(prob),), float("nan"), device="cuda")
+    B.audiokv_score(ctx, prob, q, k, scores)
+    torch.cuda.synchronize()
+    assert ctx.last_score_path() == "tcgen05" and ctx.last_device_status() == 0
+    g = scores.cpu().numpy()
+    assert np.isfinite(g).all()
+    o, wm = oracle_scores(w, 0)
+    s = w.spec
+    P = s.seq_lens[0] - s.window
+    G = s.n_q_heads // s.n_kv_heads
+    gr = g.reshape(o.shape)
+    for h in range(s.n_kv_heads):
+        assert rel_err(gr[0, h], o[0, h]) <= REL_TOL, h
+        assert abs(gr[0, h, 1500] - s.window * G) <= 1e-3 * s.window * G     # the last jump takes everything
+        assert gr[0, h, 400] < 1e-20 and gr[0, h, :400].max() < 1e-30
+
+
 # The long lengths, one layer each: 256 key tiles per head at L = 32768 (G = 7, so 224 query rows per head, and
 # W = 64 with 448), a d = 256 head at L = 19224 (the longest request of the ragged batch), and L = 131072.
 LONG_SCORE_CASES = [
